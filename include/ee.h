@@ -1,0 +1,211 @@
+/*
+ * ee.h - C ABI of the early-exit CNN stage executor for NVIDIA B200 (sm_100a).
+ *
+ * The library runs an early-exit CNN one subnet ("stage") at a time on a batch whose size
+ * changes at every exit: a stage's convolutions, its exit head, the threshold test, the
+ * compaction of the samples that stay, and the refill of the batch with new samples before
+ * the next stage.  This is the device-side work underneath the serving loop of the paper
+ * "Fluid Batching" (Section III overview, steps 2-6; Section III-B; Algorithm 1): the
+ * scheduler there calls "process until exit i", learns B_exit, and merges the remaining
+ * B_rem samples with B_incr new ones.
+ *
+ * General rules
+ *   - Plain C.  Every function returns an ee_status_t; results only through pointers.
+ *     On an error return no output buffer has been written.
+ *   - "DEVICE" pointers are CUDA device memory of the current device; "HOST" pointers are
+ *     ordinary host memory unless stated to be pinned.  The library never frees or keeps a
+ *     caller buffer beyond the call, except the stream-ordered use described per function.
+ *   - All work is enqueued on the cuda_stream argument (a cudaStream_t passed as void*;
+ *     NULL = the legacy default stream) and is asynchronous with respect to the host unless
+ *     stated otherwise.  One stream per model handle at a time.
+ *   - Activations are NHWC [B][H][W][C] in the model's dtype (float or bf16).  Convolution
+ *     weights are [Cout][kh][kw][Cin/groups], FC weights [n_classes][C], same dtype.
+ *     A convolution is executed as the product of the implicit Toeplitz matrix
+ *     (M = B*Ho*Wo rows, K = kh*kw*Cin) with the K x Cout weight matrix (Section II-C);
+ *     batching appends samples along the row dimension (Section III-A, R-batching).
+ *   - Buffers are sized once for max_batch by the caller (Section III-B, Overhead: buffers are
+ *     allocated at initialisation for the largest activation at B_max; no run-time allocation).
+ *     No entry point below allocates device memory except ee_model_create.
+ */
+#ifndef EE_H_
+#define EE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  EE_OK = 0,
+  EE_ERR_INVALID_ARG = 1,  /* NULL where a pointer is required, negative size, bad enum   */
+  EE_ERR_SHAPE = 2,        /* layer list does not chain (channel or spatial mismatch)      */
+  EE_ERR_CAPACITY = 3,     /* batch > max_batch, workspace too small                       */
+  EE_ERR_STAGE = 4,        /* stage / boundary index out of range                          */
+  EE_ERR_UNSUPPORTED = 5,  /* geometry no kernel covers; only ever returned at create time */
+  EE_ERR_CUDA = 6,         /* a CUDA runtime/driver call failed (see ee_last_cuda_error)   */
+  EE_ERR_TIMEOUT = 7,      /* a bounded device-side wait ran out (reported by ee_model_check) */
+  EE_ERR_INTERNAL = 8
+} ee_status_t;
+
+typedef enum { EE_F32 = 0, EE_BF16 = 1 } ee_dtype_t;
+typedef enum { EE_OP_CONV = 0, EE_OP_DWCONV = 1, EE_OP_MAXPOOL = 2 } ee_op_t;
+typedef enum { EE_ACT_NONE = 0, EE_ACT_RELU = 1, EE_ACT_RELU6 = 2 } ee_act_t;
+
+/* Sources for ee_layer_desc_t.input_from / residual_from. */
+#define EE_FROM_PREV (-1)         /* input_from: output of the previous layer (stage input for layer 0) */
+#define EE_FROM_STAGE_INPUT (-2)  /* the stage's input tensor */
+#define EE_NO_RESIDUAL (-1)       /* residual_from: no residual operand */
+
+/* One layer of a stage.  y = act(scale[c] * conv(x, weight) + bias[c] (+ residual)), stored in
+ * the model dtype with one round-to-nearest-even.  BN is folded into scale/bias by the caller.
+ * EE_OP_DWCONV is a depthwise convolution (groups = cin = cout, weight [C][kh][kw][1]).
+ * EE_OP_MAXPOOL takes the window maximum over in-range taps; weight/scale/bias are ignored. */
+typedef struct {
+  int op;             /* ee_op_t */
+  int cin, cout, kh, kw, stride, pad;
+  int act;            /* ee_act_t */
+  int input_from;     /* EE_FROM_PREV, EE_FROM_STAGE_INPUT, or index of an earlier layer of this stage */
+  int residual_from;  /* EE_NO_RESIDUAL, EE_FROM_STAGE_INPUT, or index of an earlier layer; same shape as y */
+  const void* weight; /* HOST or DEVICE (see ee_model_desc_t.weights_on_device); copied at create */
+  const float* scale; /* [cout] fp32, may be NULL (= 1) */
+  const float* bias;  /* [cout] fp32, may be NULL (= 0) */
+} ee_layer_desc_t;
+
+/* One stage = a subnet followed by its exit head (global average pool, one FC layer, softmax;
+ * the largest softmax probability is the confidence: Section II-B; Section IV, Benchmarks).
+ * A sample exits iff always_exit or confidence >= threshold (compared in fp32). */
+typedef struct {
+  int n_layers;
+  const ee_layer_desc_t* layers;
+  int out_layer;          /* layer whose output leaves the stage; -1 = last */
+  int n_classes;
+  const void* fc_weight;  /* [n_classes][C] model dtype */
+  const float* fc_bias;   /* [n_classes] fp32, may be NULL */
+  float threshold;
+  int always_exit;        /* 1 for the final exit */
+} ee_stage_desc_t;
+
+typedef struct {
+  int dtype;              /* ee_dtype_t: EE_F32 computes in fp32 FMA; EE_BF16 stores bf16, accumulates fp32 */
+  int in_h, in_w, in_c;
+  int n_stages;
+  const ee_stage_desc_t* stages;
+  int max_batch;          /* B_max */
+  int weights_on_device;  /* 0: all weight/scale/bias pointers are HOST; 1: DEVICE */
+} ee_model_desc_t;
+
+typedef struct ee_model ee_model_t; /* opaque; owns its device copies of the weights */
+
+typedef struct {
+  int in_h, in_w, in_c, out_h, out_w, out_c;
+  size_t in_bytes_per_sample, out_bytes_per_sample;
+  size_t workspace_bytes; /* what ee_stage_run needs for this stage at max_batch */
+  int n_layers;
+  double flops_per_sample; /* 2*M*N*K summed over the stage's convolutions, for roofline reports */
+} ee_stage_info_t;
+
+/* Validates the description, copies and repacks the weights to the device, and plans each
+ * layer's kernel.  Synchronous (returns after the uploads finished).  *out is set only on EE_OK.
+ * Errors: INVALID_ARG, SHAPE (layers do not chain), UNSUPPORTED, CUDA. */
+ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_model_t** out);
+
+/* Frees everything the model owns.  The caller must have synchronised the streams it used. */
+ee_status_t ee_model_destroy(ee_model_t* model);
+
+/* Shapes and sizes of one stage.  Errors: INVALID_ARG, STAGE. */
+ee_status_t ee_model_query(const ee_model_t* model, int stage, ee_stage_info_t* out);
+
+/* Inputs of ee_stage_run.  All pointers DEVICE. */
+typedef struct {
+  const void* features;        /* [batch][in_h][in_w][in_c], model dtype */
+  const int32_t* ids;          /* [batch] sample ids (samples finish out of order and are re-associated by id:
+                                  Section III-B, Overhead); may be NULL */
+  int batch;                   /* B_act, 0 <= batch <= max_batch */
+  const float* logit_shift;    /* optional [batch]: added to logit shift_class[b] of sample b before the softmax */
+  const int32_t* shift_class;  /* [batch], required iff logit_shift != NULL; entries outside [0, n_classes) are ignored */
+} ee_stage_in_t;
+
+/* Outputs of ee_stage_run.  Caller-owned DEVICE buffers sized for max_batch (any may be NULL
+ * except features_out, exit_mask, survivor_idx and n_surv_dev). */
+typedef struct {
+  void* features_out;     /* [n_surv][out_h][out_w][out_c]: the survivors' stage output, compacted, order kept;
+                             this is the next stage's input */
+  float* conf;            /* [batch] softmax top-1 probability, input order */
+  int32_t* pred;          /* [batch] argmax class (lowest index on ties), input order */
+  float* logits;          /* [batch][n_classes] fp32, optional */
+  uint8_t* exit_mask;     /* [batch] 1 = sample exits here */
+  int32_t* survivor_idx;  /* first n_surv entries: ascending positions (in the input batch) of the survivors */
+  int32_t* ids_out;       /* first n_surv entries: ids of the survivors (written iff ids given) */
+  int32_t* n_surv_dev;    /* [1] B_rem = B_act - B_exit */
+  int32_t* n_surv_host;   /* optional PINNED HOST [1]: receives the count by an async copy on the stream; valid once the
+                             caller has synchronised the stream (the "B_exit is communicated to the scheduler" step) */
+} ee_stage_out_t;
+
+/* Runs stage `stage` on a batch: every layer of the subnet (convolutions as implicit GEMM with the
+ * bias/BN-fold/activation epilogue fused), the exit head, the threshold test, and the stable
+ * compaction + gather of the survivors (Section III, steps 2-4; Algorithm 1 "ProcUntilExit" and
+ * B_rem = B_act - B_exit).  `workspace` is DEVICE scratch of at least ee_stage_info_t.workspace_bytes,
+ * 256-byte aligned; its contents are undefined afterwards.  features_out must not alias `features`
+ * or the workspace.  batch == 0 is legal: only n_surv = 0 is written.
+ * Errors: INVALID_ARG, STAGE, CAPACITY (batch > max_batch or workspace too small), CUDA. */
+ee_status_t ee_stage_run(ee_model_t* model, int stage, const ee_stage_in_t* in, void* workspace,
+                         size_t workspace_bytes, const ee_stage_out_t* out, void* cuda_stream);
+
+/* Merges a halted batch with new samples that stand at the same stage boundary
+ * (Section III-B, Preemption Mechanism; Algorithm 1: B_slack = B_max - B_rem,
+ * B_incr = min(N_Q, B_slack), B_merged = B_rem + B_incr).  `boundary` 0 = model input,
+ * i = output of stage i-1.  batch_feat / batch_ids (DEVICE, sized for max_batch) hold n_surv samples at
+ * the front; the first n_accepted = min(n_arr, max_batch - n_surv) arrivals (DEVICE arr_feat / arr_ids) are
+ * appended after them in order.  n_accepted and n_merged are HOST ints written before return; arrivals
+ * that did not fit stay with the caller.  ids may be NULL on both sides.
+ * Errors: INVALID_ARG, STAGE, CAPACITY (n_surv > max_batch), CUDA. */
+ee_status_t ee_batch_refill(ee_model_t* model, int boundary, void* batch_feat, int32_t* batch_ids, int n_surv,
+                            const void* arr_feat, const int32_t* arr_ids, int n_arr, int* n_accepted,
+                            int* n_merged, void* cuda_stream);
+
+/* Exit head alone on a feature map (same kernels ee_stage_run uses): GAP, FC, softmax top-1,
+ * threshold, and the stable scan that yields survivor_idx / n_surv (no feature gather).
+ * x DEVICE [batch][hw][c] model dtype; `out` as in ee_stage_run with features_out ignored;
+ * `scratch` DEVICE, at least ee_exit_head_scratch_bytes(model, stage) bytes, 256-byte aligned.
+ * Errors: INVALID_ARG, STAGE, CAPACITY, CUDA. */
+ee_status_t ee_exit_head(ee_model_t* model, int stage, const void* x, int batch, int hw,
+                         const float* logit_shift, const int32_t* shift_class, void* scratch, size_t scratch_bytes,
+                         const ee_stage_out_t* out, void* cuda_stream);
+size_t ee_exit_head_scratch_bytes(const ee_model_t* model, int stage);
+
+/* Stable compaction + gather alone: feat_out[j] = feat[survivor_idx[j]] for j < *n_surv_dev
+ * (both read from DEVICE memory, no host round trip).  Rows move as 16-byte vectors when bytes_per_sample
+ * and both base addresses are multiples of 16, in narrower units otherwise.
+ * Errors: INVALID_ARG, CUDA. */
+ee_status_t ee_gather_survivors(const void* feat, size_t bytes_per_sample, const int32_t* survivor_idx,
+                                const int32_t* n_surv_dev, int max_rows, void* feat_out, void* cuda_stream);
+
+/* Per-layer device timing.  When enabled, ee_stage_run brackets every kernel with CUDA events on the
+ * stream it launches on.  ee_model_get_timing synchronises those events and writes, for the last run
+ * of `stage`, up to `cap` entries: the layers in order, then the head and the gather kernels.
+ * names[i] points at a static string.  Errors: INVALID_ARG, STAGE, CUDA. */
+ee_status_t ee_model_set_timing(ee_model_t* model, int enabled);
+ee_status_t ee_model_get_timing(ee_model_t* model, int stage, int cap, float* ms, const char** names, int* n);
+
+/* Per-layer plan of a stage at a batch size: kernel family chosen, GEMM M/N/K, FLOPs and the
+ * algorithmic bytes (inputs + outputs + weights, each once).  Up to `cap` entries. */
+typedef struct {
+  const char* kernel;
+  int m, n, k;
+  double flops, bytes;
+} ee_layer_plan_t;
+ee_status_t ee_model_plan(const ee_model_t* model, int stage, int batch, int cap, ee_layer_plan_t* out, int* n);
+
+/* Synchronises the stream and reports device-side faults the kernels recorded instead of hanging:
+ * EE_ERR_TIMEOUT when a bounded wait on a barrier ran out.  The flag is cleared by the call. */
+ee_status_t ee_model_check(ee_model_t* model, void* cuda_stream);
+
+const char* ee_status_string(ee_status_t s);
+const char* ee_last_cuda_error(void); /* text of the last CUDA error seen by this thread, "" if none */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EE_H_ */

@@ -1,0 +1,628 @@
+// C ABI of the early-exit CNN stage executor: model creation (weight upload, per-layer kernel
+// plan, workspace layout), ee_stage_run, ee_batch_refill and the stand-alone head / gather calls.
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "conv_simt.cuh"
+#include "conv_tc.cuh"
+#include "head.cuh"
+
+using namespace ee;
+
+namespace {
+
+thread_local std::string g_cuda_err;
+
+#define EE_CUDA(expr)                                                                      \
+  do {                                                                                     \
+    cudaError_t e__ = (expr);                                                              \
+    if (e__ != cudaSuccess) {                                                              \
+      g_cuda_err = std::string(#expr) + ": " + cudaGetErrorString(e__);                    \
+      return EE_ERR_CUDA;                                                                  \
+    }                                                                                      \
+  } while (0)
+
+enum KernelKind { KK_SIMT = 0, KK_TC = 1, KK_DW = 2, KK_POOL = 3 };
+const char* kKernelNames[] = {"conv_igemm_simt", "conv_igemm_tcgen05", "dwconv", "maxpool"};
+
+struct LayerPlan {
+  ee_layer_desc_t d;
+  int in_h, in_w, out_h, out_w;
+  int src_slot;  // -1 = stage input
+  int res_slot;  // -2 = none, -1 = stage input
+  int out_slot;
+  KernelKind kind;
+  void* w_dev = nullptr;
+  float* scale_dev = nullptr;
+  float* bias_dev = nullptr;
+  TcLayer tc;  // tensor-core plan (valid iff kind == KK_TC)
+};
+
+struct StagePlan {
+  std::vector<LayerPlan> layers;
+  int in_h, in_w, in_c, out_h, out_w, out_c, out_slot;
+  std::vector<size_t> slot_off;  // byte offsets at max_batch
+  size_t head_off = 0, ws_bytes = 0, head_bytes = 0;
+  int n_classes = 0;
+  void* fc_w = nullptr;
+  float* fc_b = nullptr;
+  float threshold = 0.f;
+  int always_exit = 0;
+  double flops_per_sample = 0;
+  // timing of the last run
+  std::vector<cudaEvent_t> ev;
+  std::vector<const char*> ev_names;
+  int ev_used = 0;
+};
+
+size_t esize(int dtype) { return dtype == EE_BF16 ? 2 : 4; }
+
+// Rows of a sample's [HW][C] map summed by one CTA of the pooling kernel: a function of the
+// shape only (never of the batch), about 32 KB of input per CTA.
+int gap_rows_per_chunk(int hw, int c, size_t es) {
+  long rows = (32 * 1024) / ((long)c * (long)es);
+  if (rows < 1) rows = 1;
+  if (rows > hw) rows = hw;
+  return (int)rows;
+}
+
+struct HeadLayout {
+  int rows_per_chunk, nchunks;
+  size_t off_partial, off_gap, off_z, off_cnt, bytes;
+};
+
+HeadLayout head_layout(int max_batch, int hw, int c, int k, size_t es) {
+  HeadLayout h;
+  h.rows_per_chunk = gap_rows_per_chunk(hw, c, es);
+  h.nchunks = cdiv(hw, h.rows_per_chunk);
+  size_t o = 0;
+  h.off_cnt = o;
+  o = align_up(o + sizeof(unsigned) * (size_t)max_batch, 256);
+  h.off_partial = o;
+  o = align_up(o + sizeof(float) * (size_t)max_batch * h.nchunks * c, 256);
+  h.off_gap = o;
+  o = align_up(o + sizeof(float) * (size_t)max_batch * c, 256);
+  h.off_z = o;
+  o = align_up(o + sizeof(float) * (size_t)max_batch * k, 256);
+  h.bytes = o;
+  return h;
+}
+
+}  // namespace
+
+struct ee_model {
+  int dtype, in_h, in_w, in_c, max_batch;
+  std::vector<StagePlan> stages;
+  std::vector<void*> owned;  // device allocations
+  int* err_flag = nullptr;   // device word set by kernels whose bounded waits ran out
+  bool timing = false;
+  TcContext tc;
+};
+
+namespace {
+
+template <typename T>
+ee_status_t upload(ee_model* m, const T* src, size_t n, int on_device, cudaStream_t st, T** out) {
+  *out = nullptr;
+  if (!src || n == 0) return EE_OK;
+  void* p = nullptr;
+  EE_CUDA(cudaMalloc(&p, align_up(n * sizeof(T), 256)));
+  m->owned.push_back(p);
+  EE_CUDA(cudaMemcpyAsync(p, src, n * sizeof(T), on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, st));
+  *out = (T*)p;
+  return EE_OK;
+}
+
+ee_status_t upload_bytes(ee_model* m, const void* src, size_t bytes, int on_device, cudaStream_t st, void** out) {
+  return upload<char>(m, (const char*)src, bytes, on_device, st, (char**)out);
+}
+
+void record(ee_model* m, StagePlan& sp, cudaStream_t st, const char* name) {
+  if (!m->timing) return;
+  if ((int)sp.ev.size() <= sp.ev_used) {
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) return;
+    sp.ev.push_back(e);
+    sp.ev_names.push_back(name);
+  }
+  sp.ev_names[sp.ev_used] = name;
+  cudaEventRecord(sp.ev[sp.ev_used++], st);
+}
+
+template <typename T>
+ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const void* res, void* dst, int B,
+                         cudaStream_t st) {
+  ConvGeom g{B, L.in_h, L.in_w, L.d.cin, L.out_h, L.out_w, L.d.cout, L.d.kh, L.d.kw, L.d.stride, L.d.pad, L.d.act};
+  constexpr int V = Elem<T>::kVec;
+  switch (L.kind) {
+    case KK_SIMT: {
+      dim3 grid(cdiv((long)B * L.out_h * L.out_w, kSimtBM), cdiv(L.d.cout, kSimtBN));
+      conv_igemm_simt_kernel<T><<<grid, kSimtThreads, 0, st>>>((const T*)src, (const T*)L.w_dev, L.scale_dev, L.bias_dev,
+                                                                 (const T*)res, (T*)dst, g);
+      break;
+    }
+    case KK_TC: {
+      ee_status_t s = tc_launch(m->tc, L.tc, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st);
+      if (s != EE_OK) return s;
+      break;
+    }
+    case KK_DW: {
+      const bool vec = L.d.cin % V == 0;
+      const long total = (long)B * L.out_h * L.out_w * (vec ? L.d.cin / V : L.d.cin);
+      const int grid = (int)std::min<long>(cdiv(total, 256), 148L * 32);
+      if (vec)
+        dwconv_kernel<T, V><<<grid, 256, 0, st>>>((const T*)src, (const T*)L.w_dev, L.scale_dev, L.bias_dev, (T*)dst, g);
+      else
+        dwconv_kernel<T, 1><<<grid, 256, 0, st>>>((const T*)src, (const T*)L.w_dev, L.scale_dev, L.bias_dev, (T*)dst, g);
+      break;
+    }
+    case KK_POOL: {
+      const bool vec = L.d.cin % V == 0;
+      const long total = (long)B * L.out_h * L.out_w * (vec ? L.d.cin / V : L.d.cin);
+      const int grid = (int)std::min<long>(cdiv(total, 256), 148L * 32);
+      if (vec)
+        maxpool_kernel<T, V><<<grid, 256, 0, st>>>((const T*)src, (T*)dst, g);
+      else
+        maxpool_kernel<T, 1><<<grid, 256, 0, st>>>((const T*)src, (T*)dst, g);
+      break;
+    }
+  }
+  EE_CUDA(cudaGetLastError());
+  return EE_OK;
+}
+
+template <typename T>
+ee_status_t launch_head(ee_model* m, StagePlan& sp, const void* x, int B, int hw, const float* shift,
+                        const int32_t* shift_cls, char* scratch, const ee_stage_in_t* in_ids, const ee_stage_out_t* out,
+                        cudaStream_t st, bool timed) {
+  const int C = sp.out_c, K = sp.n_classes;
+  HeadLayout h = head_layout(m->max_batch, hw, C, K, sizeof(T));
+  unsigned* cnt = (unsigned*)(scratch + h.off_cnt);
+  float* partial = (float*)(scratch + h.off_partial);
+  float* gap = (float*)(scratch + h.off_gap);
+  float* z = out->logits ? out->logits : (float*)(scratch + h.off_z);
+  constexpr int V = Elem<T>::kVec;
+  EE_CUDA(cudaMemsetAsync(cnt, 0, sizeof(unsigned) * (size_t)B, st));
+  dim3 ggrid(h.nchunks, B);
+  if (C % V == 0)
+    gap_kernel<T, V><<<ggrid, kGapThreads, 0, st>>>((const T*)x, hw, C, h.rows_per_chunk, partial, gap, cnt);
+  else
+    gap_kernel<T, 1><<<ggrid, kGapThreads, 0, st>>>((const T*)x, hw, C, h.rows_per_chunk, partial, gap, cnt);
+  EE_CUDA(cudaGetLastError());
+  if (timed) record(m, sp, st, "head_gap");
+  if (C % V == 0)
+    fc_kernel<T, V><<<cdiv(K, kFcWarps), kFcWarps * 32, 0, st>>>(gap, (const T*)sp.fc_w, sp.fc_b, B, C, K, z);
+  else
+    fc_kernel<T, 1><<<cdiv(K, kFcWarps), kFcWarps * 32, 0, st>>>(gap, (const T*)sp.fc_w, sp.fc_b, B, C, K, z);
+  EE_CUDA(cudaGetLastError());
+  if (timed) record(m, sp, st, "head_fc");
+  exit_decide_kernel<<<1, kDecideThreads, 0, st>>>(z, B, K, shift, shift_cls, sp.threshold, sp.always_exit, out->conf,
+                                                   out->pred, out->exit_mask, in_ids ? in_ids->ids : nullptr,
+                                                   out->survivor_idx, out->ids_out, out->n_surv_dev);
+  EE_CUDA(cudaGetLastError());
+  if (timed) record(m, sp, st, "head_softmax_scan");
+  return EE_OK;
+}
+
+template <typename V>
+ee_status_t gather_launch_t(const void* feat, size_t bytes_per_sample, const int32_t* idx, const int32_t* n_dev, int max_rows,
+                            void* out, cudaStream_t st) {
+  const size_t vecs = bytes_per_sample / sizeof(V);
+  dim3 grid(cdiv((long)vecs, kCopyThreads * kCopyUnroll), max_rows);
+  gather_rows_kernel<V><<<grid, kCopyThreads, 0, st>>>((const V*)feat, vecs, idx, n_dev, (V*)out);
+  EE_CUDA(cudaGetLastError());
+  return EE_OK;
+}
+
+// Widest vector that divides the row size and both base addresses.
+int copy_width(size_t bytes_per_sample, const void* a, const void* b) {
+  const uintptr_t bits = (uintptr_t)bytes_per_sample | (uintptr_t)a | (uintptr_t)b;
+  return (bits & 15) == 0 ? 16 : (bits & 3) == 0 ? 4 : (bits & 1) == 0 ? 2 : 1;
+}
+
+ee_status_t gather_launch(const void* feat, size_t bytes_per_sample, const int32_t* idx, const int32_t* n_dev, int max_rows,
+                          void* out, cudaStream_t st) {
+  if (max_rows <= 0 || bytes_per_sample == 0) return EE_OK;
+  switch (copy_width(bytes_per_sample, feat, out)) {
+    case 16: return gather_launch_t<uint4>(feat, bytes_per_sample, idx, n_dev, max_rows, out, st);
+    case 4: return gather_launch_t<uint32_t>(feat, bytes_per_sample, idx, n_dev, max_rows, out, st);
+    case 2: return gather_launch_t<uint16_t>(feat, bytes_per_sample, idx, n_dev, max_rows, out, st);
+    default: return gather_launch_t<uint8_t>(feat, bytes_per_sample, idx, n_dev, max_rows, out, st);
+  }
+}
+
+template <typename V>
+ee_status_t append_launch_t(const void* src, void* dst, size_t bytes, const int32_t* ids_src, int32_t* ids_dst, int n_ids,
+                            cudaStream_t st) {
+  const size_t vecs = bytes / sizeof(V);
+  const int grid = (int)std::min<size_t>((vecs + kCopyThreads - 1) / kCopyThreads, 148 * 16);
+  append_rows_kernel<V><<<grid, kCopyThreads, 0, st>>>((const V*)src, (V*)dst, vecs, ids_src, ids_dst, n_ids);
+  EE_CUDA(cudaGetLastError());
+  return EE_OK;
+}
+
+bool valid_out(const ee_stage_out_t* o, bool need_feat) {
+  return o && o->exit_mask && o->survivor_idx && o->n_surv_dev && (!need_feat || o->features_out);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* ee_status_string(ee_status_t s) {
+  switch (s) {
+    case EE_OK: return "ok";
+    case EE_ERR_INVALID_ARG: return "invalid argument";
+    case EE_ERR_SHAPE: return "layer shapes do not chain";
+    case EE_ERR_CAPACITY: return "batch or workspace capacity exceeded";
+    case EE_ERR_STAGE: return "stage index out of range";
+    case EE_ERR_UNSUPPORTED: return "unsupported layer geometry";
+    case EE_ERR_CUDA: return "CUDA error";
+    case EE_ERR_TIMEOUT: return "device-side wait timed out";
+    case EE_ERR_INTERNAL: return "internal error";
+  }
+  return "unknown status";
+}
+
+const char* ee_last_cuda_error(void) { return g_cuda_err.c_str(); }
+
+ee_status_t ee_model_destroy(ee_model_t* m) {
+  if (!m) return EE_ERR_INVALID_ARG;
+  for (auto& sp : m->stages)
+    for (auto e : sp.ev) cudaEventDestroy(e);
+  for (void* p : m->owned) cudaFree(p);
+  delete m;
+  return EE_OK;
+}
+
+ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_model_t** out) {
+  if (!desc || !out || !desc->stages || desc->n_stages < 1 || desc->max_batch < 1 || desc->in_h < 1 || desc->in_w < 1 ||
+      desc->in_c < 1 || (desc->dtype != EE_F32 && desc->dtype != EE_BF16))
+    return EE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  ee_model* m = new (std::nothrow) ee_model();
+  if (!m) return EE_ERR_INTERNAL;
+  m->dtype = desc->dtype;
+  m->in_h = desc->in_h;
+  m->in_w = desc->in_w;
+  m->in_c = desc->in_c;
+  m->max_batch = desc->max_batch;
+  const size_t es = esize(desc->dtype);
+  const int ondev = desc->weights_on_device;
+  ee_status_t rc = EE_OK;
+  auto fail = [&](ee_status_t s) {
+    cudaStreamSynchronize(st);
+    ee_model_destroy(m);
+    return s;
+  };
+  {
+    void* p = nullptr;
+    if (cudaMalloc(&p, 256) != cudaSuccess) return fail(EE_ERR_CUDA);
+    m->owned.push_back(p);
+    m->err_flag = (int*)p;
+    if (cudaMemsetAsync(p, 0, 256, st) != cudaSuccess) return fail(EE_ERR_CUDA);
+  }
+  rc = tc_context_init(m->tc);
+  if (rc != EE_OK) return fail(rc);
+
+  int h = desc->in_h, w = desc->in_w, c = desc->in_c;
+  m->stages.resize(desc->n_stages);
+  for (int s = 0; s < desc->n_stages; ++s) {
+    const ee_stage_desc_t& sd = desc->stages[s];
+    StagePlan& sp = m->stages[s];
+    if (sd.n_layers < 1 || !sd.layers || sd.n_classes < 1 || !sd.fc_weight) return fail(EE_ERR_INVALID_ARG);
+    const int out_layer = sd.out_layer < 0 ? sd.n_layers - 1 : sd.out_layer;
+    if (out_layer >= sd.n_layers) return fail(EE_ERR_INVALID_ARG);
+    sp.in_h = h;
+    sp.in_w = w;
+    sp.in_c = c;
+    sp.layers.resize(sd.n_layers);
+    std::vector<int> oh(sd.n_layers), ow(sd.n_layers), oc(sd.n_layers), last_use(sd.n_layers, -1);
+    // shapes and liveness
+    for (int i = 0; i < sd.n_layers; ++i) {
+      const ee_layer_desc_t& d = sd.layers[i];
+      LayerPlan& L = sp.layers[i];
+      L.d = d;
+      if (d.op < EE_OP_CONV || d.op > EE_OP_MAXPOOL || d.kh < 1 || d.kw < 1 || d.stride < 1 || d.pad < 0 || d.cin < 1 ||
+          d.cout < 1 || d.act < EE_ACT_NONE || d.act > EE_ACT_RELU6 || d.input_from < EE_FROM_STAGE_INPUT ||
+          d.input_from >= i || d.residual_from < EE_FROM_STAGE_INPUT || d.residual_from >= i)
+        return fail(EE_ERR_INVALID_ARG);
+      if (d.op != EE_OP_MAXPOOL && !d.weight) return fail(EE_ERR_INVALID_ARG);
+      int ih, iw, ic, src = d.input_from;
+      if (src == EE_FROM_STAGE_INPUT || (src == EE_FROM_PREV && i == 0)) {
+        ih = h, iw = w, ic = c, src = -1;
+      } else {
+        if (src == EE_FROM_PREV) src = i - 1;
+        ih = oh[src], iw = ow[src], ic = oc[src];
+        last_use[src] = i;
+      }
+      if (ic != d.cin) return fail(EE_ERR_SHAPE);
+      if ((d.op == EE_OP_DWCONV || d.op == EE_OP_MAXPOOL) && d.cin != d.cout) return fail(EE_ERR_SHAPE);
+      L.in_h = ih;
+      L.in_w = iw;
+      L.out_h = (ih + 2 * d.pad - d.kh) / d.stride + 1;
+      L.out_w = (iw + 2 * d.pad - d.kw) / d.stride + 1;
+      if (ih + 2 * d.pad < d.kh || iw + 2 * d.pad < d.kw || L.out_h < 1 || L.out_w < 1) return fail(EE_ERR_SHAPE);
+      oh[i] = L.out_h, ow[i] = L.out_w, oc[i] = d.cout;
+      L.src_slot = src;  // layer index for now; mapped to slots below
+      int rs = d.residual_from;
+      if (rs == EE_NO_RESIDUAL) {
+        L.res_slot = -2;
+      } else {
+        if (d.op != EE_OP_CONV) return fail(EE_ERR_UNSUPPORTED);
+        int rh, rw, rcn;
+        if (rs == EE_FROM_STAGE_INPUT) {
+          rh = h, rw = w, rcn = c;
+          L.res_slot = -1;
+        } else {
+          rh = oh[rs], rw = ow[rs], rcn = oc[rs];
+          L.res_slot = rs;
+          last_use[rs] = i;
+        }
+        if (rh != L.out_h || rw != L.out_w || rcn != d.cout) return fail(EE_ERR_SHAPE);
+      }
+      if (d.op != EE_OP_MAXPOOL) {
+        const int cpg = d.op == EE_OP_DWCONV ? 1 : d.cin;
+        sp.flops_per_sample += 2.0 * L.out_h * L.out_w * d.cout * (double)(d.kh * d.kw * cpg);
+      }
+    }
+    last_use[out_layer] = sd.n_layers + 1;
+    // slot assignment: a slot is reused once every consumer of its tensor has run
+    std::vector<size_t> slot_bps;   // bytes per sample of each slot
+    std::vector<int> slot_free_at;  // layer index from which the slot is free
+    std::vector<int> slot_of(sd.n_layers);
+    for (int i = 0; i < sd.n_layers; ++i) {
+      const size_t need = align_up((size_t)oh[i] * ow[i] * oc[i] * es, 256);
+      int pick = -1;
+      for (size_t k = 0; k < slot_bps.size(); ++k)
+        if (slot_free_at[k] <= i && (pick < 0 || slot_bps[k] > slot_bps[pick])) pick = (int)k;
+      if (pick < 0) {
+        slot_bps.push_back(need);
+        slot_free_at.push_back(0);
+        pick = (int)slot_bps.size() - 1;
+      }
+      if (slot_bps[pick] < need) slot_bps[pick] = need;
+      // the slot stays busy until after the last consumer; a never-read tensor frees at once
+      slot_free_at[pick] = last_use[i] < 0 ? i + 1 : last_use[i] + 1;
+      slot_of[i] = pick;
+    }
+    size_t off = 0;
+    sp.slot_off.resize(slot_bps.size());
+    for (size_t k = 0; k < slot_bps.size(); ++k) {
+      sp.slot_off[k] = off;
+      off += align_up(slot_bps[k] * (size_t)desc->max_batch, 1024);
+    }
+    for (int i = 0; i < sd.n_layers; ++i) {
+      LayerPlan& L = sp.layers[i];
+      L.out_slot = slot_of[i];
+      if (L.src_slot >= 0) L.src_slot = slot_of[L.src_slot];
+      if (L.res_slot >= 0) L.res_slot = slot_of[L.res_slot];
+    }
+    sp.out_slot = slot_of[out_layer];
+    sp.out_h = oh[out_layer];
+    sp.out_w = ow[out_layer];
+    sp.out_c = oc[out_layer];
+    HeadLayout hl = head_layout(desc->max_batch, sp.out_h * sp.out_w, sp.out_c, sd.n_classes, es);
+    sp.head_off = align_up(off, 1024);
+    sp.head_bytes = hl.bytes;
+    sp.ws_bytes = sp.head_off + hl.bytes;
+    sp.n_classes = sd.n_classes;
+    sp.threshold = sd.threshold;
+    sp.always_exit = sd.always_exit;
+    // uploads and kernel choice
+    for (int i = 0; i < sd.n_layers; ++i) {
+      LayerPlan& L = sp.layers[i];
+      const ee_layer_desc_t& d = L.d;
+      if (d.op == EE_OP_MAXPOOL) {
+        L.kind = KK_POOL;
+        continue;
+      }
+      const int cpg = d.op == EE_OP_DWCONV ? 1 : d.cin;
+      const size_t wn = (size_t)d.cout * d.kh * d.kw * cpg;
+      if ((rc = upload_bytes(m, d.weight, wn * es, ondev, st, &L.w_dev)) != EE_OK) return fail(rc);
+      if ((rc = upload<float>(m, d.scale, d.cout, ondev, st, &L.scale_dev)) != EE_OK) return fail(rc);
+      if ((rc = upload<float>(m, d.bias, d.cout, ondev, st, &L.bias_dev)) != EE_OK) return fail(rc);
+      if (d.op == EE_OP_DWCONV) {
+        L.kind = KK_DW;
+      } else if (desc->dtype == EE_BF16 && tc_supported(d, L.in_h, L.in_w)) {
+        L.kind = KK_TC;
+        rc = tc_plan_layer(m->tc, d, L.in_h, L.in_w, L.out_h, L.out_w, desc->max_batch, L.w_dev, &L.tc);
+        if (rc != EE_OK) return fail(rc);
+      } else {
+        L.kind = KK_SIMT;
+      }
+    }
+    if ((rc = upload_bytes(m, sd.fc_weight, (size_t)sd.n_classes * sp.out_c * es, ondev, st, &sp.fc_w)) != EE_OK) return fail(rc);
+    if ((rc = upload<float>(m, sd.fc_bias, sd.n_classes, ondev, st, &sp.fc_b)) != EE_OK) return fail(rc);
+    h = sp.out_h, w = sp.out_w, c = sp.out_c;
+  }
+  if (cudaStreamSynchronize(st) != cudaSuccess) return fail(EE_ERR_CUDA);
+  *out = m;
+  return EE_OK;
+}
+
+ee_status_t ee_model_query(const ee_model_t* m, int stage, ee_stage_info_t* out) {
+  if (!m || !out) return EE_ERR_INVALID_ARG;
+  if (stage < 0 || stage >= (int)m->stages.size()) return EE_ERR_STAGE;
+  const StagePlan& sp = m->stages[stage];
+  const size_t es = esize(m->dtype);
+  out->in_h = sp.in_h, out->in_w = sp.in_w, out->in_c = sp.in_c;
+  out->out_h = sp.out_h, out->out_w = sp.out_w, out->out_c = sp.out_c;
+  out->in_bytes_per_sample = (size_t)sp.in_h * sp.in_w * sp.in_c * es;
+  out->out_bytes_per_sample = (size_t)sp.out_h * sp.out_w * sp.out_c * es;
+  out->workspace_bytes = sp.ws_bytes;
+  out->n_layers = (int)sp.layers.size();
+  out->flops_per_sample = sp.flops_per_sample;
+  return EE_OK;
+}
+
+ee_status_t ee_stage_run(ee_model_t* m, int stage, const ee_stage_in_t* in, void* workspace, size_t workspace_bytes,
+                         const ee_stage_out_t* out, void* cuda_stream) {
+  if (!m || !in || !valid_out(out, true) || in->batch < 0) return EE_ERR_INVALID_ARG;
+  if (stage < 0 || stage >= (int)m->stages.size()) return EE_ERR_STAGE;
+  if (in->logit_shift && !in->shift_class) return EE_ERR_INVALID_ARG;
+  StagePlan& sp = m->stages[stage];
+  const int B = in->batch;
+  if (B > m->max_batch) return EE_ERR_CAPACITY;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (B == 0) {
+    EE_CUDA(cudaMemsetAsync(out->n_surv_dev, 0, sizeof(int32_t), st));
+    if (out->n_surv_host) EE_CUDA(cudaMemcpyAsync(out->n_surv_host, out->n_surv_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    return EE_OK;
+  }
+  if (!in->features || !workspace || ((uintptr_t)workspace & 255)) return EE_ERR_INVALID_ARG;
+  if (workspace_bytes < sp.ws_bytes) return EE_ERR_CAPACITY;
+  char* ws = (char*)workspace;
+  sp.ev_used = 0;
+  record(m, sp, st, "begin");
+  for (size_t i = 0; i < sp.layers.size(); ++i) {
+    const LayerPlan& L = sp.layers[i];
+    const void* src = L.src_slot < 0 ? in->features : ws + sp.slot_off[L.src_slot];
+    const void* res = L.res_slot == -2 ? nullptr : (L.res_slot == -1 ? in->features : ws + sp.slot_off[L.res_slot]);
+    void* dst = ws + sp.slot_off[L.out_slot];
+    ee_status_t s = m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, src, res, dst, B, st)
+                                        : launch_layer<float>(m, L, src, res, dst, B, st);
+    if (s != EE_OK) return s;
+    record(m, sp, st, kKernelNames[L.kind]);
+  }
+  const void* so = ws + sp.slot_off[sp.out_slot];
+  const int hw = sp.out_h * sp.out_w;
+  ee_status_t s = m->dtype == EE_BF16
+                      ? launch_head<bf16>(m, sp, so, B, hw, in->logit_shift, in->shift_class, ws + sp.head_off, in, out, st, true)
+                      : launch_head<float>(m, sp, so, B, hw, in->logit_shift, in->shift_class, ws + sp.head_off, in, out, st, true);
+  if (s != EE_OK) return s;
+  if (!sp.always_exit) {
+    s = gather_launch(so, (size_t)hw * sp.out_c * esize(m->dtype), out->survivor_idx, out->n_surv_dev, B, out->features_out, st);
+    if (s != EE_OK) return s;
+    record(m, sp, st, "gather_survivors");
+  }
+  if (out->n_surv_host) EE_CUDA(cudaMemcpyAsync(out->n_surv_host, out->n_surv_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  return EE_OK;
+}
+
+ee_status_t ee_batch_refill(ee_model_t* m, int boundary, void* batch_feat, int32_t* batch_ids, int n_surv, const void* arr_feat,
+                            const int32_t* arr_ids, int n_arr, int* n_accepted, int* n_merged, void* cuda_stream) {
+  if (!m || !n_accepted || !n_merged || n_surv < 0 || n_arr < 0) return EE_ERR_INVALID_ARG;
+  if (boundary < 0 || boundary > (int)m->stages.size() - 1) return EE_ERR_STAGE;
+  if (n_surv > m->max_batch) return EE_ERR_CAPACITY;
+  if (n_arr > 0 && (!batch_feat || !arr_feat)) return EE_ERR_INVALID_ARG;
+  const StagePlan& sp = m->stages[boundary];
+  const size_t bps = (size_t)sp.in_h * sp.in_w * sp.in_c * esize(m->dtype);
+  const int slack = m->max_batch - n_surv;            // B_slack = B_max - B_rem
+  const int n_acc = n_arr < slack ? n_arr : slack;    // B_incr  = min(N_Q, B_slack)
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (n_acc > 0) {
+    void* dst = (char*)batch_feat + bps * (size_t)n_surv;
+    int32_t* ids_dst = batch_ids ? batch_ids + n_surv : nullptr;
+    const size_t bytes = bps * (size_t)n_acc;
+    ee_status_t s;
+    switch (copy_width(bps, arr_feat, batch_feat)) {
+      case 16: s = append_launch_t<uint4>(arr_feat, dst, bytes, arr_ids, ids_dst, n_acc, st); break;
+      case 4: s = append_launch_t<uint32_t>(arr_feat, dst, bytes, arr_ids, ids_dst, n_acc, st); break;
+      case 2: s = append_launch_t<uint16_t>(arr_feat, dst, bytes, arr_ids, ids_dst, n_acc, st); break;
+      default: s = append_launch_t<uint8_t>(arr_feat, dst, bytes, arr_ids, ids_dst, n_acc, st); break;
+    }
+    if (s != EE_OK) return s;
+  }
+  *n_accepted = n_acc;
+  *n_merged = n_surv + n_acc;                          // B_merged = B_rem + B_incr
+  return EE_OK;
+}
+
+size_t ee_exit_head_scratch_bytes(const ee_model_t* m, int stage) {
+  if (!m || stage < 0 || stage >= (int)m->stages.size()) return 0;
+  return m->stages[stage].head_bytes;
+}
+
+ee_status_t ee_exit_head(ee_model_t* m, int stage, const void* x, int batch, int hw, const float* logit_shift,
+                         const int32_t* shift_class, void* scratch, size_t scratch_bytes, const ee_stage_out_t* out,
+                         void* cuda_stream) {
+  if (!m || !valid_out(out, false) || batch < 0 || hw < 1) return EE_ERR_INVALID_ARG;
+  if (stage < 0 || stage >= (int)m->stages.size()) return EE_ERR_STAGE;
+  if (logit_shift && !shift_class) return EE_ERR_INVALID_ARG;
+  StagePlan& sp = m->stages[stage];
+  if (batch > m->max_batch) return EE_ERR_CAPACITY;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (batch == 0) {
+    EE_CUDA(cudaMemsetAsync(out->n_surv_dev, 0, sizeof(int32_t), st));
+    return EE_OK;
+  }
+  if (!x || !scratch || ((uintptr_t)scratch & 255)) return EE_ERR_INVALID_ARG;
+  // the pooling chunks follow hw, so the scratch need is re-derived for the hw given
+  HeadLayout hl = head_layout(m->max_batch, hw, sp.out_c, sp.n_classes, esize(m->dtype));
+  if (scratch_bytes < hl.bytes) return EE_ERR_CAPACITY;
+  return m->dtype == EE_BF16
+             ? launch_head<bf16>(m, sp, x, batch, hw, logit_shift, shift_class, (char*)scratch, nullptr, out, st, false)
+             : launch_head<float>(m, sp, x, batch, hw, logit_shift, shift_class, (char*)scratch, nullptr, out, st, false);
+}
+
+ee_status_t ee_gather_survivors(const void* feat, size_t bytes_per_sample, const int32_t* survivor_idx, const int32_t* n_surv_dev,
+                                int max_rows, void* feat_out, void* cuda_stream) {
+  if (!feat || !survivor_idx || !n_surv_dev || !feat_out || max_rows < 0) return EE_ERR_INVALID_ARG;
+  return gather_launch(feat, bytes_per_sample, survivor_idx, n_surv_dev, max_rows, feat_out, (cudaStream_t)cuda_stream);
+}
+
+ee_status_t ee_model_set_timing(ee_model_t* m, int enabled) {
+  if (!m) return EE_ERR_INVALID_ARG;
+  m->timing = enabled != 0;
+  return EE_OK;
+}
+
+ee_status_t ee_model_get_timing(ee_model_t* m, int stage, int cap, float* ms, const char** names, int* n) {
+  if (!m || !ms || !n || cap < 0) return EE_ERR_INVALID_ARG;
+  if (stage < 0 || stage >= (int)m->stages.size()) return EE_ERR_STAGE;
+  StagePlan& sp = m->stages[stage];
+  *n = 0;
+  if (sp.ev_used < 2) return EE_OK;
+  EE_CUDA(cudaEventSynchronize(sp.ev[sp.ev_used - 1]));
+  for (int i = 1; i < sp.ev_used && *n < cap; ++i) {
+    float t = 0.f;
+    EE_CUDA(cudaEventElapsedTime(&t, sp.ev[i - 1], sp.ev[i]));
+    ms[*n] = t;
+    if (names) names[*n] = sp.ev_names[i];
+    ++*n;
+  }
+  return EE_OK;
+}
+
+ee_status_t ee_model_plan(const ee_model_t* m, int stage, int batch, int cap, ee_layer_plan_t* out, int* n) {
+  if (!m || !out || !n || cap < 0 || batch < 0) return EE_ERR_INVALID_ARG;
+  if (stage < 0 || stage >= (int)m->stages.size()) return EE_ERR_STAGE;
+  const StagePlan& sp = m->stages[stage];
+  const double es = (double)esize(m->dtype);
+  *n = 0;
+  for (size_t i = 0; i < sp.layers.size() && *n < cap; ++i) {
+    const LayerPlan& L = sp.layers[i];
+    ee_layer_plan_t& p = out[(*n)++];
+    const int cpg = L.d.op == EE_OP_CONV ? L.d.cin : 1;
+    p.kernel = kKernelNames[L.kind];
+    p.m = batch * L.out_h * L.out_w;
+    p.n = L.d.cout;
+    p.k = L.d.kh * L.d.kw * cpg;
+    p.flops = L.d.op == EE_OP_MAXPOOL ? 0.0 : 2.0 * p.m * (double)p.n * p.k;
+    const double in_b = (double)batch * L.in_h * L.in_w * L.d.cin * es, out_b = (double)p.m * p.n * es;
+    const double w_b = L.d.op == EE_OP_MAXPOOL ? 0.0 : (double)L.d.cout * p.k * es;
+    p.bytes = in_b + out_b + w_b + (L.res_slot != -2 ? out_b : 0.0);
+  }
+  return EE_OK;
+}
+
+ee_status_t ee_model_check(ee_model_t* m, void* cuda_stream) {
+  if (!m) return EE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int flag = 0;
+  EE_CUDA(cudaMemcpyAsync(&flag, m->err_flag, sizeof(int), cudaMemcpyDeviceToHost, st));
+  EE_CUDA(cudaStreamSynchronize(st));
+  if (flag) {
+    EE_CUDA(cudaMemsetAsync(m->err_flag, 0, sizeof(int), st));
+    EE_CUDA(cudaStreamSynchronize(st));
+    return EE_ERR_TIMEOUT;
+  }
+  return EE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,250 @@
+// Exit head and batch bookkeeping kernels: global average pool, FC, softmax top-1 + threshold,
+// stable compaction scan, survivor gather, refill copy.
+//
+// The exit head is the intermediate classifier whose softmax top-1 probability is the
+// confidence that is compared with the exit's threshold (paper Section II-B; Section IV,
+// Benchmarks).  The scan produces B_rem = B_act - B_exit and the order-preserving list of the
+// remaining samples, the gather is their write-back to the next subnet's input buffer
+// (Section III-B, Preemption Mechanism), the refill copy appends B_incr new samples
+// (Algorithm 1: B_merged = B_rem + B_incr).
+//
+// All reductions run in a fixed order that depends on the layer shape only, never on the
+// batch size or on scheduling, so a sample's logits are bit-identical in any batch.
+#pragma once
+#include "common.cuh"
+
+namespace ee {
+
+constexpr int kGapThreads = 256;
+
+// Partial column sums of one sample's [HW][C] map over rows [chunk*rows_per_chunk, ...), written to
+// partial[b][chunk][C]; the last CTA to finish a sample adds the chunks in ascending order and
+// writes gap[b][c] = sum / HW.  counters[b] must be zero on entry and is zero again on exit.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(kGapThreads)
+gap_kernel(const T* __restrict__ x, int HW, int C, int rows_per_chunk, float* __restrict__ partial,
+           float* __restrict__ gap, unsigned* __restrict__ counters) {
+  __shared__ float red[kGapThreads * VEC];
+  __shared__ bool is_last;
+  const int tid = threadIdx.x, b = blockIdx.y, chunk = blockIdx.x, nchunks = gridDim.x;
+  const int cv = C / VEC;
+  const int per = cv < kGapThreads ? cv : kGapThreads;
+  const int groups = kGapThreads / per;
+  const int grp = tid / per, lv = tid - grp * per;
+  const bool active = grp < groups;
+  const int r0 = chunk * rows_per_chunk;
+  const int r1 = min(HW, r0 + rows_per_chunk);
+  const T* xb = x + (size_t)b * HW * C;
+  float* pout = partial + ((size_t)b * nchunks + chunk) * C;
+  for (int vb = 0; vb < cv; vb += per) {
+    const int v = vb + lv;
+    float acc[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+    if (active && v < cv) {
+      for (int r = r0 + grp; r < r1; r += groups) {
+        const T* p = xb + (size_t)r * C + (size_t)v * VEC;
+        if constexpr (VEC > 1) {
+          Vec16<T> t;
+          t.load(p);
+#pragma unroll
+          for (int e = 0; e < VEC; ++e) acc[e] += t.v[e];
+        } else {
+          acc[0] += Elem<T>::ld(p);
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) red[(grp * per + lv) * VEC + e] = acc[e];
+    }
+    __syncthreads();
+    if (grp == 0 && v < cv) {
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) {
+        float s = 0.f;
+        for (int q = 0; q < groups; ++q) s += red[(q * per + lv) * VEC + e];
+        pout[v * VEC + e] = s;
+      }
+    }
+    __syncthreads();
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) is_last = atomicAdd(&counters[b], 1u) == (unsigned)(nchunks - 1);
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  const float inv = 1.0f / (float)HW;
+  const float* pb = partial + (size_t)b * nchunks * C;
+  for (int c = tid; c < C; c += kGapThreads) {
+    float s = 0.f;
+    for (int q = 0; q < nchunks; ++q) s += __ldcg(pb + (size_t)q * C + c);
+    gap[(size_t)b * C + c] = s * inv;
+  }
+  if (tid == 0) counters[b] = 0;
+}
+
+constexpr int kFcWarps = 8, kFcSamples = 8;
+
+// z[b][k] = bfc[k] + sum_c wfc[k][c] * gap[b][c].  One warp per class, samples in tiles of eight so
+// that a weight vector is loaded once per eight samples.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(kFcWarps * 32)
+fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float* __restrict__ bfc, int B, int C, int K,
+          float* __restrict__ z) {
+  const int lane = threadIdx.x & 31, k = blockIdx.x * kFcWarps + (threadIdx.x >> 5);
+  if (k >= K) return;
+  const T* wr = wfc + (size_t)k * C;
+  const float bk = bfc ? bfc[k] : 0.f;
+  for (int b0 = 0; b0 < B; b0 += kFcSamples) {
+    float acc[kFcSamples];
+#pragma unroll
+    for (int s = 0; s < kFcSamples; ++s) acc[s] = 0.f;
+    for (int c = lane * VEC; c < C; c += 32 * VEC) {
+      float wv[VEC];
+      if constexpr (VEC > 1) {
+        Vec16<T> t;
+        t.load(wr + c);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) wv[e] = t.v[e];
+      } else {
+        wv[0] = Elem<T>::ld(wr + c);
+      }
+#pragma unroll
+      for (int s = 0; s < kFcSamples; ++s) {
+        if (b0 + s < B) {
+          const float* gp = gap + (size_t)(b0 + s) * C + c;
+#pragma unroll
+          for (int e = 0; e < VEC; ++e) acc[s] = fmaf(wv[e], gp[e], acc[s]);
+        }
+      }
+    }
+#pragma unroll
+    for (int s = 0; s < kFcSamples; ++s) {
+      float v = acc[s];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0 && b0 + s < B) z[(size_t)(b0 + s) * K + k] = v + bk;
+    }
+  }
+}
+
+constexpr int kDecideThreads = 1024;
+
+// One CTA.  Per sample (one warp each): optional logit shift, max / lowest argmax, conf = 1 / sum exp(z - max),
+// exit = always || conf >= thr (NaN never exits).  Then a ballot + prefix-sum scan over the not-exit flags
+// gives the ascending survivor list, the survivors' ids and their count.
+__global__ void __launch_bounds__(kDecideThreads)
+exit_decide_kernel(float* __restrict__ z, int B, int K, const float* __restrict__ shift, const int32_t* __restrict__ shift_cls,
+                   float thr, int always_exit, float* __restrict__ conf, int32_t* __restrict__ pred,
+                   uint8_t* __restrict__ mask, const int32_t* __restrict__ ids, int32_t* __restrict__ surv_idx,
+                   int32_t* __restrict__ ids_out, int32_t* __restrict__ n_surv) {
+  __shared__ int warp_tot[32];
+  __shared__ int pass_total;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int b = warp; b < B; b += kDecideThreads / 32) {
+    float* zb = z + (size_t)b * K;
+    const int cls = (shift && shift_cls) ? shift_cls[b] : -1;
+    float m = -INFINITY;
+    int arg = 0x7fffffff;
+    for (int k = lane; k < K; k += 32) {
+      float v = zb[k];
+      if (k == cls) {
+        v += shift[b];
+        zb[k] = v;
+      }
+      if (v > m) {
+        m = v;
+        arg = k;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float om = __shfl_xor_sync(0xffffffffu, m, o);
+      const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
+      if (om > m || (om == m && oa < arg)) {
+        m = om;
+        arg = oa;
+      }
+    }
+    __syncwarp();
+    float s = 0.f;
+    for (int k = lane; k < K; k += 32) s += expf(zb[k] - m);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) {
+      const float cf = 1.0f / s;
+      if (conf) conf[b] = cf;
+      if (pred) pred[b] = arg == 0x7fffffff ? 0 : arg;
+      mask[b] = (uint8_t)((always_exit || cf >= thr) ? 1 : 0);
+    }
+  }
+  __syncthreads();
+  int base = 0;  // identical in every thread
+  for (int p0 = 0; p0 < B; p0 += kDecideThreads) {
+    const int b = p0 + tid;
+    const bool keep = b < B && mask[b] == 0;
+    const unsigned bal = __ballot_sync(0xffffffffu, keep);
+    const int pre = __popc(bal & ((1u << lane) - 1u));
+    if (lane == 0) warp_tot[warp] = __popc(bal);
+    __syncthreads();
+    if (warp == 0) {
+      const int t = warp_tot[lane];
+      int inc = t;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+      }
+      warp_tot[lane] = inc - t;  // exclusive offset of each warp
+      if (lane == 31) pass_total = inc;
+    }
+    __syncthreads();
+    if (keep) {
+      const int pos = base + warp_tot[warp] + pre;
+      surv_idx[pos] = b;
+      if (ids && ids_out) ids_out[pos] = ids[b];
+    }
+    base += pass_total;
+    __syncthreads();
+  }
+  if (tid == 0) n_surv[0] = base;
+}
+
+constexpr int kCopyThreads = 256, kCopyUnroll = 8;
+
+// feat_out[j] = feat[surv_idx[j]] for j < *n_surv, in vectors of type V (16 bytes whenever the row size
+// allows), grid (chunks, max_rows).
+template <typename V>
+__global__ void __launch_bounds__(kCopyThreads)
+gather_rows_kernel(const V* __restrict__ src, size_t vecs_per_row, const int32_t* __restrict__ surv_idx,
+                   const int32_t* __restrict__ n_surv, V* __restrict__ dst) {
+  const int j = blockIdx.y;
+  if (j >= *n_surv) return;
+  const V* s = src + (size_t)surv_idx[j] * vecs_per_row;
+  V* d = dst + (size_t)j * vecs_per_row;
+  const size_t v0 = (size_t)blockIdx.x * (kCopyThreads * kCopyUnroll) + threadIdx.x;
+  V r[kCopyUnroll];
+#pragma unroll
+  for (int u = 0; u < kCopyUnroll; ++u) {
+    const size_t v = v0 + (size_t)u * kCopyThreads;
+    if (v < vecs_per_row) r[u] = __ldcs(s + v);
+  }
+#pragma unroll
+  for (int u = 0; u < kCopyUnroll; ++u) {
+    const size_t v = v0 + (size_t)u * kCopyThreads;
+    if (v < vecs_per_row) d[v] = r[u];
+  }
+}
+
+// Flat copy of n vectors plus n_ids int32 (the appended arrivals of a refill).
+template <typename V>
+__global__ void __launch_bounds__(kCopyThreads)
+append_rows_kernel(const V* __restrict__ src, V* __restrict__ dst, size_t n, const int32_t* __restrict__ ids_src,
+                   int32_t* __restrict__ ids_dst, int n_ids) {
+  const size_t stride = (size_t)gridDim.x * kCopyThreads;
+  for (size_t v = (size_t)blockIdx.x * kCopyThreads + threadIdx.x; v < n; v += stride) dst[v] = __ldcs(src + v);
+  if (ids_src && ids_dst && blockIdx.x == 0)
+    for (int i = threadIdx.x; i < n_ids; i += kCopyThreads) ids_dst[i] = ids_src[i];
+}
+
+}  // namespace ee

@@ -1,0 +1,295 @@
+"""Parity of the CUDA library (through its C ABI) against the CPU oracle, element by element,
+on seeded inputs small enough for the oracle to finish in seconds yet spanning several tiles
+and ragged tails.  Every stage is fed the ORACLE's stage input (stage-local parity)."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ee_oracle as eo
+from paper_2209_13443_b200 import binding as eb
+from paper_2209_13443_b200 import workloads as wl
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+# ----------------------------------------------------------------------------- config 1
+
+@pytest.mark.parametrize("B", [1, 2, 3, 5, 7, 8])
+def test_tiny_fp32_stagewise(B):
+    spec = wl.tiny_ee_cnn(seed=0)
+    run = util.GpuRunner(spec)
+    x = wl.make_input(spec, B, seed=0)
+    ids = 100 + np.arange(B, dtype=np.int32)
+    exited = 0
+    for s in range(3):
+        o = util.oracle_stage(spec, s, x, ids)
+        g = run.stage(s, x, ids)
+        util.check_stage(spec, g, o, f"tiny B={B} stage {s}")
+        exited += int(o["exit"].sum())
+        x, ids = o["features_out"], o["ids_out"]
+        if len(ids) == 0:
+            break
+    assert exited == B                                              # every sample leaves exactly once
+
+
+def test_tiny_end_to_end_schedule_reproduces_serial_reference():
+    """GPU-only chain with a refill at the first boundary; per id the exit and prediction must be
+    those of the sample run alone through the oracle (samples finish out of order, matched by id)."""
+    spec = wl.tiny_ee_cnn(seed=0)
+    run = util.GpuRunner(spec)
+    m = run.m
+    x = wl.make_input(spec, 8, seed=0)
+    serial = [eo.run_sample_serial(spec, x[i]) for i in range(8)]
+    near = [i for i in range(8) if any(abs(c - 0.6) < util.BAND for c in serial[i][2][:2])]
+    done = {}
+
+    def harvest(s, ids_np, B):
+        out = run.bufs[s]
+        mask = out.exit_mask[:B].cpu().numpy()
+        pred = out.pred[:B].cpu().numpy()
+        for j in np.nonzero(mask)[0]:
+            assert int(ids_np[j]) not in done
+            done[int(ids_np[j])] = (s, int(pred[j]))
+
+    xd = eb.to_device("f32", x)
+    ids_a = torch.arange(0, 5, dtype=torch.int32, device="cuda")
+    ids_b = torch.arange(5, 8, dtype=torch.int32, device="cuda")
+    # active batch {0..4} to exit 0, parked in `park`
+    m.stage_run(0, xd[:5], 5, run.bufs[0], run.ws, ids_a)
+    torch.cuda.synchronize()
+    harvest(0, ids_a.cpu().numpy(), 5)
+    n_rem = int(run.bufs[0].n_surv_host[0])
+    park = run.bufs[0].features_out.clone()
+    park_ids = run.bufs[0].ids_out.clone()
+    # catch-up batch {5,6,7} to exit 0, then merged behind the parked survivors
+    m.stage_run(0, xd[5:], 3, run.bufs[0], run.ws, ids_b)
+    torch.cuda.synchronize()
+    harvest(0, ids_b.cpu().numpy(), 3)
+    n_new = int(run.bufs[0].n_surv_host[0])
+    n_acc, n_mer = m.batch_refill(1, park, park_ids, n_rem, run.bufs[0].features_out, run.bufs[0].ids_out, n_new)
+    assert n_acc == min(n_new, spec.max_batch - n_rem) and n_mer == n_rem + n_acc
+    feat, ids, n = park, park_ids, n_mer
+    for s in (1, 2):
+        if n == 0:
+            break
+        m.stage_run(s, feat, n, run.bufs[s], run.ws, ids)
+        torch.cuda.synchronize()
+        harvest(s, ids[:n].cpu().numpy(), n)
+        feat, ids, n = run.bufs[s].features_out, run.bufs[s].ids_out, int(run.bufs[s].n_surv_host[0])
+    assert n == 0 and sorted(done) == list(range(8))
+    for i in range(8):
+        if i not in near:
+            assert done[i] == serial[i][:2], (i, done[i], serial[i])
+
+
+# ----------------------------------------------------------------------------- single layers
+
+GEOMS = [
+    # H, W, cin, cout, k, stride, pad, act, residual
+    (9, 7, 3, 5, 3, 1, 1, wl.ACT_RELU, False),          # odd sizes, ragged M and N
+    (13, 11, 3, 64, 7, 2, 3, wl.ACT_RELU, False),       # stem-like
+    (8, 8, 16, 24, 1, 1, 0, wl.ACT_NONE, True),         # pointwise + residual, linear
+    (10, 6, 24, 32, 3, 2, 1, wl.ACT_RELU6, False),
+    (7, 7, 64, 64, 3, 1, 1, wl.ACT_RELU, True),
+    (14, 14, 64, 256, 1, 1, 0, wl.ACT_RELU, True),
+    (15, 9, 64, 128, 1, 2, 0, wl.ACT_NONE, False),      # strided projection, odd input
+    (12, 12, 128, 128, 3, 2, 1, wl.ACT_RELU, False),
+    (6, 6, 320, 96, 1, 1, 0, wl.ACT_NONE, False),
+    (5, 5, 136, 72, 3, 1, 1, wl.ACT_RELU, False),       # K and N not multiples of 64
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("geom", GEOMS)
+def test_conv_layer(dtype, geom):
+    H, W, cin, cout, k, stride, pad, act, residual = geom
+    spec = util.single_layer_model(dtype, H, W, cin, cout, k, stride, pad, act, residual, seed=hash(geom) % 1000, max_batch=5)
+    run = util.GpuRunner(spec)
+    for B in (1, 5):
+        x = wl.random_features((B, H, W, cin), seed=B, bf16=dtype == "bf16", relu=False)
+        o = util.oracle_stage(spec, 0, x)
+        g = run.stage(0, x)
+        r = util.check_stage(spec, g, o, f"{dtype} {geom} B={B}", elementwise=True)
+        assert g["n_surv"] == B
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("C,stride,H,W", [(32, 1, 9, 9), (96, 2, 10, 7), (144, 1, 6, 6), (12, 2, 8, 8)])
+def test_depthwise_layer(dtype, C, stride, H, W):
+    spec = util.single_layer_model(dtype, H, W, C, C, 3, stride, 1, wl.ACT_RELU6, False, seed=C, op=wl.OP_DWCONV)
+    run = util.GpuRunner(spec)
+    x = wl.random_features((3, H, W, C), seed=3, bf16=dtype == "bf16", relu=False)
+    util.check_stage(spec, run.stage(0, x), util.oracle_stage(spec, 0, x), f"dw {dtype} C={C}", elementwise=True)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_maxpool_layer(dtype):
+    rng = wl._rng(5, 901)
+    bf16 = dtype == "bf16"
+    layers = [wl.Layer(wl.OP_MAXPOOL, 16, 16, 3, 3, 2, 1)]
+    fw, fb = wl._head(rng, 16, 5, 1.0, bf16)
+    spec = wl.Model("pool", dtype, 11, 9, 16, [wl.Stage(layers, 5, fw, fb, 2.0, False)], 3)
+    run = util.GpuRunner(spec)
+    x = -np.abs(wl.random_features((3, 11, 9, 16), seed=4, bf16=bf16)) - 1.0    # zero padding would win if it took part
+    x = wl.to_bf16_grid(x) if bf16 else x
+    o = util.oracle_stage(spec, 0, x)
+    g = run.stage(0, x)
+    assert np.array_equal(g["features_out"], o["features_out"])
+
+
+# ----------------------------------------------------------------------------- configs 2-3 at reduced size
+
+def _stagewise(spec, B, seed, tol=None):
+    run = util.GpuRunner(spec)
+    x = wl.make_input(spec, B, seed=seed)
+    ids = np.arange(B, dtype=np.int32)
+    stats = []
+    for s in range(len(spec.stages)):
+        o = util.oracle_stage(spec, s, x, ids)
+        g = run.stage(s, x, ids)
+        stats.append(util.check_stage(spec, g, o, f"{spec.name} B={B} stage {s}", tol))
+        # next stage is fed ALL samples' oracle output (not only survivors) to keep every stage busy
+        x = o["stage_out"]
+    return stats
+
+
+@pytest.mark.parametrize("B", [1, 6])
+def test_resnet50_shaped_small(B):
+    spec = wl.resnet50_ee(seed=1, in_hw=64, n_classes=100, max_batch=6)
+    _stagewise(spec, B, seed=1)
+
+
+@pytest.mark.parametrize("B", [1, 5])
+def test_mobilenetv2_shaped_small(B):
+    spec = wl.mobilenetv2_ee(seed=2, in_hw=64, n_classes=100, max_batch=5)
+    _stagewise(spec, B, seed=2)
+
+
+# ----------------------------------------------------------------------------- head, compaction, refill
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,HW,C,K", [(1, 1, 8, 3), (5, 49, 64, 10), (64, 196, 256, 1000), (33, 50, 40, 17), (7, 3136, 32, 100),
+                                     (3, 7, 2048, 1000), (4, 9, 6, 5)])
+def test_exit_head_alone(dtype, B, HW, C, K):
+    bf16 = dtype == "bf16"
+    rng = wl._rng(B * 1000 + C, 902)
+    fw, fb = wl._head(rng, C, K, 8.0, bf16)
+    layers = [wl._conv(rng, wl.OP_CONV, C, C, 1, 1, 0, wl.ACT_NONE, bf16=bf16)]
+    spec = wl.Model("head", dtype, 1, HW, C, [wl.Stage(layers, K, fw, fb, 0.5, False)], max(B, 1))
+    m = eb.EEModel(spec)
+    out = eb.StageBuffers(m, 0)
+    scratch = torch.empty(m.exit_head_scratch_bytes(0) + 256, dtype=torch.uint8, device="cuda")
+    x = wl.random_features((B, HW, C), seed=HW, bf16=bf16)
+    shift = (np.arange(B) % 3 == 0).astype(np.float32) * 9.0
+    cls = (np.arange(B) * 5 % K).astype(np.int32)
+    m.exit_head(0, eb.to_device(dtype, x), B, HW, out, scratch, torch.as_tensor(shift, device="cuda"), torch.as_tensor(cls, device="cuda"))
+    torch.cuda.synchronize()
+    o = eo.exit_head(x, fw, fb, 0.5, False, shift, cls)
+    g = {"z": out.logits[:B].cpu().numpy(), "conf": out.conf[:B].cpu().numpy(), "pred": out.pred[:B].cpu().numpy(),
+         "exit": out.exit_mask[:B].cpu().numpy()}
+    n = int(out.n_surv_dev.cpu()[0])
+    assert util.rel_err(g["z"], o["z"]) <= (2e-3 if bf16 else 1e-5)
+    band = np.abs(o["conf"] - 0.5) < util.BAND
+    assert np.array_equal(g["exit"][~band], o["exit"][~band])
+    assert np.array_equal(out.survivor_idx[:n].cpu().numpy(), np.nonzero(g["exit"] == 0)[0])
+    # a second call on the same scratch must give bit-identical results (scratch is re-initialised by the call)
+    z1 = out.logits[:B].clone()
+    m.exit_head(0, eb.to_device(dtype, x), B, HW, out, scratch, torch.as_tensor(shift, device="cuda"), torch.as_tensor(cls, device="cuda"))
+    torch.cuda.synchronize()
+    assert torch.equal(z1, out.logits[:B])
+
+
+def test_compaction_masks_and_gather_bit_exact():
+    """Force every mask pattern of a small batch through the head (identity-like FC on 1x1 maps with a
+    decisive logit) and check indices, ids, count and the gathered rows bit for bit."""
+    K = 4
+    spec = wl.Model("mask", "f32", 1, 1, K, [wl.Stage([wl.Layer(wl.OP_CONV, K, K, 1, 1, 1, 0, wl.ACT_NONE, weight=np.eye(K, dtype=np.float32).reshape(K, 1, 1, K),
+                                                              scale=np.ones(K, np.float32), bias=np.zeros(K, np.float32))],
+                                                    K, np.eye(K, dtype=np.float32), np.zeros(K, np.float32), 0.9, False)], 8)
+    run = util.GpuRunner(spec)
+    for B in (1, 2, 5, 8):
+        for bits in itertools.product([0, 1], repeat=B):
+            x = np.zeros((B, 1, 1, K), np.float32)
+            x[:, 0, 0, 1] = np.array(bits, np.float32) * 12.0          # exits iff the decisive logit is present
+            x[:, 0, 0, 2] = np.arange(B) * 0.01                        # make rows distinguishable
+            ids = 50 + np.arange(B, dtype=np.int32)
+            g = run.stage(0, x, ids)
+            want = [b for b in range(B) if not bits[b]]
+            assert g["exit"].tolist() == list(bits)
+            assert g["surv_idx"].tolist() == want and g["n_surv"] == len(want) == B - sum(bits)
+            assert g["ids_out"].tolist() == [50 + b for b in want]
+            assert np.array_equal(g["features_out"], x[want])
+
+
+@pytest.mark.parametrize("dtype,row_elems", [("bf16", 56 * 56 * 256), ("f32", 1000), ("bf16", 8)])
+def test_gather_survivors_large_rows(dtype, row_elems):
+    td = eb.torch_dtype(dtype)
+    B = 19
+    g = torch.Generator(device="cpu").manual_seed(1)
+    feat = torch.randn((B, row_elems), generator=g).to(td).cuda()
+    mask = (torch.arange(B) % 3 == 1)
+    idx = torch.nonzero(~mask).flatten().to(torch.int32).cuda()
+    n = torch.tensor([idx.numel()], dtype=torch.int32, device="cuda")
+    idx_full = torch.zeros(B, dtype=torch.int32, device="cuda")
+    idx_full[: idx.numel()] = idx
+    out = torch.full((B, row_elems), -1.0, dtype=td, device="cuda")
+    eb.gather_survivors(feat, row_elems * feat.element_size(), idx_full, n, B, out)
+    torch.cuda.synchronize()
+    assert torch.equal(out[: idx.numel()], feat[idx.long()])
+    assert torch.all(out[idx.numel():] == -1.0)                        # rows past n_surv are untouched
+
+
+def test_refill_matches_oracle_and_clamps():
+    spec = wl.tiny_ee_cnn(seed=0)
+    m = eb.EEModel(spec)
+    info = m.query(1)
+    shape = (info["in_h"], info["in_w"], info["in_c"])
+    for n_surv, n_arr in [(0, 3), (2, 4), (6, 5), (8, 2), (3, 0)]:
+        surv = wl.random_features((n_surv,) + shape, seed=n_surv + 10, bf16=False)
+        arr = wl.random_features((n_arr,) + shape, seed=n_arr + 20, bf16=False)
+        sid, aid = np.arange(n_surv, dtype=np.int32), 40 + np.arange(n_arr, dtype=np.int32)
+        f_o, id_o, acc_o = eo.refill(surv, sid, arr, aid, spec.max_batch)
+        buf = torch.zeros((spec.max_batch,) + shape, device="cuda")
+        ids = torch.zeros(spec.max_batch, dtype=torch.int32, device="cuda")
+        buf[:n_surv] = torch.from_numpy(surv).cuda()
+        ids[:n_surv] = torch.from_numpy(sid).cuda()
+        n_acc, n_mer = m.batch_refill(1, buf, ids, n_surv, torch.from_numpy(arr).cuda(), torch.from_numpy(aid).cuda(), n_arr)
+        torch.cuda.synchronize()
+        assert (n_acc, n_mer) == (acc_o, n_surv + acc_o)
+        assert np.array_equal(buf[:n_mer].cpu().numpy(), f_o) and np.array_equal(ids[:n_mer].cpu().numpy(), id_o)
+
+
+# ----------------------------------------------------------------------------- API errors and degenerate cases
+
+def test_error_codes_and_empty_batch():
+    spec = wl.tiny_ee_cnn(seed=0)
+    run = util.GpuRunner(spec)
+    m = run.m
+    x = eb.to_device("f32", wl.make_input(spec, 8, seed=0))
+    with pytest.raises(eb.EEError) as e:
+        m.stage_run(5, x, 8, run.bufs[0], run.ws)
+    assert e.value.status == 4
+    with pytest.raises(eb.EEError) as e:
+        m.stage_run(0, x, 9, run.bufs[0], run.ws)
+    assert e.value.status == 3
+    with pytest.raises(eb.EEError) as e:
+        m.stage_run(0, x, 8, run.bufs[0], run.ws[:1024])
+    assert e.value.status == 3
+    with pytest.raises(eb.EEError) as e:
+        m.stage_run(0, None, 8, run.bufs[0], run.ws)
+    assert e.value.status == 1
+    with pytest.raises(eb.EEError) as e:
+        m.batch_refill(7, x, None, 0, x, None, 1)
+    assert e.value.status == 4
+    run.bufs[0].n_surv_dev.fill_(99)
+    m.stage_run(0, None, 0, run.bufs[0], run.ws)                       # empty batch: only the count is written
+    torch.cuda.synchronize()
+    assert int(run.bufs[0].n_surv_dev.cpu()[0]) == 0 and int(run.bufs[0].n_surv_host[0]) == 0
+    bad = wl.tiny_ee_cnn(seed=0)
+    bad.stages[1].layers[0].cin = 5                                    # does not chain
+    with pytest.raises(eb.EEError) as e:
+        eb.EEModel(bad)
+    assert e.value.status == 2
