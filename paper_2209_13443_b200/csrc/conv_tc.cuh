@@ -1,21 +1,423 @@
-// Tensor-core convolution path (tcgen05 / TMEM / TMA).  Placeholder interface: no layer is
-// claimed yet, every convolution runs on the CUDA-core kernel.
+// Tensor-core convolution for bf16 models on sm_100a: implicit GEMM on tcgen05.mma with the
+// accumulator in TMEM, both operands staged in shared memory by TMA.
+//
+// GEMM view (paper Section II-C): D[M = B*Ho*Wo][N = Cout] = A[M][K] * W[N][K]^T with
+// K = kh*kw*Cin.  The Toeplitz matrix A is never built: the TMA unit gathers each 128-pixel x
+// 64-channel tile of it straight from the NHWC feature map (im2col tensor map: one filter tap per
+// K block, zero fill for the padding halo), or reads it as a plain 2-D tile for 1x1 stride-1
+// layers.  Batching appends samples along M, so one weight tile serves every sample of the batch.
+//
+// One CTA computes one 128 x BN output tile.  Warp roles: warp 0 issues TMA loads into a ring of
+// shared-memory stages, warp 1 owns the TMEM allocation and issues the MMAs (one thread), warps
+// 2-5 run the epilogue: tcgen05.ld of the fp32 accumulator, folded-BN scale/bias, residual add,
+// activation, one rounding to bf16, 16-byte stores.  The K loop visits (tap, channel block) in a
+// fixed order that does not depend on the batch size.
+//
+// Every wait on an mbarrier is bounded by a clock: on expiry the thread records EE_ERR_TIMEOUT in
+// the model's error word and falls through to the common exit, which frees the TMEM columns.
 #pragma once
+#include <cuda.h>
+
+#include <vector>
+
 #include "common.cuh"
 
 namespace ee {
 
-struct TcContext {};
-struct TcLayer {};
+constexpr int kTcBM = 128;       // output pixels per CTA (= TMEM lanes)
+constexpr int kTcBK = 64;        // bf16 elements per K block: 128 bytes = one swizzle span
+constexpr int kTcStages = 4;
+constexpr int kTcThreads = 192;  // producer warp, MMA warp, four epilogue warps
+constexpr long long kTcWaitCycles = 4000000000LL;  // ~2 s at boost clock; far beyond any healthy wait
 
-inline ee_status_t tc_context_init(TcContext&) { return EE_OK; }
-inline bool tc_supported(const ee_layer_desc_t&, int, int) { return false; }
-inline ee_status_t tc_plan_layer(TcContext&, const ee_layer_desc_t&, int, int, int, int, int, const void*, TcLayer*) {
-  return EE_ERR_UNSUPPORTED;
+struct TcParams {
+  int M, N;             // valid rows (B*Ho*Wo) and Cout
+  int taps, kw;         // kh*kw and kw
+  int cblocks;          // Cin / 64
+  int Ho, Wo, stride, pad;
+  int im2col;           // 0: A is a plain [rows][Cin] matrix, 1: im2col tensor map
+  int act;
+  const float* scale;
+  const float* bias;
+  const bf16* residual;
+  bf16* out;
+  int* err_flag;
+};
+
+// ----------------------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
-inline ee_status_t tc_launch(TcContext&, const TcLayer&, const void*, const void*, void*, int, const float*, const float*,
-                             int*, cudaStream_t) {
-  return EE_ERR_UNSUPPORTED;
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (and records the fault) if the phase did not complete in time.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* err_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > kTcWaitCycles) {
+      atomicExch(err_flag, (int)EE_ERR_TIMEOUT);
+      return false;
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1)
+               : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+               ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
+// im2col gather: 128 consecutive output pixels starting at base pixel (w, h, n), channels [c, c+64), filter tap (woff, hoff).
+__device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c, int w, int h, int n,
+                                                   uint16_t woff, uint16_t hoff) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(woff), "h"(hoff)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major tile, rows of 128 bytes, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);   // start address
+  d |= (uint64_t)(1024 >> 4) << 32;              // stride between 8-row groups
+  d |= (uint64_t)1 << 46;                        // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                        // 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__host__ __device__ constexpr uint32_t umma_idesc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane.  Load and wait sit in one statement so that no
+// use of the registers can be scheduled before the wait.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+
+// ----------------------------------------------------------------------------- kernel
+
+template <int BN>
+struct TcSmem {
+  static constexpr int kABytes = kTcBM * kTcBK * 2;
+  static constexpr int kBBytes = BN * kTcBK * 2;
+  static constexpr int kStage = kABytes + kBBytes;
+  static constexpr int kTiles = kTcStages * kStage;
+  static constexpr int kBytes = kTiles + 2 * BN * 4 + 256 + 1024;  // tiles, scale/bias, barriers, alignment slack
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kTcThreads, 1)
+conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  using S = TcSmem<BN>;
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
+  uint8_t* gen = smem_raw + (base - raw);
+  float* s_scale = reinterpret_cast<float*>(gen + S::kTiles);
+  float* s_bias = s_scale + BN;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kTiles + 2 * BN * 4);
+  const uint32_t bar0 = base + S::kTiles + 2 * BN * 4;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kTcStages + s); };
+  const uint32_t accum_bar = bar0 + 8u * (2 * kTcStages);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * kTcBM, n0 = blockIdx.y * BN;
+  const int num_kb = p.taps * p.cblocks;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kTcStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    mbar_init(accum_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // TMEM: BN fp32 columns x 128 lanes
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int cw = 0, ch = 0, cn = 0;
+      if (p.im2col) {
+        const int hw = p.Ho * p.Wo;
+        cn = m0 / hw;
+        const int rem = m0 - cn * hw;
+        const int ho = rem / p.Wo;
+        cw = (rem - ho * p.Wo) * p.stride - p.pad;
+        ch = ho * p.stride - p.pad;
+      }
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % kTcStages;
+        const uint32_t ph = (uint32_t)(kb / kTcStages) & 1u;
+        if (!mbar_wait(empty_bar(s), ph ^ 1u, p.err_flag)) break;
+        const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
+        const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
+        mbar_expect_tx(full_bar(s), S::kStage);
+        if (p.im2col) {
+          const int r = tap / p.kw;
+          tma_load_im2col_4d(sa, &tmA, full_bar(s), cb * kTcBK, cw, ch, cn, (uint16_t)(tap - r * p.kw), (uint16_t)r);
+        } else {
+          tma_load_2d(sa, &tmA, full_bar(s), cb * kTcBK, m0);
+        }
+        tma_load_3d(sb, &tmW, full_bar(s), cb * kTcBK, tap, n0);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc(BN);
+      bool ok = true;
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % kTcStages;
+        const uint32_t ph = (uint32_t)(kb / kTcStages) & 1u;
+        ok = mbar_wait(full_bar(s), ph, p.err_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
+#pragma unroll
+        for (int k = 0; k < kTcBK / 16; ++k)
+          umma_bf16(tmem_base, umma_desc(sa + k * 32), umma_desc(sb + k * 32), idesc, (uint32_t)((kb | k) != 0));
+        umma_commit(empty_bar(s));  // frees the stage once these MMAs have read it
+      }
+      if (ok) umma_commit(accum_bar);  // accumulator complete
+    }
+  } else {
+    const int et = threadIdx.x - 64;  // 0..127
+    for (int i = et; i < BN; i += 128) {
+      s_scale[i] = p.scale ? p.scale[n0 + i] : 1.f;
+      s_bias[i] = p.bias ? p.bias[n0 + i] : 0.f;
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    // warp-uniform outcome: tcgen05.ld is a warp-wide instruction
+    const bool ok = __all_sync(0xffffffffu, mbar_wait(accum_bar, 0, p.err_flag));
+    tc_fence_after();
+    if (ok) {
+      const int q = warp & 3;  // TMEM lane quarter this warp may read
+      const int m = m0 + q * 32 + lane;
+      const size_t row = (size_t)m * p.N + n0;
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        float v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+        if (m < p.M) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = fmaf(s_scale[c0 + j], v[j], s_bias[c0 + j]);
+          if (p.residual) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              Vec16<bf16> r;
+              r.load(p.residual + row + c0 + g * 8);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) v[g * 8 + e] += r.v[e];
+            }
+          }
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            Vec16<bf16> o;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) o.v[e] = apply_act(v[g * 8 + e], p.act);
+            o.store(p.out + row + c0 + g * 8);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
+  }
+}
+
+// ----------------------------------------------------------------------------- host side
+
+typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+typedef CUresult (*PFN_encodeIm2col)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                     const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*, CUtensorMapInterleave,
+                                     CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TcContext {
+  PFN_encodeTiled encode_tiled = nullptr;
+  PFN_encodeIm2col encode_im2col = nullptr;
+};
+
+struct TcLayer {
+  int cin = 0, cout = 0, kh = 1, kw = 1, stride = 1, pad = 0, act = 0;
+  int in_h = 0, in_w = 0, out_h = 0, out_w = 0, max_batch = 0;
+  int bn = 128;
+  bool im2col = false;
+  CUtensorMap tm_w;
+  struct Cached {
+    const void* ptr;
+    int batch;
+    CUtensorMap tm;
+  };
+  mutable std::vector<Cached> a_maps;  // activation tensor maps by (source pointer, batch)
+  mutable size_t next_evict = 0;
+};
+
+inline ee_status_t tc_context_init(TcContext& c) {
+  cudaDriverEntryPointQueryResult q;
+  void* f = nullptr;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess || !f) return EE_ERR_CUDA;
+  c.encode_tiled = (PFN_encodeTiled)f;
+  f = nullptr;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f, cudaEnableDefault, &q) != cudaSuccess || !f) return EE_ERR_CUDA;
+  c.encode_im2col = (PFN_encodeIm2col)f;
+  if (cudaFuncSetAttribute(conv_igemm_tcgen05_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<64>::kBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(conv_igemm_tcgen05_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<128>::kBytes) != cudaSuccess)
+    return EE_ERR_CUDA;
+  return EE_OK;
+}
+
+// Layers this path covers: dense convolutions whose channel counts fill whole 64-wide K blocks and N tiles.
+inline bool tc_supported(const ee_layer_desc_t& d, int in_h, int in_w) {
+  (void)in_h;
+  (void)in_w;
+  return d.op == EE_OP_CONV && d.cin % kTcBK == 0 && d.cout % 64 == 0 && d.kh == d.kw && d.kh <= 7 && d.stride <= 8 &&
+         d.pad < d.kh && d.pad <= 127;
+}
+
+inline ee_status_t tc_plan_layer(TcContext& c, const ee_layer_desc_t& d, int in_h, int in_w, int out_h, int out_w, int max_batch,
+                                 const void* w_dev, TcLayer* L) {
+  L->cin = d.cin, L->cout = d.cout, L->kh = d.kh, L->kw = d.kw, L->stride = d.stride, L->pad = d.pad, L->act = d.act;
+  L->in_h = in_h, L->in_w = in_w, L->out_h = out_h, L->out_w = out_w, L->max_batch = max_batch;
+  L->bn = d.cout % 128 == 0 ? 128 : 64;
+  L->im2col = !(d.kh == 1 && d.stride == 1 && d.pad == 0);
+  // weights [Cout][taps][Cin] as a 3-D tensor, box = 64 channels x 1 tap x BN filters
+  const cuuint64_t dims[3] = {(cuuint64_t)d.cin, (cuuint64_t)(d.kh * d.kw), (cuuint64_t)d.cout};
+  const cuuint64_t strides[2] = {(cuuint64_t)d.cin * 2, (cuuint64_t)d.cin * d.kh * d.kw * 2};
+  const cuuint32_t box[3] = {kTcBK, 1, (cuuint32_t)L->bn};
+  const cuuint32_t es[3] = {1, 1, 1};
+  CUresult r = c.encode_tiled(&L->tm_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(w_dev), dims, strides, box, es,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? EE_OK : EE_ERR_CUDA;
+}
+
+// The map covers exactly `batch` samples: rows past them are out of bounds for the TMA unit and read as zero,
+// so no byte beyond the caller's [batch] samples is ever touched.
+inline ee_status_t tc_activation_map(const TcContext& c, const TcLayer& L, const void* src, int batch, const CUtensorMap** out) {
+  for (auto& e : L.a_maps)
+    if (e.ptr == src && e.batch == batch) {
+      *out = &e.tm;
+      return EE_OK;
+    }
+  TcLayer::Cached e;
+  e.ptr = src;
+  e.batch = batch;
+  CUresult r;
+  if (!L.im2col) {
+    const cuuint64_t dims[2] = {(cuuint64_t)L.cin, (cuuint64_t)batch * L.in_h * L.in_w};
+    const cuuint64_t strides[1] = {(cuuint64_t)L.cin * 2};
+    const cuuint32_t box[2] = {kTcBK, kTcBM};
+    const cuuint32_t es[2] = {1, 1};
+    r = c.encode_tiled(&e.tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(src), dims, strides, box, es,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else {
+    // NHWC as (C, W, H, N).  Base pixels (filter tap 0,0) range over [-pad, dim - 1 + pad - (k - 1)] in steps of `stride`.
+    const cuuint64_t dims[4] = {(cuuint64_t)L.cin, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)batch};
+    const cuuint64_t strides[3] = {(cuuint64_t)L.cin * 2, (cuuint64_t)L.cin * 2 * L.in_w, (cuuint64_t)L.cin * 2 * L.in_w * L.in_h};
+    const int lower[2] = {-L.pad, -L.pad};
+    const int upper[2] = {L.pad - (L.kw - 1), L.pad - (L.kh - 1)};
+    const cuuint32_t es[4] = {1, (cuuint32_t)L.stride, (cuuint32_t)L.stride, 1};
+    r = c.encode_im2col(&e.tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(src), dims, strides, lower, upper, kTcBK,
+                        kTcBM, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
+  if (r != CUDA_SUCCESS) return EE_ERR_CUDA;
+  if (L.a_maps.size() < 16) {
+    L.a_maps.push_back(e);
+    *out = &L.a_maps.back().tm;
+  } else {
+    L.a_maps[L.next_evict] = e;
+    *out = &L.a_maps[L.next_evict].tm;
+    L.next_evict = (L.next_evict + 1) % L.a_maps.size();
+  }
+  return EE_OK;
+}
+
+inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, const void* res, void* dst, int B, const float* scale,
+                             const float* bias, int* err_flag, cudaStream_t st) {
+  if (((uintptr_t)src & 15) || ((uintptr_t)dst & 15) || ((uintptr_t)res & 15)) return EE_ERR_INVALID_ARG;
+  const CUtensorMap* tmA = nullptr;
+  ee_status_t s = tc_activation_map(c, L, src, B, &tmA);
+  if (s != EE_OK) return s;
+  TcParams p;
+  p.M = B * L.out_h * L.out_w;
+  p.N = L.cout;
+  p.taps = L.kh * L.kw;
+  p.kw = L.kw;
+  p.cblocks = L.cin / kTcBK;
+  p.Ho = L.out_h, p.Wo = L.out_w, p.stride = L.stride, p.pad = L.pad;
+  p.im2col = L.im2col ? 1 : 0;
+  p.act = L.act;
+  p.scale = scale, p.bias = bias;
+  p.residual = (const bf16*)res;
+  p.out = (bf16*)dst;
+  p.err_flag = err_flag;
+  dim3 grid(cdiv(p.M, kTcBM), L.cout / L.bn);
+  if (L.bn == 128)
+    conv_igemm_tcgen05_kernel<128><<<grid, kTcThreads, TcSmem<128>::kBytes, st>>>(*tmA, L.tm_w, p);
+  else
+    conv_igemm_tcgen05_kernel<64><<<grid, kTcThreads, TcSmem<64>::kBytes, st>>>(*tmA, L.tm_w, p);
+  return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
 }
 
 }  // namespace ee

@@ -146,6 +146,12 @@ def _conv(rng, op, cin, cout, k, stride, pad, act, *, gamma=1.0, jitter=True, bf
     return Layer(op, cin, cout, k, k, stride, pad, act, input_from, residual_from, w, scale, bias)
 
 
+def head_weights(seed: int, stream: int, c: int, n_classes: int, alpha: float, bf16: bool):
+    """FC head of one exit from its own random stream, so that it can be regenerated for another
+    scale factor ``alpha`` without touching the backbone weights."""
+    return _head(_rng(seed, 5000 + stream), c, n_classes, alpha, bf16)
+
+
 def _head(rng, c, n_classes, alpha, bf16):
     w = rng.standard_normal((n_classes, c), dtype=np.float32) * np.float32(alpha / np.sqrt(c))
     b = (0.01 * rng.standard_normal(n_classes)).astype(np.float32)
@@ -230,7 +236,7 @@ def resnet50_ee(seed: int = 1, max_batch: int = 64, alphas=None, thresholds=(0.5
             idx = _bottleneck(rng, layers, cin, width, 2 if (b == 0 and s > 0) else 1, b == 0, bf16, idx)
             cin = 4 * width
         last = s == len(blocks) - 1
-        fw, fb = _head(rng, cin, n_classes, alphas[s], bf16)
+        fw, fb = head_weights(seed, 200 + s, cin, n_classes, alphas[s], bf16)
         stages.append(Stage(layers, n_classes, fw, fb, 1.0 if last else thresholds[s], last))
     return Model("resnet50_ee", dtype, in_hw, in_hw, 3, stages, max_batch,
                  {"seed": seed, "alphas": list(alphas), "thresholds": list(thresholds)})
@@ -285,7 +291,7 @@ def mobilenetv2_ee(seed: int = 2, max_batch: int = 32, alphas=None, threshold: f
         if last:
             layers.append(_conv(rng, OP_CONV, c_out, 1280, 1, 1, 0, ACT_RELU6, bf16=bf16))
             c_out = 1280
-        fw, fb = _head(rng, c_out, n_classes, alphas[s], bf16)
+        fw, fb = head_weights(seed, 300 + s, c_out, n_classes, alphas[s], bf16)
         stages.append(Stage(layers, n_classes, fw, fb, 1.0 if last else threshold, last))
         b0 = b1
     return Model("mobilenetv2_ee", dtype, in_hw, in_hw, 3, stages, max_batch,
