@@ -1,0 +1,365 @@
+"""Throughput of the early-exit CNN stage executor on B200: samples/s of the whole hot path.
+
+One "step" is one pass of the whole path over one batch of synthetic requests:
+  ee_batch_refill (the arrivals are appended to the empty batch buffer) -> for every stage:
+  ee_stage_run (convolutions, exit head, threshold, compaction + gather of the survivors) ->
+  the survivor count reaches the host (pinned word + stream sync) and sizes the next stage.
+The batch shrinks stage by stage at the calibrated exit rates, exactly as in serving.
+
+Default workload (N = 1): the ResNet-50-shaped 4-exit model, bf16, batch 64, 224x224 inputs.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--batch B] [--workload resnet50|mobilenetv2|tiny]
+  python bench.py --impl reference ...     # the CPU oracle timed on the host cores (bounded sample)
+
+Prints ONE JSON line (rank 0).  With N > 1 every rank runs an independent replica on its own
+GPU (samples are independent; there is no collective on the data path) and the time is the max
+over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "EE-CNN samples/sec on 1 B200 vs exit rate & batch 1-64; tensor-pipe % of peak"
+UNIT = "samples/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "tf_burst": d["bf16_tflops"], "tf_sustained": d["bf16_tflops_sustained"], "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tf_burst": 1590.0, "tf_sustained": 1400.0, "source": "fallback"}
+
+
+def make_spec(workload: str, batch: int):
+    from paper_2209_13443_b200 import workloads as wl
+
+    if workload == "resnet50":
+        return wl.resnet50_ee(seed=1, max_batch=batch), 1
+    if workload == "mobilenetv2":
+        return wl.mobilenetv2_ee(seed=2, max_batch=batch), 2
+    if workload == "tiny":
+        return wl.tiny_ee_cnn(seed=0, max_batch=batch), 0
+    raise SystemExit(f"unknown workload {workload}")
+
+
+def workload_name(spec, batch):
+    return f"{spec.name} {spec.dtype} B={batch} {spec.in_h}x{spec.in_w}x{spec.in_c}, {len(spec.stages)} exits, calibrated exit rates"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.lines, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- reference arm (CPU oracle)
+
+def oracle_pass(spec, x, ids):
+    """The whole path on the CPU oracle for the samples in ``x``; returns the per-stage batch sizes."""
+    from oracle import ee_oracle as eo
+
+    sizes = []
+    for s in range(len(spec.stages)):
+        sizes.append(len(ids))
+        r = eo.run_stage(spec, s, x, ids)
+        x, ids = r["features_out"], r["ids_out"]
+        if len(ids) == 0:
+            break
+    return sizes
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import ee_oracle as eo
+    from paper_2209_13443_b200 import workloads as wl
+
+    spec, seed = make_spec(args.workload, args.batch)
+    x_all = wl.make_input(spec, args.batch, seed=seed)
+    ids_all = np.arange(args.batch, dtype=np.int32)
+    t0 = time.perf_counter()
+    oracle_pass(spec, x_all[:1], ids_all[:1])
+    t1 = max(time.perf_counter() - t0, 1e-4)
+    budget = 150.0                                         # seconds for the whole run
+    n = int(max(1, min(args.batch, budget / ((args.steps + args.warmup) * t1))))
+    for _ in range(args.warmup):
+        oracle_pass(spec, x_all[:n], ids_all[:n])
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_pass(spec, x_all[:n], ids_all[:n])
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    cores = eo.n_threads()
+    sample = f"first {n} of {args.batch} samples per step, whole path (all stages, heads, compaction), fp64 oracle as it stands"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(spec, args.batch)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ----------------------------------------------------------------------------- our arm
+
+def run_ours(args):
+    import torch
+
+    from paper_2209_13443_b200 import binding as eb
+    from paper_2209_13443_b200 import workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = load_peaks()
+    B, K, W = args.batch, args.steps, max(args.warmup, 3)
+    spec, seed = make_spec(args.workload, B)
+    model = eb.EEModel(spec)
+    nst = model.n_stages
+    bufs = [eb.StageBuffers(model, s, with_logits=False) for s in range(nst)]
+    ws = model.workspace()
+    td = eb.torch_dtype(spec.dtype)
+    # every rank serves its own requests (ids are global)
+    x_host = torch.from_numpy(wl.make_input(spec, B, seed=seed, first_id=rank * B)).to(td).pin_memory()
+    ids_host = (torch.arange(B, dtype=torch.int32) + rank * B).pin_memory()
+    x_dev, ids_dev = x_host.cuda(), ids_host.cuda()
+    batch0 = torch.empty_like(x_dev)
+    ids0 = torch.empty_like(ids_dev)
+    res_host = [dict(conf=torch.empty(B).pin_memory(), pred=torch.empty(B, dtype=torch.int32).pin_memory(),
+                     mask=torch.empty(B, dtype=torch.uint8).pin_memory()) for _ in range(nst)]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # larger than the 126 MB L2
+    stream = torch.cuda.current_stream()
+    launches = [0]
+    sizes_last = []
+
+    def step(e2e: bool):
+        """One pass of the whole path.  Returns (#kernel launches, h2d bytes, d2h bytes, per-stage batch)."""
+        h2d = d2h = 0
+        if e2e:
+            x_dev.copy_(x_host, non_blocking=True)
+            ids_dev.copy_(ids_host, non_blocking=True)
+            h2d = x_host.numel() * x_host.element_size() + ids_host.numel() * 4
+        n_acc, n = model.batch_refill(0, batch0, ids0, 0, x_dev, ids_dev, B)
+        nl = 1
+        feat, ids = batch0, ids0
+        sizes = []
+        for s in range(nst):
+            sizes.append(n)
+            model.stage_run(s, feat, n, bufs[s], ws, ids)
+            nl += len(spec.stages[s].layers) + 3 + (0 if spec.stages[s].always_exit else 1)
+            if e2e:
+                res_host[s]["conf"][:n].copy_(bufs[s].conf[:n], non_blocking=True)
+                res_host[s]["pred"][:n].copy_(bufs[s].pred[:n], non_blocking=True)
+                res_host[s]["mask"][:n].copy_(bufs[s].exit_mask[:n], non_blocking=True)
+                d2h += n * 9 + 4
+            stream.synchronize()                           # B_exit reaches the host: it sizes the next launch
+            n = int(bufs[s].n_surv_host[0])
+            feat, ids = bufs[s].features_out, bufs[s].ids_out
+            if n == 0:
+                break
+        return nl, h2d, d2h, sizes
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(e2e: bool, steps: int):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        nl = h2d = d2h = 0
+        sizes = []
+        barrier()
+        for a, b in ev:
+            flush.zero_()                                   # evict L2 between timed iterations (not timed)
+            a.record()
+            l, hi, do, sizes = step(e2e)
+            b.record()
+            nl += l; h2d = hi; d2h = do
+        barrier()
+        total_ms = sum(a.elapsed_time(b) for a, b in ev)
+        if dist is not None:
+            t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            total_ms = float(t.item())
+        return total_ms, nl, h2d, d2h, sizes
+
+    for _ in range(W):
+        step(False)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    total_ms, nl, _, _, sizes_last = timed(False, K)
+    clocks = sampler.stop() if rank == 0 else None
+    for _ in range(2):
+        step(True)
+    e2e_ms, _, h2d, d2h, _ = timed(True, K)
+
+    # instrumented pass: per-kernel device time by CUDA events on the launching stream
+    model.set_timing(True)
+    fam = {}
+    inst_ms = 0.0
+    for _ in range(K):
+        flush.zero_()
+        model.batch_refill(0, batch0, ids0, 0, x_dev, ids_dev, B)
+        feat, ids, n = batch0, ids0, B
+        for s in range(nst):
+            model.stage_run(s, feat, n, bufs[s], ws, ids)
+            stream.synchronize()
+            plan = model.plan(s, n)
+            tm = model.get_timing(s)
+            for i, (name, ms) in enumerate(tm):
+                f = fam.setdefault(name, {"ms": 0.0, "launches": 0, "flops": 0.0, "bytes": 0.0})
+                f["ms"] += ms; f["launches"] += 1
+                inst_ms += ms
+                if i < len(plan):
+                    f["flops"] += plan[i]["flops"]; f["bytes"] += plan[i]["bytes"]
+            info = model.query(s)
+            ns = int(bufs[s].n_surv_host[0])
+            es = 2 if spec.dtype == "bf16" else 4
+            fam["head_gap"]["bytes"] += n * info["out_bytes_per_sample"]
+            fam["head_fc"]["bytes"] += info["out_c"] * spec.stages[s].n_classes * es + n * info["out_c"] * 4
+            if "gather_survivors" in fam and not spec.stages[s].always_exit:
+                fam["gather_survivors"]["bytes"] += 2 * ns * info["out_bytes_per_sample"]
+            n = ns
+            feat, ids = bufs[s].features_out, bufs[s].ids_out
+            if n == 0:
+                break
+    model.set_timing(False)
+    model.check()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    kernels = {}
+    for name, f in fam.items():
+        sec = f["ms"] * 1e-3
+        kernels[name] = {"launches_per_step": f["launches"] / K, "ms_per_step": f["ms"] / K,
+                         "tflops": f["flops"] / sec / 1e12 if sec > 0 else 0.0, "gbs": f["bytes"] / sec / 1e9 if sec > 0 else 0.0,
+                         "share": f["ms"] / inst_ms if inst_ms else 0.0}
+    dom = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
+    if dom.startswith("conv_igemm_tcgen05"):
+        roof = {"bound": "tensor", "kernel": dom, "achieved": kernels[dom]["tflops"], "peak": peaks["tf_sustained"], "unit": "TFLOP/s",
+                "peak_source": f"bf16 sustained, {peaks['source']}"}
+    else:
+        roof = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "peak_source": f"copy bandwidth, {peaks['source']}"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = None
+    roof["avg_launch_ms"] = fam[dom]["ms"] / max(fam[dom]["launches"], 1)
+    roof["per_launch"] = (fam[dom]["flops"] if roof["bound"] == "tensor" else fam[dom]["bytes"]) / max(fam[dom]["launches"], 1)
+    roof["hbm_kernels"] = {k: {"gbs": kernels[k]["gbs"], "frac": kernels[k]["gbs"] / peaks["hbm_gbs"]}
+                           for k in ("head_gap", "gather_survivors", "maxpool", "dwconv") if k in kernels}
+
+    # CPU baseline: the oracle as it stands on a bounded sample of the same workload
+    from oracle import ee_oracle as eo
+
+    n_cpu = min(B, args.cpu_samples)
+    x_np = x_host[:n_cpu].float().numpy()
+    t0 = time.perf_counter()
+    oracle_pass(spec, x_np, np.arange(n_cpu, dtype=np.int32))
+    cpu_dt = time.perf_counter() - t0
+    cpu = {"value": n_cpu / cpu_dt, "unit": UNIT, "cores": eo.n_threads(), "kind": "oracle",
+           "sample": f"first {n_cpu} of {B} samples, whole path once, {cpu_dt:.1f} s"}
+
+    value = world * B * K / (total_ms * 1e-3)
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": spec.dtype, "data": "synthetic",
+        "config": {"workload": workload_name(spec, B), "global_batch": world * B, "parallelism": f"replicas x{world}",
+                   "l2": "flushed between timed steps (256 MB write)", "batch_per_stage": sizes_last},
+        "clocks": clocks,
+        "e2e": {"value": world * B * K / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms / K},
+        "gpu_launches": nl,
+        "roofline": roof,
+        "cpu_baseline": cpu,
+        "kernels": kernels,
+        "instrumented_ms_per_step": inst_ms / K,
+    }
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=64)
+    ap.add_argument("--workload", default="resnet50", choices=["resnet50", "mobilenetv2", "tiny"])
+    ap.add_argument("--cpu-samples", type=int, default=16)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
