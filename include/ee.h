@@ -175,6 +175,27 @@ ee_status_t ee_exit_head(ee_model_t* model, int stage, const void* x, int batch,
                          const ee_stage_out_t* out, void* cuda_stream);
 size_t ee_exit_head_scratch_bytes(const ee_model_t* model, int stage);
 
+/* ee_exit_head without any caller scratch and without any allocation.  The paper has no counterpart: this is
+ * a convenience of this library.  It is for callers that may not allocate device memory when they need an exit
+ * decision: code living inside a host application that hands out all device memory at start-up and forbids
+ * later cudaMalloc calls (inference-server plug-ins, engines running under a fixed memory budget), and latency-bound
+ * serving threads, for which an allocation's implicit synchronisation and unpredictable duration are not
+ * acceptable.  Same arguments, results and errors as ee_exit_head, minus `scratch`: the partial sums, pooled vectors,
+ * logits (when out->logits is NULL) and counters go to an array of EE_STATIC_HEAD_SCRATCH_BYTES bytes that is part of
+ * the library image (each GPU that loads the library holds it until the process exits).
+ *   - A model/shape whose head needs more than EE_STATIC_HEAD_SCRATCH_BYTES (what ee_exit_head_scratch_bytes reports
+ *     for the stage's own hw) is refused with EE_ERR_CAPACITY and an explanatory ee_last_cuda_error() text.
+ *   - The first call on a device resolves the array's device address (the calling thread's current device must be the
+ *     one the model lives on); make that first call outside any stream capture.
+ *   - No cudaMalloc / cudaFree or allocating library routine is called.
+ *   - All calls, from every model and stream, share the one array and it keeps the previous call's contents; the call
+ *     clears what has to start at zero.  Two calls whose kernels overlap on the GPU race on it: serialise them
+ *     (same stream, or an event between streams). */
+#define EE_STATIC_HEAD_SCRATCH_BYTES (8u << 20)
+ee_status_t ee_exit_head_static(ee_model_t* model, int stage, const void* x, int batch, int hw,
+                                const float* logit_shift, const int32_t* shift_class, const ee_stage_out_t* out,
+                                void* cuda_stream);
+
 /* Stable compaction + gather alone: feat_out[j] = feat[survivor_idx[j]] for j < *n_surv_dev
  * (both read from DEVICE memory, no host round trip).  Rows move as 16-byte vectors when bytes_per_sample
  * and both base addresses are multiples of 16, in narrower units otherwise.

@@ -20,7 +20,7 @@ EE_OK = 0
 STATUS_NAMES = ["EE_OK", "EE_ERR_INVALID_ARG", "EE_ERR_SHAPE", "EE_ERR_CAPACITY", "EE_ERR_STAGE", "EE_ERR_UNSUPPORTED",
                 "EE_ERR_CUDA", "EE_ERR_TIMEOUT", "EE_ERR_INTERNAL"]
 EXPORTS = ["ee_model_create", "ee_model_destroy", "ee_model_query", "ee_stage_run", "ee_batch_refill", "ee_exit_head",
-           "ee_exit_head_scratch_bytes", "ee_gather_survivors", "ee_model_set_timing", "ee_model_get_timing",
+           "ee_exit_head_scratch_bytes", "ee_exit_head_static", "ee_gather_survivors", "ee_model_set_timing", "ee_model_get_timing",
            "ee_model_plan", "ee_model_check", "ee_status_string", "ee_last_cuda_error"]
 
 
@@ -87,6 +87,7 @@ def load_library() -> C.CDLL:
     L.ee_stage_run.argtypes = [vp, i, C.POINTER(StageIn), vp, C.c_size_t, C.POINTER(StageOut), vp]
     L.ee_batch_refill.argtypes = [vp, i, vp, vp, i, vp, vp, i, C.POINTER(i), C.POINTER(i), vp]
     L.ee_exit_head.argtypes = [vp, i, vp, i, i, vp, vp, vp, C.c_size_t, C.POINTER(StageOut), vp]
+    L.ee_exit_head_static.argtypes = [vp, i, vp, i, i, vp, vp, C.POINTER(StageOut), vp]
     L.ee_exit_head_scratch_bytes.argtypes = [vp, i]
     L.ee_exit_head_scratch_bytes.restype = C.c_size_t
     L.ee_gather_survivors.argtypes = [vp, C.c_size_t, vp, vp, i, vp, vp]
@@ -237,6 +238,14 @@ class EEModel:
         so = out.as_struct() if isinstance(out, StageBuffers) else out
         _check(self._L.ee_exit_head(self._h, stage, _ptr(x), int(batch), int(hw), _ptr(logit_shift), _ptr(shift_class), aligned,
                                     scratch.numel() - (aligned - base), C.byref(so), _stream(stream)), "ee_exit_head")
+
+    def exit_head_static(self, stage: int, x, batch: int, hw: int, out: StageBuffers, logit_shift=None, shift_class=None,
+                         stream=None):
+        """ee_exit_head on the library's built-in scratch array: nothing is allocated, here or in the library.
+        For callers that must not allocate device memory at decision time; calls that overlap on the GPU race."""
+        so = out.as_struct() if isinstance(out, StageBuffers) else out
+        _check(self._L.ee_exit_head_static(self._h, stage, _ptr(x), int(batch), int(hw), _ptr(logit_shift), _ptr(shift_class),
+                                           C.byref(so), _stream(stream)), "ee_exit_head_static")
 
     def set_timing(self, enabled: bool):
         _check(self._L.ee_model_set_timing(self._h, int(enabled)), "ee_model_set_timing")

@@ -560,6 +560,50 @@ ee_status_t ee_exit_head(ee_model_t* m, int stage, const void* x, int batch, int
              : launch_head<float>(m, sp, x, batch, hw, logit_shift, shift_class, (char*)scratch, nullptr, out, st, false);
 }
 
+// Scratch of ee_exit_head_static: lives in the library image, so every GPU that loads the library holds these
+// bytes until the process exits.  In host code this name is only a handle for the runtime, never a device address.
+static __device__ __align__(256) unsigned char g_static_head_scratch[EE_STATIC_HEAD_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_head_ptr[kMaxDevices];   // device address of the array, resolved once per device
+}  // namespace
+
+ee_status_t ee_exit_head_static(ee_model_t* m, int stage, const void* x, int batch, int hw, const float* logit_shift,
+                                const int32_t* shift_class, const ee_stage_out_t* out, void* cuda_stream) {
+  if (!m || !valid_out(out, false) || batch < 0 || hw < 1) return EE_ERR_INVALID_ARG;
+  if (stage < 0 || stage >= (int)m->stages.size()) return EE_ERR_STAGE;
+  if (logit_shift && !shift_class) return EE_ERR_INVALID_ARG;
+  StagePlan& sp = m->stages[stage];
+  if (batch > m->max_batch) return EE_ERR_CAPACITY;
+  HeadLayout hl = head_layout(m->max_batch, hw, sp.out_c, sp.n_classes, esize(m->dtype));
+  if (hl.bytes > (size_t)EE_STATIC_HEAD_SCRATCH_BYTES) {
+    g_cuda_err = "ee_exit_head_static: this model/shape needs " + std::to_string(hl.bytes) + " scratch bytes, the built-in array holds " +
+                 std::to_string((size_t)EE_STATIC_HEAD_SCRATCH_BYTES);
+    return EE_ERR_CAPACITY;
+  }
+  int dev = -1;
+  EE_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return EE_ERR_UNSUPPORTED;
+  if (!g_static_head_ptr[dev]) {  // first call on this device (the device is current): ask the runtime where the array lives
+    void* ptr = nullptr;
+    EE_CUDA(cudaGetSymbolAddress(&ptr, g_static_head_scratch));
+    if (!ptr) return EE_ERR_INTERNAL;
+    g_static_head_ptr[dev] = ptr;
+  }
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (batch == 0) {
+    EE_CUDA(cudaMemsetAsync(out->n_surv_dev, 0, sizeof(int32_t), st));
+    return EE_OK;
+  }
+  if (!x) return EE_ERR_INVALID_ARG;
+  char* scratch = (char*)g_static_head_ptr[dev];
+  // launch_head zeroes the per-sample counters it needs; everything else in the array is overwritten before it is read
+  return m->dtype == EE_BF16
+             ? launch_head<bf16>(m, sp, x, batch, hw, logit_shift, shift_class, scratch, nullptr, out, st, false)
+             : launch_head<float>(m, sp, x, batch, hw, logit_shift, shift_class, scratch, nullptr, out, st, false);
+}
+
 ee_status_t ee_gather_survivors(const void* feat, size_t bytes_per_sample, const int32_t* survivor_idx, const int32_t* n_surv_dev,
                                 int max_rows, void* feat_out, void* cuda_stream) {
   if (!feat || !survivor_idx || !n_surv_dev || !feat_out || max_rows < 0) return EE_ERR_INVALID_ARG;

@@ -1,0 +1,65 @@
+"""ee_exit_head_static: the exit head on the library's built-in scratch array.
+
+Some users of this library cannot allocate device memory at the moment they need an exit decision (a host
+application that owns all device memory and forbids later cudaMalloc calls, or a latency-bound serving thread).
+For them the library carries its own fixed scratch array.  This test drives the entry point through the C ABI and
+holds it to the existing ee_exit_head on the same inputs, twice in a row with different batches, so that whatever
+the first call left behind in the shared array must not leak into the second.  Collected last on purpose."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2209_13443_b200 import binding as eb
+from paper_2209_13443_b200 import workloads as wl
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+def _head_model(dtype, HW, C, K, max_batch):
+    rng = wl._rng(C + K, 903)
+    bf16 = dtype == "bf16"
+    fw, fb = wl._head(rng, C, K, 0.5, bf16)          # flat logits: only the shifted samples reach the threshold
+    layers = [wl._conv(rng, wl.OP_CONV, C, C, 1, 1, 0, wl.ACT_NONE, bf16=bf16)]
+    return wl.Model("head", dtype, 1, HW, C, [wl.Stage(layers, K, fw, fb, 0.5, False)], max_batch)
+
+
+def _run(m, out, fn, x, B, HW, shift, cls):
+    out.logits.fill_(float("nan"))
+    out.n_surv_dev.fill_(-1)
+    fn(0, x, B, HW, out, logit_shift=shift, shift_class=cls)
+    torch.cuda.synchronize()
+    n = int(out.n_surv_dev.cpu()[0])
+    return {"z": out.logits[:B].cpu().numpy(), "conf": out.conf[:B].cpu().numpy(), "pred": out.pred[:B].cpu().numpy(),
+            "exit": out.exit_mask[:B].cpu().numpy(), "idx": out.survivor_idx[:n].cpu().numpy(), "n": n}
+
+
+@pytest.mark.parametrize("dtype,HW,C,K", [("bf16", 196, 256, 1000), ("f32", 50, 40, 17)])
+def test_static_scratch_head_matches_caller_scratch_head_twice(dtype, HW, C, K):
+    spec = _head_model(dtype, HW, C, K, max_batch=48)
+    m = eb.EEModel(spec)
+    out_ref, out_new = eb.StageBuffers(m, 0), eb.StageBuffers(m, 0)
+    scratch = torch.empty(m.exit_head_scratch_bytes(0) + 256, dtype=torch.uint8, device="cuda")
+    tol = util.TOL[dtype]
+    for call, B in enumerate((48, 19)):                                  # second call: smaller batch on a dirty array
+        x = eb.to_device(dtype, wl.random_features((B, HW, C), seed=60 + call, bf16=dtype == "bf16"))
+        shift = torch.as_tensor((np.arange(B) % 4 == 0).astype(np.float32) * 9.0, device="cuda")
+        cls = torch.as_tensor((np.arange(B) * 3 % K).astype(np.int32), device="cuda")
+        ref = _run(m, out_ref, lambda *a, **k: m.exit_head(*a[:5], scratch, **k), x, B, HW, shift, cls)
+        new = _run(m, out_new, m.exit_head_static, x, B, HW, shift, cls)
+        assert util.norm_err(new["z"], ref["z"]) <= tol and util.rel_err(new["z"], ref["z"]) <= tol
+        assert np.max(np.abs(new["conf"] - ref["conf"])) <= tol
+        assert np.array_equal(new["pred"], ref["pred"]) and np.array_equal(new["exit"], ref["exit"])
+        assert new["n"] == ref["n"] and np.array_equal(new["idx"], ref["idx"])
+        assert new["n"] == B - len(range(0, B, 4))                       # every fourth sample was pushed over the threshold
+
+
+def test_static_scratch_head_refuses_what_does_not_fit():
+    # 8 MiB array: 64 samples x 98 pooling chunks x 2048 channels of fp32 partial sums alone need 51 MB
+    spec = _head_model("bf16", 784, 2048, 10, max_batch=64)
+    m = eb.EEModel(spec)
+    out = eb.StageBuffers(m, 0)
+    x = torch.zeros((1, 784, 2048), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(eb.EEError) as e:
+        m.exit_head_static(0, x, 1, 784, out)
+    assert e.value.status == 3 and "scratch bytes" in str(e.value)
