@@ -190,8 +190,10 @@ def run_ours(args):
                      mask=torch.empty(B, dtype=torch.uint8).pin_memory()) for _ in range(nst)]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # larger than the 126 MB L2
     stream = torch.cuda.current_stream()
-    launches = [0]
     sizes_last = []
+    # kernels launched by one ee_stage_run: one per layer (two for a packed stem), three for the head, one gather
+    stage_launches = [sum(2 if pl["kernel"].endswith("_packed") else 1 for pl in model.plan(s, 1)) + 3 +
+                      (0 if spec.stages[s].always_exit else 1) for s in range(nst)]
 
     def step(e2e: bool):
         """One pass of the whole path.  Returns (#kernel launches, h2d bytes, d2h bytes, per-stage batch)."""
@@ -207,7 +209,7 @@ def run_ours(args):
         for s in range(nst):
             sizes.append(n)
             model.stage_run(s, feat, n, bufs[s], ws, ids)
-            nl += len(spec.stages[s].layers) + 3 + (0 if spec.stages[s].always_exit else 1)
+            nl += stage_launches[s]
             if e2e:
                 res_host[s]["conf"][:n].copy_(bufs[s].conf[:n], non_blocking=True)
                 res_host[s]["pred"][:n].copy_(bufs[s].pred[:n], non_blocking=True)
@@ -259,6 +261,7 @@ def run_ours(args):
     # instrumented pass: per-kernel device time by CUDA events on the launching stream
     model.set_timing(True)
     fam = {}
+    per_layer = {}
     inst_ms = 0.0
     for _ in range(K):
         flush.zero_()
@@ -275,6 +278,9 @@ def run_ours(args):
                 inst_ms += ms
                 if i < len(plan):
                     f["flops"] += plan[i]["flops"]; f["bytes"] += plan[i]["bytes"]
+                    pl = per_layer.setdefault((s, i), {"kernel": name, "m": plan[i]["m"], "n": plan[i]["n"], "k": plan[i]["k"],
+                                                       "ms": 0.0, "flops": plan[i]["flops"], "bytes": plan[i]["bytes"]})
+                    pl["ms"] += ms / K
             info = model.query(s)
             ns = int(bufs[s].n_surv_host[0])
             es = 2 if spec.dtype == "bf16" else 4
@@ -340,6 +346,15 @@ def run_ours(args):
         "kernels": kernels,
         "instrumented_ms_per_step": inst_ms / K,
     }
+    if args.report_layers:
+        rows = []
+        for (s, i), pl in sorted(per_layer.items()):
+            sec = pl["ms"] * 1e-3
+            bound_ms = max(pl["flops"] / (peaks["tf_sustained"] * 1e12), pl["bytes"] / (peaks["hbm_gbs"] * 1e9)) * 1e3
+            rows.append({"stage": s, "layer": i, **{k: pl[k] for k in ("kernel", "m", "n", "k")}, "us": pl["ms"] * 1e3,
+                         "tflops": pl["flops"] / sec / 1e12 if sec else 0, "gbs": pl["bytes"] / sec / 1e9 if sec else 0,
+                         "bound_us": bound_ms * 1e3})
+        out["layers"] = rows
     print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
@@ -354,6 +369,7 @@ def main():
     ap.add_argument("--batch", type=int, default=64)
     ap.add_argument("--workload", default="resnet50", choices=["resnet50", "mobilenetv2", "tiny"])
     ap.add_argument("--cpu-samples", type=int, default=16)
+    ap.add_argument("--report-layers", action="store_true", help="add a per-layer table (time, TFLOP/s, GB/s, roofline bound) to the JSON line")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

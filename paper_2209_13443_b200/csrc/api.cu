@@ -26,8 +26,8 @@ thread_local std::string g_cuda_err;
     }                                                                                      \
   } while (0)
 
-enum KernelKind { KK_SIMT = 0, KK_TC = 1, KK_DW = 2, KK_POOL = 3 };
-const char* kKernelNames[] = {"conv_igemm_simt", "conv_igemm_tcgen05", "dwconv", "maxpool"};
+enum KernelKind { KK_SIMT = 0, KK_TC = 1, KK_DW = 2, KK_POOL = 3, KK_TC_PACKED = 4 };
+const char* kKernelNames[] = {"conv_igemm_simt", "conv_igemm_tcgen05", "dwconv", "maxpool", "conv_igemm_tcgen05_packed"};
 
 struct LayerPlan {
   ee_layer_desc_t d;
@@ -39,14 +39,15 @@ struct LayerPlan {
   void* w_dev = nullptr;
   float* scale_dev = nullptr;
   float* bias_dev = nullptr;
-  TcLayer tc;  // tensor-core plan (valid iff kind == KK_TC)
+  TcLayer tc;  // tensor-core plan (valid iff kind == KK_TC or KK_TC_PACKED)
+  int kp = 0;  // KK_TC_PACKED: columns of the packed Toeplitz matrix (K rounded up to whole K blocks)
 };
 
 struct StagePlan {
   std::vector<LayerPlan> layers;
   int in_h, in_w, in_c, out_h, out_w, out_c, out_slot;
   std::vector<size_t> slot_off;  // byte offsets at max_batch
-  size_t head_off = 0, ws_bytes = 0, head_bytes = 0;
+  size_t head_off = 0, ws_bytes = 0, head_bytes = 0, pack_off = 0;
   int n_classes = 0;
   void* fc_w = nullptr;
   float* fc_b = nullptr;
@@ -134,7 +135,7 @@ void record(ee_model* m, StagePlan& sp, cudaStream_t st, const char* name) {
 }
 
 template <typename T>
-ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const void* res, void* dst, int B,
+ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const void* res, void* dst, void* pack, int B,
                          cudaStream_t st) {
   ConvGeom g{B, L.in_h, L.in_w, L.d.cin, L.out_h, L.out_w, L.d.cout, L.d.kh, L.d.kw, L.d.stride, L.d.pad, L.d.act};
   constexpr int V = Elem<T>::kVec;
@@ -148,6 +149,20 @@ ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const
     case KK_TC: {
       ee_status_t s = tc_launch(m->tc, L.tc, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st);
       if (s != EE_OK) return s;
+      break;
+    }
+    case KK_TC_PACKED: {
+      if constexpr (sizeof(T) == 2) {
+        const long groups = (long)B * L.out_h * L.out_w * (L.kp / 8);
+        const int grid = (int)std::min<long>(cdiv(groups, 256), 148L * 64);
+        im2col_pack_kernel<<<grid, 256, 0, st>>>((const bf16*)src, (bf16*)pack, B, L.in_h, L.in_w, L.d.cin, L.out_h, L.out_w, L.d.kh,
+                                                 L.d.kw, L.d.stride, L.d.pad, L.kp);
+        EE_CUDA(cudaGetLastError());
+        ee_status_t s = tc_launch(m->tc, L.tc, pack, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st);
+        if (s != EE_OK) return s;
+      } else {
+        return EE_ERR_INTERNAL;
+      }
       break;
     }
     case KK_DW: {
@@ -414,6 +429,7 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
     sp.threshold = sd.threshold;
     sp.always_exit = sd.always_exit;
     // uploads and kernel choice
+    size_t pack_bytes = 0;
     for (int i = 0; i < sd.n_layers; ++i) {
       LayerPlan& L = sp.layers[i];
       const ee_layer_desc_t& d = L.d;
@@ -432,9 +448,28 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
         L.kind = KK_TC;
         rc = tc_plan_layer(m->tc, d, L.in_h, L.in_w, L.out_h, L.out_w, desc->max_batch, L.w_dev, &L.tc);
         if (rc != EE_OK) return fail(rc);
+      } else if (desc->dtype == EE_BF16 && d.cout % 8 == 0 && d.kh * d.kw * d.cin <= 512) {
+        // pixel rows are not 16-byte units (e.g. a 3-channel stem): explicit Toeplitz rows, then the tensor-core GEMM
+        L.kind = KK_TC_PACKED;
+        const int K = d.kh * d.kw * d.cin;
+        L.kp = cdiv(K, kTcBK) * kTcBK;
+        void* wp = nullptr;
+        if (cudaMalloc(&wp, (size_t)d.cout * L.kp * 2) != cudaSuccess) return fail(EE_ERR_CUDA);
+        m->owned.push_back(wp);
+        pad_rows_kernel<<<cdiv((long)d.cout * L.kp, 256), 256, 0, st>>>((const bf16*)L.w_dev, (bf16*)wp, d.cout, K, L.kp);
+        if (cudaGetLastError() != cudaSuccess) return fail(EE_ERR_CUDA);
+        ee_layer_desc_t g = d;
+        g.cin = L.kp, g.kh = g.kw = 1, g.stride = 1, g.pad = 0;
+        rc = tc_plan_layer(m->tc, g, L.out_h, L.out_w, L.out_h, L.out_w, desc->max_batch, wp, &L.tc);
+        if (rc != EE_OK) return fail(rc);
+        pack_bytes = std::max(pack_bytes, (size_t)desc->max_batch * L.out_h * L.out_w * L.kp * 2);
       } else {
         L.kind = KK_SIMT;
       }
+    }
+    if (pack_bytes) {  // the packed matrix lives behind the head scratch
+      sp.pack_off = align_up(sp.ws_bytes, 1024);
+      sp.ws_bytes = sp.pack_off + pack_bytes;
     }
     if ((rc = upload_bytes(m, sd.fc_weight, (size_t)sd.n_classes * sp.out_c * es, ondev, st, &sp.fc_w)) != EE_OK) return fail(rc);
     if ((rc = upload<float>(m, sd.fc_bias, sd.n_classes, ondev, st, &sp.fc_b)) != EE_OK) return fail(rc);
@@ -484,8 +519,9 @@ ee_status_t ee_stage_run(ee_model_t* m, int stage, const ee_stage_in_t* in, void
     const void* src = L.src_slot < 0 ? in->features : ws + sp.slot_off[L.src_slot];
     const void* res = L.res_slot == -2 ? nullptr : (L.res_slot == -1 ? in->features : ws + sp.slot_off[L.res_slot]);
     void* dst = ws + sp.slot_off[L.out_slot];
-    ee_status_t s = m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, src, res, dst, B, st)
-                                        : launch_layer<float>(m, L, src, res, dst, B, st);
+    void* pack = ws + sp.pack_off;
+    ee_status_t s = m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, src, res, dst, pack, B, st)
+                                        : launch_layer<float>(m, L, src, res, dst, pack, B, st);
     if (s != EE_OK) return s;
     record(m, sp, st, kKernelNames[L.kind]);
   }

@@ -26,14 +26,14 @@ namespace ee {
 
 constexpr int kTcBM = 128;       // output pixels per CTA (= TMEM lanes)
 constexpr int kTcBK = 64;        // bf16 elements per K block: 128 bytes = one swizzle span
-constexpr int kTcStages = 4;
+constexpr int kTcStages = 3;      // 96 KB of tiles at BN = 128: two CTAs per SM, one's epilogue overlaps the other's main loop
 constexpr int kTcThreads = 192;  // producer warp, MMA warp, four epilogue warps
 constexpr long long kTcWaitCycles = 4000000000LL;  // ~2 s at boost clock; far beyond any healthy wait
 
 struct TcParams {
   int M, N;             // valid rows (B*Ho*Wo) and Cout
   int taps, kw;         // kh*kw and kw
-  int cblocks;          // Cin / 64
+  int cblocks;          // ceil(Cin / 64); the TMA unit zero-fills channels past Cin in both operands
   int Ho, Wo, stride, pad;
   int im2col;           // 0: A is a plain [rows][Cin] matrix, 1: im2col tensor map
   int act;
@@ -151,7 +151,7 @@ struct TcSmem {
 };
 
 template <int BN>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, 2)
 conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   using S = TcSmem<BN>;
@@ -236,8 +236,9 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
   } else {
     const int et = threadIdx.x - 64;  // 0..127
     for (int i = et; i < BN; i += 128) {
-      s_scale[i] = p.scale ? p.scale[n0 + i] : 1.f;
-      s_bias[i] = p.bias ? p.bias[n0 + i] : 0.f;
+      const bool in = n0 + i < p.N;
+      s_scale[i] = (p.scale && in) ? p.scale[n0 + i] : 1.f;
+      s_bias[i] = (p.bias && in) ? p.bias[n0 + i] : 0.f;
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");
     // warp-uniform outcome: tcgen05.ld is a warp-wide instruction
@@ -257,18 +258,22 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
           if (p.residual) {
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
-              Vec16<bf16> r;
-              r.load(p.residual + row + c0 + g * 8);
+              if (n0 + c0 + g * 8 < p.N) {  // N is a multiple of 8: a group of eight channels is all in or all out
+                Vec16<bf16> r;
+                r.load(p.residual + row + c0 + g * 8);
 #pragma unroll
-              for (int e = 0; e < 8; ++e) v[g * 8 + e] += r.v[e];
+                for (int e = 0; e < 8; ++e) v[g * 8 + e] += r.v[e];
+              }
             }
           }
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
-            Vec16<bf16> o;
+            if (n0 + c0 + g * 8 < p.N) {
+              Vec16<bf16> o;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) o.v[e] = apply_act(v[g * 8 + e], p.act);
-            o.store(p.out + row + c0 + g * 8);
+              for (int e = 0; e < 8; ++e) o.v[e] = apply_act(v[g * 8 + e], p.act);
+              o.store(p.out + row + c0 + g * 8);
+            }
           }
         }
       }
@@ -279,6 +284,50 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
+  }
+}
+
+// Explicit Toeplitz rows for layers whose pixel rows are not 16-byte units (a 3-channel stem): row m of `out`
+// holds the kh*kw*Cin taps of output pixel m in (r, s, ci) order, zero for padding taps, zero-padded to Kp
+// columns.  One thread writes one 16-byte group of eight columns.  The packed matrix then feeds the
+// tensor-core kernel as a 1x1 layer with Kp input channels.
+__global__ void __launch_bounds__(256)
+im2col_pack_kernel(const bf16* __restrict__ x, bf16* __restrict__ out, int B, int H, int W, int Cin, int Ho, int Wo, int kh, int kw,
+                   int stride, int pad, int Kp) {
+  const int groups = Kp / 8, K = kh * kw * Cin;
+  const long total = (long)B * Ho * Wo * groups;
+  for (long idx = (long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long)gridDim.x * blockDim.x) {
+    const int g = (int)(idx % groups);
+    long m = idx / groups;
+    const int wo = (int)(m % Wo);
+    const long q = m / Wo;
+    const int ho = (int)(q % Ho);
+    const long b = q / Ho;
+    const bf16* xb = x + b * H * W * Cin;
+    Vec16<bf16> o;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int k = g * 8 + e;
+      float v = 0.f;
+      if (k < K) {
+        const int tap = k / Cin, ci = k - tap * Cin;
+        const int r = tap / kw, sx = tap - r * kw;
+        const int hi = ho * stride - pad + r, wi = wo * stride - pad + sx;
+        if (hi >= 0 && hi < H && wi >= 0 && wi < W) v = __bfloat162float(xb[((long)hi * W + wi) * Cin + ci]);
+      }
+      o.v[e] = v;
+    }
+    o.store(out + (size_t)m * Kp + g * 8);
+  }
+}
+
+// Weight rows [Cout][K] copied into rows of Kp columns, zero tail.
+__global__ void pad_rows_kernel(const bf16* __restrict__ w, bf16* __restrict__ out, int rows, int K, int Kp) {
+  const long total = (long)rows * Kp;
+  for (long idx = (long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long)gridDim.x * blockDim.x) {
+    const int k = (int)(idx % Kp);
+    const long r = idx / Kp;
+    out[idx] = k < K ? w[r * K + k] : __float2bfloat16_rn(0.f);
   }
 }
 
@@ -325,11 +374,13 @@ inline ee_status_t tc_context_init(TcContext& c) {
   return EE_OK;
 }
 
-// Layers this path covers: dense convolutions whose channel counts fill whole 64-wide K blocks and N tiles.
+// Layers this path covers: dense convolutions whose pixel rows are whole 16-byte units (Cin and Cout multiples
+// of 8).  Channel counts need not fill the 64-wide K block or the N tile: the TMA unit zero-fills what lies past
+// the tensor, and the epilogue masks columns past Cout.
 inline bool tc_supported(const ee_layer_desc_t& d, int in_h, int in_w) {
   (void)in_h;
   (void)in_w;
-  return d.op == EE_OP_CONV && d.cin % kTcBK == 0 && d.cout % 64 == 0 && d.kh == d.kw && d.kh <= 7 && d.stride <= 8 &&
+  return d.op == EE_OP_CONV && d.cin % 8 == 0 && d.cout % 8 == 0 && d.kh == d.kw && d.kh <= 7 && d.stride <= 8 &&
          d.pad < d.kh && d.pad <= 127;
 }
 
@@ -337,7 +388,7 @@ inline ee_status_t tc_plan_layer(TcContext& c, const ee_layer_desc_t& d, int in_
                                  const void* w_dev, TcLayer* L) {
   L->cin = d.cin, L->cout = d.cout, L->kh = d.kh, L->kw = d.kw, L->stride = d.stride, L->pad = d.pad, L->act = d.act;
   L->in_h = in_h, L->in_w = in_w, L->out_h = out_h, L->out_w = out_w, L->max_batch = max_batch;
-  L->bn = d.cout % 128 == 0 ? 128 : 64;
+  L->bn = d.cout > 64 ? 128 : 64;
   L->im2col = !(d.kh == 1 && d.stride == 1 && d.pad == 0);
   // weights [Cout][taps][Cin] as a 3-D tensor, box = 64 channels x 1 tap x BN filters
   const cuuint64_t dims[3] = {(cuuint64_t)d.cin, (cuuint64_t)(d.kh * d.kw), (cuuint64_t)d.cout};
@@ -404,7 +455,7 @@ inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, co
   p.N = L.cout;
   p.taps = L.kh * L.kw;
   p.kw = L.kw;
-  p.cblocks = L.cin / kTcBK;
+  p.cblocks = cdiv(L.cin, kTcBK);
   p.Ho = L.out_h, p.Wo = L.out_w, p.stride = L.stride, p.pad = L.pad;
   p.im2col = L.im2col ? 1 : 0;
   p.act = L.act;
@@ -412,7 +463,7 @@ inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, co
   p.residual = (const bf16*)res;
   p.out = (bf16*)dst;
   p.err_flag = err_flag;
-  dim3 grid(cdiv(p.M, kTcBM), L.cout / L.bn);
+  dim3 grid(cdiv(p.M, kTcBM), cdiv(L.cout, L.bn));
   if (L.bn == 128)
     conv_igemm_tcgen05_kernel<128><<<grid, kTcThreads, TcSmem<128>::kBytes, st>>>(*tmA, L.tm_w, p);
   else
