@@ -191,9 +191,10 @@ def run_ours(args):
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # larger than the 126 MB L2
     stream = torch.cuda.current_stream()
     sizes_last = []
-    # kernels launched by one ee_stage_run: one per layer (two for a packed stem), three for the head, one gather
-    stage_launches = [sum(2 if pl["kernel"].endswith("_packed") else 1 for pl in model.plan(s, 1)) + 3 +
-                      (0 if spec.stages[s].always_exit else 1) for s in range(nst)]
+    def stage_launches(s, n):
+        """Kernels one ee_stage_run launches: the layers' (a packed stem packs and multiplies chunk by chunk),
+        three for the head, one gather."""
+        return sum(pl["launches"] for pl in model.plan(s, n)) + 3 + (0 if spec.stages[s].always_exit else 1)
 
     def step(e2e: bool):
         """One pass of the whole path.  Returns (#kernel launches, h2d bytes, d2h bytes, per-stage batch)."""
@@ -209,7 +210,7 @@ def run_ours(args):
         for s in range(nst):
             sizes.append(n)
             model.stage_run(s, feat, n, bufs[s], ws, ids)
-            nl += stage_launches[s]
+            nl += stage_launches(s, n)
             if e2e:
                 res_host[s]["conf"][:n].copy_(bufs[s].conf[:n], non_blocking=True)
                 res_host[s]["pred"][:n].copy_(bufs[s].pred[:n], non_blocking=True)

@@ -216,6 +216,7 @@ typedef struct {
   const char* kernel;
   int m, n, k;
   double flops, bytes;
+  int launches; /* kernels this layer launches at this batch size */
 } ee_layer_plan_t;
 ee_status_t ee_model_plan(const ee_model_t* model, int stage, int batch, int cap, ee_layer_plan_t* out, int* n);
 

@@ -66,7 +66,7 @@ class StageOut(C.Structure):
 
 class LayerPlan(C.Structure):
     _fields_ = [("kernel", C.c_char_p), ("m", C.c_int), ("n", C.c_int), ("k", C.c_int), ("flops", C.c_double),
-                ("bytes", C.c_double)]
+                ("bytes", C.c_double), ("launches", C.c_int)]
 
 
 _lib = None
@@ -261,7 +261,8 @@ class EEModel:
         arr = (LayerPlan * cap)()
         n = C.c_int(0)
         _check(self._L.ee_model_plan(self._h, stage, int(batch), cap, arr, C.byref(n)), "ee_model_plan")
-        return [dict(kernel=arr[i].kernel.decode(), m=arr[i].m, n=arr[i].n, k=arr[i].k, flops=arr[i].flops, bytes=arr[i].bytes)
+        return [dict(kernel=arr[i].kernel.decode(), m=arr[i].m, n=arr[i].n, k=arr[i].k, flops=arr[i].flops, bytes=arr[i].bytes,
+                     launches=arr[i].launches)
                 for i in range(n.value)]
 
     def check(self, stream=None):

@@ -40,7 +40,8 @@ struct LayerPlan {
   float* scale_dev = nullptr;
   float* bias_dev = nullptr;
   TcLayer tc;  // tensor-core plan (valid iff kind == KK_TC or KK_TC_PACKED)
-  int kp = 0;  // KK_TC_PACKED: columns of the packed Toeplitz matrix (K rounded up to whole K blocks)
+  int kp = 0, runp = 0;  // KK_TC_PACKED: columns of the packed Toeplitz matrix and of one filter-row run
+  int pack_chunk = 0;    // KK_TC_PACKED: samples packed per launch, so that the packed chunk stays in L2
 };
 
 struct StagePlan {
@@ -153,13 +154,24 @@ ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const
     }
     case KK_TC_PACKED: {
       if constexpr (sizeof(T) == 2) {
-        const long groups = (long)B * L.out_h * L.out_w * (L.kp / 8);
-        const int grid = (int)std::min<long>(cdiv(groups, 256), 148L * 64);
-        im2col_pack_kernel<<<grid, 256, 0, st>>>((const bf16*)src, (bf16*)pack, B, L.in_h, L.in_w, L.d.cin, L.out_h, L.out_w, L.d.kh,
-                                                 L.d.kw, L.d.stride, L.d.pad, L.kp);
-        EE_CUDA(cudaGetLastError());
-        ee_status_t s = tc_launch(m->tc, L.tc, pack, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st);
-        if (s != EE_OK) return s;
+        // chunk by chunk: pack a few samples' Toeplitz rows (they stay in L2), multiply, next chunk
+        const size_t in_ps = (size_t)L.in_h * L.in_w * L.d.cin, out_ps = (size_t)L.out_h * L.out_w * L.d.cout;
+        for (int b0 = 0; b0 < B; b0 += L.pack_chunk) {
+          const int nb = std::min(L.pack_chunk, B - b0);
+          const long runs = (long)nb * L.out_h * L.out_w * L.d.kh;
+          const int grid = (int)std::min<long>(cdiv(runs, 256), 148L * 64);
+          const bf16* xs = (const bf16*)src + in_ps * b0;
+          if (L.d.cin == 3)
+            im2col_pack_kernel<3><<<grid, 256, 0, st>>>(xs, (bf16*)pack, nb, L.in_h, L.in_w, 3, L.out_h, L.out_w, L.d.kh, L.d.kw,
+                                                         L.d.stride, L.d.pad, L.runp, L.kp);
+          else
+            im2col_pack_kernel<0><<<grid, 256, 0, st>>>(xs, (bf16*)pack, nb, L.in_h, L.in_w, L.d.cin, L.out_h, L.out_w, L.d.kh,
+                                                         L.d.kw, L.d.stride, L.d.pad, L.runp, L.kp);
+          EE_CUDA(cudaGetLastError());
+          const bf16* rs = res ? (const bf16*)res + out_ps * b0 : nullptr;
+          ee_status_t s = tc_launch(m->tc, L.tc, pack, rs, (bf16*)dst + out_ps * b0, nb, L.scale_dev, L.bias_dev, m->err_flag, st);
+          if (s != EE_OK) return s;
+        }
       } else {
         return EE_ERR_INTERNAL;
       }
@@ -210,9 +222,9 @@ ee_status_t launch_head(ee_model* m, StagePlan& sp, const void* x, int B, int hw
   EE_CUDA(cudaGetLastError());
   if (timed) record(m, sp, st, "head_gap");
   if (C % V == 0)
-    fc_kernel<T, V><<<cdiv(K, kFcWarps), kFcWarps * 32, 0, st>>>(gap, (const T*)sp.fc_w, sp.fc_b, B, C, K, z);
+    fc_kernel<T, V><<<cdiv(K, kFcClasses), kFcWarps * 32, 0, st>>>(gap, (const T*)sp.fc_w, sp.fc_b, B, C, K, z);
   else
-    fc_kernel<T, 1><<<cdiv(K, kFcWarps), kFcWarps * 32, 0, st>>>(gap, (const T*)sp.fc_w, sp.fc_b, B, C, K, z);
+    fc_kernel<T, 1><<<cdiv(K, kFcClasses), kFcWarps * 32, 0, st>>>(gap, (const T*)sp.fc_w, sp.fc_b, B, C, K, z);
   EE_CUDA(cudaGetLastError());
   if (timed) record(m, sp, st, "head_fc");
   exit_decide_kernel<<<1, kDecideThreads, 0, st>>>(z, B, K, shift, shift_cls, sp.threshold, sp.always_exit, out->conf,
@@ -448,21 +460,24 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
         L.kind = KK_TC;
         rc = tc_plan_layer(m->tc, d, L.in_h, L.in_w, L.out_h, L.out_w, desc->max_batch, L.w_dev, &L.tc);
         if (rc != EE_OK) return fail(rc);
-      } else if (desc->dtype == EE_BF16 && d.cout % 8 == 0 && d.kh * d.kw * d.cin <= 512) {
+      } else if (desc->dtype == EE_BF16 && d.cout % 8 == 0 && d.kh * d.kw * d.cin <= 512 && d.kw * d.cin <= 64) {
         // pixel rows are not 16-byte units (e.g. a 3-channel stem): explicit Toeplitz rows, then the tensor-core GEMM
         L.kind = KK_TC_PACKED;
-        const int K = d.kh * d.kw * d.cin;
-        L.kp = cdiv(K, kTcBK) * kTcBK;
+        const int run = d.kw * d.cin;
+        L.runp = cdiv(run, 8) * 8;
+        L.kp = cdiv(d.kh * L.runp, kTcBK) * kTcBK;
+        const size_t per_sample = (size_t)L.out_h * L.out_w * L.kp * 2;
+        L.pack_chunk = (int)std::max<size_t>(1, std::min<size_t>((size_t)desc->max_batch, ((size_t)32 << 20) / per_sample));
         void* wp = nullptr;
         if (cudaMalloc(&wp, (size_t)d.cout * L.kp * 2) != cudaSuccess) return fail(EE_ERR_CUDA);
         m->owned.push_back(wp);
-        pad_rows_kernel<<<cdiv((long)d.cout * L.kp, 256), 256, 0, st>>>((const bf16*)L.w_dev, (bf16*)wp, d.cout, K, L.kp);
+        pack_weights_kernel<<<cdiv((long)d.cout * L.kp, 256), 256, 0, st>>>((const bf16*)L.w_dev, (bf16*)wp, d.cout, d.kh, run, L.runp, L.kp);
         if (cudaGetLastError() != cudaSuccess) return fail(EE_ERR_CUDA);
         ee_layer_desc_t g = d;
         g.cin = L.kp, g.kh = g.kw = 1, g.stride = 1, g.pad = 0;
-        rc = tc_plan_layer(m->tc, g, L.out_h, L.out_w, L.out_h, L.out_w, desc->max_batch, wp, &L.tc);
+        rc = tc_plan_layer(m->tc, g, L.out_h, L.out_w, L.out_h, L.out_w, L.pack_chunk, wp, &L.tc);
         if (rc != EE_OK) return fail(rc);
-        pack_bytes = std::max(pack_bytes, (size_t)desc->max_batch * L.out_h * L.out_w * L.kp * 2);
+        pack_bytes = std::max(pack_bytes, per_sample * L.pack_chunk);
       } else {
         L.kind = KK_SIMT;
       }
@@ -687,6 +702,7 @@ ee_status_t ee_model_plan(const ee_model_t* m, int stage, int batch, int cap, ee
     const double in_b = (double)batch * L.in_h * L.in_w * L.d.cin * es, out_b = (double)p.m * p.n * es;
     const double w_b = L.d.op == EE_OP_MAXPOOL ? 0.0 : (double)L.d.cout * p.k * es;
     p.bytes = in_b + out_b + w_b + (L.res_slot != -2 ? out_b : 0.0);
+    p.launches = L.kind == KK_TC_PACKED ? 2 * cdiv(batch, L.pack_chunk) : 1;
   }
   return EE_OK;
 }

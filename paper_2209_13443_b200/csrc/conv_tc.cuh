@@ -287,47 +287,55 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
   }
 }
 
-// Explicit Toeplitz rows for layers whose pixel rows are not 16-byte units (a 3-channel stem): row m of `out`
-// holds the kh*kw*Cin taps of output pixel m in (r, s, ci) order, zero for padding taps, zero-padded to Kp
-// columns.  One thread writes one 16-byte group of eight columns.  The packed matrix then feeds the
-// tensor-core kernel as a 1x1 layer with Kp input channels.
+// Explicit Toeplitz rows for layers whose pixel rows are not 16-byte units (a 3-channel stem).  Row m of `out`
+// holds, for every filter row r, the kw*Cin taps of output pixel m (contiguous in the NHWC input), zero for
+// padding taps, each run zero-padded to `runp` columns; the row is zero-padded to Kp columns.  One thread writes
+// one run.  The packed matrix then feeds the tensor-core kernel as a 1x1 layer with Kp input channels; the
+// weights are laid out to match by pack_weights_kernel.
+template <int CIN>
 __global__ void __launch_bounds__(256)
-im2col_pack_kernel(const bf16* __restrict__ x, bf16* __restrict__ out, int B, int H, int W, int Cin, int Ho, int Wo, int kh, int kw,
-                   int stride, int pad, int Kp) {
-  const int groups = Kp / 8, K = kh * kw * Cin;
-  const long total = (long)B * Ho * Wo * groups;
+im2col_pack_kernel(const bf16* __restrict__ x, bf16* __restrict__ out, int B, int H, int W, int cin_rt, int Ho, int Wo, int kh, int kw,
+                   int stride, int pad, int runp, int Kp) {
+  const int Cin = CIN > 0 ? CIN : cin_rt;
+  const long total = (long)B * Ho * Wo * kh;
+  const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
   for (long idx = (long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long)gridDim.x * blockDim.x) {
-    const int g = (int)(idx % groups);
-    long m = idx / groups;
+    const int r = (int)(idx % kh);
+    const long m = idx / kh;
     const int wo = (int)(m % Wo);
     const long q = m / Wo;
     const int ho = (int)(q % Ho);
     const long b = q / Ho;
-    const bf16* xb = x + b * H * W * Cin;
-    Vec16<bf16> o;
+    const int hi = ho * stride - pad + r;
+    const bool row_in = hi >= 0 && hi < H;
+    const int wi0 = wo * stride - pad;
+    const bf16* xr = x + ((b * H + (row_in ? hi : 0)) * W) * (long)Cin;
+    bf16* orow = out + (size_t)m * Kp + (size_t)r * runp;
+    int j = 0;
+    for (int g = 0; g < runp; g += 8) {
+      __align__(16) bf16 v[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const int k = g * 8 + e;
-      float v = 0.f;
-      if (k < K) {
-        const int tap = k / Cin, ci = k - tap * Cin;
-        const int r = tap / kw, sx = tap - r * kw;
-        const int hi = ho * stride - pad + r, wi = wo * stride - pad + sx;
-        if (hi >= 0 && hi < H && wi >= 0 && wi < W) v = __bfloat162float(xb[((long)hi * W + wi) * Cin + ci]);
+      for (int e = 0; e < 8; ++e, ++j) {
+        const int sx = j / Cin, ci = j - sx * Cin;   // CIN is a compile-time constant on the hot instantiation
+        const int wi = wi0 + sx;
+        v[e] = (row_in && sx < kw && wi >= 0 && wi < W) ? xr[(long)wi * Cin + ci] : zero;
       }
-      o.v[e] = v;
+      *reinterpret_cast<uint4*>(orow + g) = *reinterpret_cast<const uint4*>(v);
     }
-    o.store(out + (size_t)m * Kp + g * 8);
+    if (r == 0) {  // zero tail of the row: the matching weight columns are zero, but 0 * NaN is NaN
+      for (int k = kh * runp; k < Kp; k += 8) *reinterpret_cast<uint4*>(out + (size_t)m * Kp + k) = make_uint4(0, 0, 0, 0);
+    }
   }
 }
 
-// Weight rows [Cout][K] copied into rows of Kp columns, zero tail.
-__global__ void pad_rows_kernel(const bf16* __restrict__ w, bf16* __restrict__ out, int rows, int K, int Kp) {
+// Weight rows [Cout][kh][kw*Cin] copied into rows [Cout][kh][runp] padded to Kp columns, zeros elsewhere.
+__global__ void pack_weights_kernel(const bf16* __restrict__ w, bf16* __restrict__ out, int rows, int kh, int run, int runp, int Kp) {
   const long total = (long)rows * Kp;
   for (long idx = (long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long)gridDim.x * blockDim.x) {
     const int k = (int)(idx % Kp);
-    const long r = idx / Kp;
-    out[idx] = k < K ? w[r * K + k] : __float2bfloat16_rn(0.f);
+    const long co = idx / Kp;
+    const int r = k / runp, j = k - r * runp;
+    out[idx] = (r < kh && j < run) ? w[(co * kh + r) * run + j] : __float2bfloat16_rn(0.f);
   }
 }
 

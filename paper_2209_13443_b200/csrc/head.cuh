@@ -42,8 +42,22 @@ gap_kernel(const T* __restrict__ x, int HW, int C, int rows_per_chunk, float* __
 #pragma unroll
     for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
     if (active && v < cv) {
-      for (int r = r0 + grp; r < r1; r += groups) {
-        const T* p = xb + (size_t)r * C + (size_t)v * VEC;
+      const T* p0 = xb + (size_t)v * VEC;
+      int r = r0 + grp;
+      if constexpr (VEC > 1) {
+        // four independent 16-byte loads in flight; the additions keep the ascending row order
+        for (; r + 3 * groups < r1; r += 4 * groups) {
+          Vec16<T> t0, t1, t2, t3;
+          t0.load(p0 + (size_t)r * C);
+          t1.load(p0 + (size_t)(r + groups) * C);
+          t2.load(p0 + (size_t)(r + 2 * groups) * C);
+          t3.load(p0 + (size_t)(r + 3 * groups) * C);
+#pragma unroll
+          for (int e = 0; e < VEC; ++e) acc[e] = (((acc[e] + t0.v[e]) + t1.v[e]) + t2.v[e]) + t3.v[e];
+        }
+      }
+      for (; r < r1; r += groups) {
+        const T* p = p0 + (size_t)r * C;
         if constexpr (VEC > 1) {
           Vec16<T> t;
           t.load(p);
@@ -83,47 +97,78 @@ gap_kernel(const T* __restrict__ x, int HW, int C, int rows_per_chunk, float* __
   if (tid == 0) counters[b] = 0;
 }
 
-constexpr int kFcWarps = 8, kFcSamples = 8;
+constexpr int kFcWarps = 8, kFcClassesPerWarp = 2, kFcSamples = 16, kFcChunk = 256;
+constexpr int kFcClasses = kFcWarps * kFcClassesPerWarp;
 
-// z[b][k] = bfc[k] + sum_c wfc[k][c] * gap[b][c].  One warp per class, samples in tiles of eight so
-// that a weight vector is loaded once per eight samples.
+// z[b][k] = bfc[k] + sum_c wfc[k][c] * gap[b][c].  A CTA owns 16 classes (two per warp) and walks the samples in
+// tiles of 16; the tile's pooled vectors are staged in shared memory 256 channels at a time, so the pooled matrix
+// crosses L2 once per CTA.  Per (b, k): every lane adds its channels in ascending order, then a shuffle tree;
+// the order does not depend on the batch size.
 template <typename T, int VEC>
 __global__ void __launch_bounds__(kFcWarps * 32)
 fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float* __restrict__ bfc, int B, int C, int K,
           float* __restrict__ z) {
-  const int lane = threadIdx.x & 31, k = blockIdx.x * kFcWarps + (threadIdx.x >> 5);
-  if (k >= K) return;
-  const T* wr = wfc + (size_t)k * C;
-  const float bk = bfc ? bfc[k] : 0.f;
+  __shared__ __align__(16) float gs[kFcSamples][kFcChunk];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int k0 = blockIdx.x * kFcClasses + warp * kFcClassesPerWarp;
+  constexpr int PER = kFcChunk / 32;  // channels per lane per chunk (8)
   for (int b0 = 0; b0 < B; b0 += kFcSamples) {
-    float acc[kFcSamples];
+    float acc[kFcClassesPerWarp][kFcSamples];
 #pragma unroll
-    for (int s = 0; s < kFcSamples; ++s) acc[s] = 0.f;
-    for (int c = lane * VEC; c < C; c += 32 * VEC) {
-      float wv[VEC];
-      if constexpr (VEC > 1) {
-        Vec16<T> t;
-        t.load(wr + c);
+    for (int q = 0; q < kFcClassesPerWarp; ++q)
 #pragma unroll
-        for (int e = 0; e < VEC; ++e) wv[e] = t.v[e];
-      } else {
-        wv[0] = Elem<T>::ld(wr + c);
+      for (int s = 0; s < kFcSamples; ++s) acc[q][s] = 0.f;
+    for (int c0 = 0; c0 < C; c0 += kFcChunk) {
+      __syncthreads();
+      for (int i = threadIdx.x; i < kFcSamples * kFcChunk; i += kFcWarps * 32) {
+        const int s = i / kFcChunk, c = i - s * kFcChunk;
+        gs[s][c] = (b0 + s < B && c0 + c < C) ? gap[(size_t)(b0 + s) * C + c0 + c] : 0.f;
+      }
+      __syncthreads();
+      const int c = c0 + lane * PER;
+      float wv[kFcClassesPerWarp][PER];
+#pragma unroll
+      for (int q = 0; q < kFcClassesPerWarp; ++q) {
+        const int k = k0 + q;
+#pragma unroll
+        for (int e = 0; e < PER; ++e) wv[q][e] = 0.f;
+        if (k < K) {
+          if constexpr (VEC == 8) {
+            if (c + PER <= C) {
+              Vec16<T> t;
+              t.load(wfc + (size_t)k * C + c);
+#pragma unroll
+              for (int e = 0; e < PER; ++e) wv[q][e] = t.v[e];
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < PER; ++e)
+              if (c + e < C) wv[q][e] = Elem<T>::ld(wfc + (size_t)k * C + c + e);
+          }
+        }
       }
 #pragma unroll
       for (int s = 0; s < kFcSamples; ++s) {
-        if (b0 + s < B) {
-          const float* gp = gap + (size_t)(b0 + s) * C + c;
+        const float4 g0 = *reinterpret_cast<const float4*>(&gs[s][lane * PER]);
+        const float4 g1 = *reinterpret_cast<const float4*>(&gs[s][lane * PER + 4]);
+        const float gv[PER] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
 #pragma unroll
-          for (int e = 0; e < VEC; ++e) acc[s] = fmaf(wv[e], gp[e], acc[s]);
-        }
+        for (int q = 0; q < kFcClassesPerWarp; ++q)
+#pragma unroll
+          for (int e = 0; e < PER; ++e) acc[q][s] = fmaf(wv[q][e], gv[e], acc[q][s]);
       }
     }
 #pragma unroll
-    for (int s = 0; s < kFcSamples; ++s) {
-      float v = acc[s];
+    for (int q = 0; q < kFcClassesPerWarp; ++q) {
+      const int k = k0 + q;
+      const float bk = (bfc && k < K) ? bfc[k] : 0.f;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      if (lane == 0 && b0 + s < B) z[(size_t)(b0 + s) * K + k] = v + bk;
+      for (int s = 0; s < kFcSamples; ++s) {
+        float v = acc[q][s];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0 && k < K && b0 + s < B) z[(size_t)(b0 + s) * K + k] = v + bk;
+      }
     }
   }
 }
@@ -141,15 +186,35 @@ exit_decide_kernel(float* __restrict__ z, int B, int K, const float* __restrict_
   __shared__ int warp_tot[32];
   __shared__ int pass_total;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int kRegs = 32;  // logits per lane held in registers: one pass over memory for K <= 1024
   for (int b = warp; b < B; b += kDecideThreads / 32) {
     float* zb = z + (size_t)b * K;
     const int cls = (shift && shift_cls) ? shift_cls[b] : -1;
+    const float sh = cls >= 0 && cls < K ? shift[b] : 0.f;
     float m = -INFINITY;
     int arg = 0x7fffffff;
-    for (int k = lane; k < K; k += 32) {
+    float zr[kRegs];
+#pragma unroll
+    for (int i = 0; i < kRegs; ++i) {
+      const int k = lane + 32 * i;
+      zr[i] = k < K ? zb[k] : -INFINITY;
+    }
+#pragma unroll
+    for (int i = 0; i < kRegs; ++i) {
+      const int k = lane + 32 * i;
+      if (k == cls) {
+        zr[i] += sh;
+        zb[k] = zr[i];
+      }
+      if (zr[i] > m) {
+        m = zr[i];
+        arg = k;
+      }
+    }
+    for (int k = lane + 32 * kRegs; k < K; k += 32) {  // classes past the register window
       float v = zb[k];
       if (k == cls) {
-        v += shift[b];
+        v += sh;
         zb[k] = v;
       }
       if (v > m) {
@@ -168,7 +233,10 @@ exit_decide_kernel(float* __restrict__ z, int B, int K, const float* __restrict_
     }
     __syncwarp();
     float s = 0.f;
-    for (int k = lane; k < K; k += 32) s += expf(zb[k] - m);
+#pragma unroll
+    for (int i = 0; i < kRegs; ++i)
+      if (lane + 32 * i < K) s += expf(zr[i] - m);
+    for (int k = lane + 32 * kRegs; k < K; k += 32) s += expf(zb[k] - m);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     if (lane == 0) {
