@@ -9,8 +9,9 @@
 //
 // One CTA computes one 128 x BN output tile.  Warp roles: warp 0 issues TMA loads into a ring of
 // shared-memory stages, warp 1 owns the TMEM allocation and issues the MMAs (one thread), warps
-// 2-5 run the epilogue: tcgen05.ld of the fp32 accumulator, folded-BN scale/bias, residual add,
-// activation, one rounding to bf16, 16-byte stores.  The K loop visits (tap, channel block) in a
+// 2-5 run the epilogue: tcgen05.ld of the fp32 accumulator, folded-BN scale/bias, residual add (the
+// residual tile was brought into shared memory by TMA while the main loop ran), activation, one
+// rounding to bf16, then a TMA store of the tile from shared memory.  The K loop visits (tap, channel block) in a
 // fixed order that does not depend on the batch size.
 //
 // Every wait on an mbarrier is bounded by a clock: on expiry the thread records EE_ERR_TIMEOUT in
@@ -141,42 +142,62 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 
 // ----------------------------------------------------------------------------- kernel
 
-template <int BN>
+// Shared-memory plan of one CTA.  Layers with a residual operand keep a dedicated 128 x BN bf16 tile that the
+// producer fills with the residual at kernel start and the epilogue overwrites in place with the output; they run
+// a two-stage operand ring.  Layers without one run three stages and stage their output in ring slot 0 once the
+// main loop has drained it.  Either way 96 KB at BN = 128: two CTAs per SM.
+template <int BN, bool RES>
 struct TcSmem {
+  static constexpr int kStages = RES ? 2 : 3;
   static constexpr int kABytes = kTcBM * kTcBK * 2;
   static constexpr int kBBytes = BN * kTcBK * 2;
   static constexpr int kStage = kABytes + kBBytes;
-  static constexpr int kTiles = kTcStages * kStage;
-  static constexpr int kBytes = kTiles + 2 * BN * 4 + 256 + 1024;  // tiles, scale/bias, barriers, alignment slack
+  static constexpr int kTiles = kStages * kStage;
+  static constexpr int kIoBytes = kTcBM * BN * 2;
+  static constexpr int kIoOff = RES ? kTiles : 0;
+  static constexpr int kAfter = kTiles + (RES ? kIoBytes : 0);
+  static constexpr int kBytes = kAfter + 2 * BN * 4 + 256 + 1024;  // + scale/bias, barriers, alignment slack
+  static_assert(RES || kIoBytes <= kStage, "output staging must fit in ring slot 0");
 };
 
-template <int BN>
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tm), "r"(src), "r"(c0), "r"(c1)
+               : "memory");
+}
+
+// tmA: activations (2-D tile map or im2col map), tmW: weights [Cin][taps][Cout], tmR / tmO: residual and output as
+// [rows][Cout] matrices with a 64-column x 32-row box (128-byte swizzle).
+template <int BN, bool RES>
 __global__ void __launch_bounds__(kTcThreads, 2)
-conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, TcParams p) {
+conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+                          const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmO, TcParams p) {
   extern __shared__ uint8_t smem_raw[];
-  using S = TcSmem<BN>;
+  using S = TcSmem<BN, RES>;
+  constexpr int kStages = S::kStages;
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
   uint8_t* gen = smem_raw + (base - raw);
-  float* s_scale = reinterpret_cast<float*>(gen + S::kTiles);
+  float* s_scale = reinterpret_cast<float*>(gen + S::kAfter);
   float* s_bias = s_scale + BN;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kTiles + 2 * BN * 4);
-  const uint32_t bar0 = base + S::kTiles + 2 * BN * 4;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kAfter + 2 * BN * 4);
+  const uint32_t bar0 = base + S::kAfter + 2 * BN * 4;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (kTcStages + s); };
-  const uint32_t accum_bar = bar0 + 8u * (2 * kTcStages);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcStages + 1);
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+  const uint32_t accum_bar = bar0 + 8u * (2 * kStages);
+  const uint32_t res_bar = bar0 + 8u * (2 * kStages + 1);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * kTcBM, n0 = blockIdx.y * BN;
   const int num_kb = p.taps * p.cblocks;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kTcStages; ++s) {
+    for (int s = 0; s < kStages; ++s) {
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
     mbar_init(accum_bar, 1);
+    mbar_init(res_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {  // TMEM: BN fp32 columns x 128 lanes
@@ -187,9 +208,22 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Programmatic dependent launch: everything above overlapped the tail of the previous kernel in the stream.
+  // From here on this kernel touches activations, so it waits for that kernel's memory; the next kernel in
+  // the stream may begin its own prologue now.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == 0) {
     if (lane == 0) {
+      if (RES) {
+        mbar_expect_tx(res_bar, S::kIoBytes);
+#pragma unroll
+        for (int h = 0; h < BN / 64; ++h)
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            tma_load_2d(base + S::kIoOff + h * 16384 + q * 4096, &tmR, res_bar, n0 + h * 64, m0 + q * 32);
+      }
       int cw = 0, ch = 0, cn = 0;
       if (p.im2col) {
         const int hw = p.Ho * p.Wo;
@@ -200,8 +234,8 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
         ch = ho * p.stride - p.pad;
       }
       for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % kTcStages;
-        const uint32_t ph = (uint32_t)(kb / kTcStages) & 1u;
+        const int s = kb % kStages;
+        const uint32_t ph = (uint32_t)(kb / kStages) & 1u;
         if (!mbar_wait(empty_bar(s), ph ^ 1u, p.err_flag)) break;
         const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
         const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
@@ -220,8 +254,8 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
       constexpr uint32_t idesc = umma_idesc(BN);
       bool ok = true;
       for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % kTcStages;
-        const uint32_t ph = (uint32_t)(kb / kTcStages) & 1u;
+        const int s = kb % kStages;
+        const uint32_t ph = (uint32_t)(kb / kStages) & 1u;
         ok = mbar_wait(full_bar(s), ph, p.err_flag);
         if (!ok) break;
         tc_fence_after();
@@ -231,7 +265,7 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
           umma_bf16(tmem_base, umma_desc(sa + k * 32), umma_desc(sb + k * 32), idesc, (uint32_t)((kb | k) != 0));
         umma_commit(empty_bar(s));  // frees the stage once these MMAs have read it
       }
-      if (ok) umma_commit(accum_bar);  // accumulator complete
+      if (ok) umma_commit(accum_bar);  // accumulator complete: every MMA has also finished reading the ring
     }
   } else {
     const int et = threadIdx.x - 64;  // 0..127
@@ -241,42 +275,51 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
       s_bias[i] = (p.bias && in) ? p.bias[n0 + i] : 0.f;
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");
-    // warp-uniform outcome: tcgen05.ld is a warp-wide instruction
-    const bool ok = __all_sync(0xffffffffu, mbar_wait(accum_bar, 0, p.err_flag));
+    // warp-uniform outcomes: tcgen05.ld is a warp-wide instruction
+    bool ok = __all_sync(0xffffffffu, mbar_wait(accum_bar, 0, p.err_flag));
+    if (RES) ok = __all_sync(0xffffffffu, mbar_wait(res_bar, 0, p.err_flag)) && ok;
     tc_fence_after();
     if (ok) {
-      const int q = warp & 3;  // TMEM lane quarter this warp may read
-      const int m = m0 + q * 32 + lane;
-      const size_t row = (size_t)m * p.N + n0;
+      const int q = warp & 3;  // TMEM lane quarter this warp may read = rows [32q, 32q + 32) of the tile
+      uint8_t* io = gen + S::kIoOff;
+      const uint32_t io_s = base + S::kIoOff;
+      bool stored = false;
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        float v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
-        if (m < p.M) {
+      for (int h = 0; h < BN / 64; ++h) {
+        if (n0 + h * 64 >= p.N) break;
+        // this thread's 128-byte line of the 64-column half; its eight 16-byte chunks are XOR-swizzled with the
+        // row index so that the TMA unit (128-byte swizzle) finds row-major data
+        uint8_t* line = io + h * 16384 + (q * 32 + lane) * 128;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = fmaf(s_scale[c0 + j], v[j], s_bias[c0 + j]);
-          if (p.residual) {
+        for (int sub = 0; sub < 2; ++sub) {
+          float v[32];
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 64 + sub * 32), v);
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              if (n0 + c0 + g * 8 < p.N) {  // N is a multiple of 8: a group of eight channels is all in or all out
-                Vec16<bf16> r;
-                r.load(p.residual + row + c0 + g * 8);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) v[g * 8 + e] += r.v[e];
-              }
-            }
-          }
+          for (int j = 0; j < 32; ++j) v[j] = fmaf(s_scale[h * 64 + sub * 32 + j], v[j], s_bias[h * 64 + sub * 32 + j]);
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
-            if (n0 + c0 + g * 8 < p.N) {
-              Vec16<bf16> o;
+            bf16* chunk = reinterpret_cast<bf16*>(line + (((sub * 4 + g) ^ (lane & 7)) << 4));
+            if (RES) {
+              Vec16<bf16> r;
+              r.load(chunk);
 #pragma unroll
-              for (int e = 0; e < 8; ++e) o.v[e] = apply_act(v[g * 8 + e], p.act);
-              o.store(p.out + row + c0 + g * 8);
+              for (int e = 0; e < 8; ++e) v[g * 8 + e] += r.v[e];
             }
+            Vec16<bf16> o;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) o.v[e] = apply_act(v[g * 8 + e], p.act);
+            o.store(chunk);
           }
         }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the TMA unit
+        __syncwarp();
+        if (lane == 0 && m0 + q * 32 < p.M) {  // rows past M and columns past N are clipped by the TMA unit
+          tma_store_2d(&tmO, io_s + h * 16384 + q * 4096, n0 + h * 64, m0 + q * 32);
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          stored = true;
+        }
       }
+      if (stored) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // shared memory is read before the CTA retires
     }
   }
   tc_fence_before();
@@ -362,9 +405,10 @@ struct TcLayer {
   struct Cached {
     const void* ptr;
     int batch;
+    int kind;  // 0: operand A, 1: residual / output matrix
     CUtensorMap tm;
   };
-  mutable std::vector<Cached> a_maps;  // activation tensor maps by (source pointer, batch)
+  mutable std::vector<Cached> a_maps;  // tensor maps of caller buffers by (pointer, batch, kind)
   mutable size_t next_evict = 0;
 };
 
@@ -376,8 +420,10 @@ inline ee_status_t tc_context_init(TcContext& c) {
   f = nullptr;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f, cudaEnableDefault, &q) != cudaSuccess || !f) return EE_ERR_CUDA;
   c.encode_im2col = (PFN_encodeIm2col)f;
-  if (cudaFuncSetAttribute(conv_igemm_tcgen05_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<64>::kBytes) != cudaSuccess ||
-      cudaFuncSetAttribute(conv_igemm_tcgen05_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<128>::kBytes) != cudaSuccess)
+  if (cudaFuncSetAttribute(conv_igemm_tcgen05_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<64, false>::kBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(conv_igemm_tcgen05_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<64, true>::kBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(conv_igemm_tcgen05_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<128, false>::kBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(conv_igemm_tcgen05_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<128, true>::kBytes) != cudaSuccess)
     return EE_ERR_CUDA;
   return EE_OK;
 }
@@ -409,24 +455,35 @@ inline ee_status_t tc_plan_layer(TcContext& c, const ee_layer_desc_t& d, int in_
   return r == CUDA_SUCCESS ? EE_OK : EE_ERR_CUDA;
 }
 
-// The map covers exactly `batch` samples: rows past them are out of bounds for the TMA unit and read as zero,
-// so no byte beyond the caller's [batch] samples is ever touched.
-inline ee_status_t tc_activation_map(const TcContext& c, const TcLayer& L, const void* src, int batch, const CUtensorMap** out) {
+// Tensor map of a caller buffer, cached by (pointer, batch, kind).  kind 0: operand A of the layer; kind 1: a
+// [batch*Ho*Wo][Cout] matrix (residual or output) with a 64 x 32 box.  A map covers exactly `batch` samples: rows
+// past them are out of bounds for the TMA unit (reads give zero, writes are dropped), so no byte beyond the
+// caller's [batch] samples is ever touched.
+inline ee_status_t tc_buffer_map(const TcContext& c, const TcLayer& L, const void* ptr, int batch, int kind, const CUtensorMap** out) {
   for (auto& e : L.a_maps)
-    if (e.ptr == src && e.batch == batch) {
+    if (e.ptr == ptr && e.batch == batch && e.kind == kind) {
       *out = &e.tm;
       return EE_OK;
     }
   TcLayer::Cached e;
-  e.ptr = src;
+  e.ptr = ptr;
   e.batch = batch;
+  e.kind = kind;
   CUresult r;
-  if (!L.im2col) {
+  if (kind == 1) {
+    const cuuint64_t dims[2] = {(cuuint64_t)L.cout, (cuuint64_t)batch * L.out_h * L.out_w};
+    const cuuint64_t strides[1] = {(cuuint64_t)L.cout * 2};
+    const cuuint32_t box[2] = {64, 32};
+    const cuuint32_t es[2] = {1, 1};
+    r = c.encode_tiled(&e.tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else if (!L.im2col) {
     const cuuint64_t dims[2] = {(cuuint64_t)L.cin, (cuuint64_t)batch * L.in_h * L.in_w};
     const cuuint64_t strides[1] = {(cuuint64_t)L.cin * 2};
     const cuuint32_t box[2] = {kTcBK, kTcBM};
     const cuuint32_t es[2] = {1, 1};
-    r = c.encode_tiled(&e.tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(src), dims, strides, box, es,
+    r = c.encode_tiled(&e.tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else {
@@ -436,12 +493,12 @@ inline ee_status_t tc_activation_map(const TcContext& c, const TcLayer& L, const
     const int lower[2] = {-L.pad, -L.pad};
     const int upper[2] = {L.pad - (L.kw - 1), L.pad - (L.kh - 1)};
     const cuuint32_t es[4] = {1, (cuuint32_t)L.stride, (cuuint32_t)L.stride, 1};
-    r = c.encode_im2col(&e.tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(src), dims, strides, lower, upper, kTcBK,
+    r = c.encode_im2col(&e.tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, lower, upper, kTcBK,
                         kTcBM, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   }
   if (r != CUDA_SUCCESS) return EE_ERR_CUDA;
-  if (L.a_maps.size() < 16) {
+  if (L.a_maps.size() < 48) {
     L.a_maps.push_back(e);
     *out = &L.a_maps.back().tm;
   } else {
@@ -452,12 +509,37 @@ inline ee_status_t tc_activation_map(const TcContext& c, const TcLayer& L, const
   return EE_OK;
 }
 
+template <int BN, bool RES>
+inline cudaError_t tc_launch_t(dim3 grid, cudaStream_t st, const CUtensorMap& a, const CUtensorMap& w, const CUtensorMap& r,
+                               const CUtensorMap& o, const TcParams& p) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = TcSmem<BN, RES>::kBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;  // prologue may overlap the previous kernel's tail
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_kernel<BN, RES>, a, w, r, o, p);
+}
+
 inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, const void* res, void* dst, int B, const float* scale,
                              const float* bias, int* err_flag, cudaStream_t st) {
   if (((uintptr_t)src & 15) || ((uintptr_t)dst & 15) || ((uintptr_t)res & 15)) return EE_ERR_INVALID_ARG;
-  const CUtensorMap* tmA = nullptr;
-  ee_status_t s = tc_activation_map(c, L, src, B, &tmA);
+  // copies: a later lookup may grow the cache and move its entries
+  const CUtensorMap* t = nullptr;
+  ee_status_t s = tc_buffer_map(c, L, src, B, 0, &t);
   if (s != EE_OK) return s;
+  const CUtensorMap tmA = *t;
+  if ((s = tc_buffer_map(c, L, dst, B, 1, &t)) != EE_OK) return s;
+  const CUtensorMap tmO = *t;
+  CUtensorMap tmR = tmO;
+  if (res) {
+    if ((s = tc_buffer_map(c, L, res, B, 1, &t)) != EE_OK) return s;
+    tmR = *t;
+  }
   TcParams p;
   p.M = B * L.out_h * L.out_w;
   p.N = L.cout;
@@ -472,11 +554,12 @@ inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, co
   p.out = (bf16*)dst;
   p.err_flag = err_flag;
   dim3 grid(cdiv(p.M, kTcBM), cdiv(L.cout, L.bn));
+  cudaError_t e;
   if (L.bn == 128)
-    conv_igemm_tcgen05_kernel<128><<<grid, kTcThreads, TcSmem<128>::kBytes, st>>>(*tmA, L.tm_w, p);
+    e = res ? tc_launch_t<128, true>(grid, st, tmA, L.tm_w, tmR, tmO, p) : tc_launch_t<128, false>(grid, st, tmA, L.tm_w, tmR, tmO, p);
   else
-    conv_igemm_tcgen05_kernel<64><<<grid, kTcThreads, TcSmem<64>::kBytes, st>>>(*tmA, L.tm_w, p);
-  return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+    e = res ? tc_launch_t<64, true>(grid, st, tmA, L.tm_w, tmR, tmO, p) : tc_launch_t<64, false>(grid, st, tmA, L.tm_w, tmR, tmO, p);
+  return e == cudaSuccess ? EE_OK : EE_ERR_CUDA;
 }
 
 }  // namespace ee
