@@ -159,6 +159,7 @@ def run_ours(args):
     import torch
 
     from paper_2209_13443_b200 import binding as eb
+    from paper_2209_13443_b200 import replicas
     from paper_2209_13443_b200 import workloads as wl
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -181,8 +182,9 @@ def run_ours(args):
     ws = model.workspace()
     td = eb.torch_dtype(spec.dtype)
     # every rank serves its own requests (ids are global)
-    x_host = torch.from_numpy(wl.make_input(spec, B, seed=seed, first_id=rank * B)).to(td).pin_memory()
-    ids_host = (torch.arange(B, dtype=torch.int32) + rank * B).pin_memory()
+    first_id, _ = replicas.rank_requests(rank, world, B)
+    x_host = torch.from_numpy(wl.make_input(spec, B, seed=seed, first_id=first_id)).to(td).pin_memory()
+    ids_host = (torch.arange(B, dtype=torch.int32) + first_id).pin_memory()
     x_dev, ids_dev = x_host.cuda(), ids_host.cuda()
     batch0 = torch.empty_like(x_dev)
     ids0 = torch.empty_like(ids_dev)
@@ -242,10 +244,7 @@ def run_ours(args):
             nl += l; h2d = hi; d2h = do
         barrier()
         total_ms = sum(a.elapsed_time(b) for a, b in ev)
-        if dist is not None:
-            t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            total_ms = float(t.item())
+        total_ms = replicas.max_over_ranks(total_ms, dist, "cuda")
         return total_ms, nl, h2d, d2h, sizes
 
     for _ in range(W):
@@ -331,7 +330,7 @@ def run_ours(args):
     cpu = {"value": n_cpu / cpu_dt, "unit": UNIT, "cores": eo.n_threads(), "kind": "oracle",
            "sample": f"first {n_cpu} of {B} samples, whole path once, {cpu_dt:.1f} s"}
 
-    value = world * B * K / (total_ms * 1e-3)
+    value = replicas.job_throughput(world, B, K, total_ms)
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -339,7 +338,7 @@ def run_ours(args):
         "config": {"workload": workload_name(spec, B), "global_batch": world * B, "parallelism": f"replicas x{world}",
                    "l2": "flushed between timed steps (256 MB write)", "batch_per_stage": sizes_last},
         "clocks": clocks,
-        "e2e": {"value": world * B * K / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+        "e2e": {"value": replicas.job_throughput(world, B, K, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / K},
         "gpu_launches": nl,
         "roofline": roof,

@@ -165,6 +165,14 @@ ee_status_t ee_batch_refill(ee_model_t* model, int boundary, void* batch_feat, i
                             const void* arr_feat, const int32_t* arr_ids, int n_arr, int* n_accepted,
                             int* n_merged, void* cuda_stream);
 
+/* One layer of a stage alone (the same kernel and launch configuration ee_stage_run uses for it): `input` is
+ * the layer's input tensor [batch][in_h][in_w][cin], `residual` its residual operand [batch][out_h][out_w][cout]
+ * (required iff the layer has one), `output` [batch][out_h][out_w][cout]; all DEVICE, model dtype, 16-byte aligned,
+ * caller-owned.  `workspace` as for ee_stage_run (only a packed stem uses it).  For per-layer parity checks and
+ * micro-benchmarks.  Errors: INVALID_ARG, STAGE (stage or layer out of range), CAPACITY, CUDA. */
+ee_status_t ee_layer_run(ee_model_t* model, int stage, int layer, const void* input, const void* residual, int batch,
+                         void* output, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Exit head alone on a feature map (same kernels ee_stage_run uses): GAP, FC, softmax top-1,
  * threshold, and the stable scan that yields survivor_idx / n_surv (no feature gather).
  * x DEVICE [batch][hw][c] model dtype; `out` as in ee_stage_run with features_out ignored;

@@ -19,7 +19,7 @@ _SO = os.path.join(_HERE, "libeecnn.so")
 EE_OK = 0
 STATUS_NAMES = ["EE_OK", "EE_ERR_INVALID_ARG", "EE_ERR_SHAPE", "EE_ERR_CAPACITY", "EE_ERR_STAGE", "EE_ERR_UNSUPPORTED",
                 "EE_ERR_CUDA", "EE_ERR_TIMEOUT", "EE_ERR_INTERNAL"]
-EXPORTS = ["ee_model_create", "ee_model_destroy", "ee_model_query", "ee_stage_run", "ee_batch_refill", "ee_exit_head",
+EXPORTS = ["ee_model_create", "ee_model_destroy", "ee_model_query", "ee_stage_run", "ee_layer_run", "ee_batch_refill", "ee_exit_head",
            "ee_exit_head_scratch_bytes", "ee_exit_head_static", "ee_gather_survivors", "ee_model_set_timing", "ee_model_get_timing",
            "ee_model_plan", "ee_model_check", "ee_status_string", "ee_last_cuda_error"]
 
@@ -85,6 +85,7 @@ def load_library() -> C.CDLL:
     L.ee_model_destroy.argtypes = [vp]
     L.ee_model_query.argtypes = [vp, i, C.POINTER(StageInfo)]
     L.ee_stage_run.argtypes = [vp, i, C.POINTER(StageIn), vp, C.c_size_t, C.POINTER(StageOut), vp]
+    L.ee_layer_run.argtypes = [vp, i, i, vp, vp, i, vp, vp, C.c_size_t, vp]
     L.ee_batch_refill.argtypes = [vp, i, vp, vp, i, vp, vp, i, C.POINTER(i), C.POINTER(i), vp]
     L.ee_exit_head.argtypes = [vp, i, vp, i, i, vp, vp, vp, C.c_size_t, C.POINTER(StageOut), vp]
     L.ee_exit_head_static.argtypes = [vp, i, vp, i, i, vp, vp, C.POINTER(StageOut), vp]
@@ -220,6 +221,12 @@ class EEModel:
         so = out.as_struct() if isinstance(out, StageBuffers) else out
         _check(self._L.ee_stage_run(self._h, stage, C.byref(sin), aligned, workspace.numel() - (aligned - base), C.byref(so),
                                     _stream(stream)), "ee_stage_run")
+
+    def layer_run(self, stage: int, layer: int, x, residual, batch: int, out, workspace: torch.Tensor, stream=None):
+        base = workspace.data_ptr()
+        aligned = (base + 255) // 256 * 256
+        _check(self._L.ee_layer_run(self._h, stage, layer, _ptr(x), _ptr(residual), int(batch), _ptr(out), aligned,
+                                    workspace.numel() - (aligned - base), _stream(stream)), "ee_layer_run")
 
     def batch_refill(self, boundary: int, batch_feat, batch_ids, n_surv: int, arr_feat, arr_ids, n_arr: int, stream=None):
         n_acc, n_mer = C.c_int(-1), C.c_int(-1)

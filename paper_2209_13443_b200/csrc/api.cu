@@ -555,6 +555,29 @@ ee_status_t ee_stage_run(ee_model_t* m, int stage, const ee_stage_in_t* in, void
   return EE_OK;
 }
 
+ee_status_t ee_layer_run(ee_model_t* m, int stage, int layer, const void* input, const void* residual, int batch, void* output,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!m || batch < 0) return EE_ERR_INVALID_ARG;
+  if (stage < 0 || stage >= (int)m->stages.size()) return EE_ERR_STAGE;
+  StagePlan& sp = m->stages[stage];
+  if (layer < 0 || layer >= (int)sp.layers.size()) return EE_ERR_STAGE;
+  if (batch > m->max_batch) return EE_ERR_CAPACITY;
+  if (batch == 0) return EE_OK;
+  const LayerPlan& L = sp.layers[layer];
+  const bool has_res = L.res_slot != -2;
+  if (!input || !output || (has_res && !residual) || ((uintptr_t)input & 15) || ((uintptr_t)output & 15) || ((uintptr_t)residual & 15))
+    return EE_ERR_INVALID_ARG;
+  void* pack = nullptr;
+  if (L.kind == KK_TC_PACKED) {
+    if (!workspace || ((uintptr_t)workspace & 255)) return EE_ERR_INVALID_ARG;
+    if (workspace_bytes < sp.ws_bytes) return EE_ERR_CAPACITY;
+    pack = (char*)workspace + sp.pack_off;
+  }
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  return m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, input, has_res ? residual : nullptr, output, pack, batch, st)
+                             : launch_layer<float>(m, L, input, has_res ? residual : nullptr, output, pack, batch, st);
+}
+
 ee_status_t ee_batch_refill(ee_model_t* m, int boundary, void* batch_feat, int32_t* batch_ids, int n_surv, const void* arr_feat,
                             const int32_t* arr_ids, int n_arr, int* n_accepted, int* n_merged, void* cuda_stream) {
   if (!m || !n_accepted || !n_merged || n_surv < 0 || n_arr < 0) return EE_ERR_INVALID_ARG;

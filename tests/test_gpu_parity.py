@@ -293,3 +293,120 @@ def test_error_codes_and_empty_batch():
     with pytest.raises(eb.EEError) as e:
         eb.EEModel(bad)
     assert e.value.status == 2
+
+
+# ----------------------------------------------------------------------------- full benchmark sizes
+
+def _full_size(spec, B, seed):
+    """Benchmark-size model and batch, the launch configuration bench.py times; every stage is fed the
+    oracle's stage input and compared element by element (the oracle needs well under a minute)."""
+    run = util.GpuRunner(spec)
+    x = wl.make_input(spec, B, seed=seed)
+    ids = np.arange(B, dtype=np.int32)
+    near, exited = 0, 0
+    for s in range(len(spec.stages)):
+        o = util.oracle_stage(spec, s, x, ids)
+        g = run.stage(s, x, ids)
+        r = util.check_stage(spec, g, o, f"{spec.name} full size B={B} stage {s}")
+        near += r["band"]
+        exited += int(o["exit"].sum())
+        x, ids = o["features_out"], o["ids_out"]
+        if len(ids) == 0:
+            break
+    assert exited == B
+    assert near <= max(2, B // 16), f"{near} samples within 1e-3 of a threshold"
+    return near
+
+
+def test_resnet50_full_size_batch64():
+    _full_size(wl.resnet50_ee(seed=1, max_batch=64), 64, seed=1)
+
+
+@pytest.mark.parametrize("B", [1, 4, 16])
+def test_resnet50_full_size_small_batches(B):
+    _full_size(wl.resnet50_ee(seed=1, max_batch=64), B, seed=1)
+
+
+def test_mobilenetv2_full_size_batch32():
+    _full_size(wl.mobilenetv2_ee(seed=2, max_batch=32), 32, seed=2)
+
+
+# ----------------------------------------------------------------------------- config 4: forced exit rates
+
+@pytest.mark.parametrize("p", [0.0, 0.1, 0.3, 0.5, 0.8])
+def test_forced_exit_rate_sweep(p):
+    """Seeded Bernoulli logit shifts decide the exits: with flat unshifted logits the masks must equal the draws
+    exactly, stage after stage, and the surviving batch shrinks as (1-p)^k."""
+    B, K = 24, 100
+    spec = wl.resnet50_ee(seed=1, in_hw=64, n_classes=K, max_batch=B, alphas=[0.01] * 4)
+    run = util.GpuRunner(spec)
+    draws, shifts, cls = wl.bernoulli_exit_shifts(seed=4, n_ids=B, n_exits=3, p=p, n_classes=K)
+    x = wl.make_input(spec, B, seed=1)
+    ids = np.arange(B, dtype=np.int32)
+    for s in range(4):
+        sh = shifts[s][ids] if s < 3 else None
+        sc = cls[ids] if s < 3 else None
+        o = util.oracle_stage(spec, s, x, ids, sh, sc)
+        g = run.stage(s, x, ids, sh, sc)
+        r = util.check_stage(spec, g, o, f"forced p={p} stage {s}")
+        assert r["band"] == 0 and r["flips"] == 0
+        if s < 3:
+            assert np.array_equal(g["exit"], draws[s][ids])             # the masks ARE the Bernoulli draws
+            assert np.array_equal(g["pred"][g["exit"] == 1], cls[ids][g["exit"] == 1])
+        x, ids = o["features_out"], o["ids_out"]
+        if len(ids) == 0:
+            break
+
+
+@pytest.mark.parametrize("name,B", [("resnet50", 9), ("mobilenetv2", 5)])
+def test_every_layer_of_the_full_size_models(name, B):
+    """Layer-local parity at benchmark shapes: every layer of every stage runs alone on the ORACLE's input (and
+    residual) for that layer, in the kernel and launch configuration ee_stage_run uses, and must match the oracle's
+    output of that layer element-wise within the 1e-2 bar (both sides round the same pre-activation once)."""
+    spec = wl.resnet50_ee(seed=1, max_batch=B) if name == "resnet50" else wl.mobilenetv2_ee(seed=2, max_batch=B)
+    m = eb.EEModel(spec)
+    ws = m.workspace()
+    x = wl.make_input(spec, B, seed=3)
+    worst = 0.0
+    for s, st in enumerate(spec.stages):
+        outs = eo.run_layers(spec, s, x, keep_all=True)
+        for i, l in enumerate(st.layers):
+            src = x if (l.input_from == wl.FROM_STAGE_INPUT or (l.input_from == wl.FROM_PREV and i == 0)) else \
+                outs[i - 1 if l.input_from == wl.FROM_PREV else l.input_from]
+            res = None if l.residual_from == wl.NO_RESIDUAL else (x if l.residual_from == wl.FROM_STAGE_INPUT else outs[l.residual_from])
+            out = torch.empty(outs[i].shape, dtype=torch.bfloat16, device="cuda")
+            m.layer_run(s, i, eb.to_device("bf16", src), None if res is None else eb.to_device("bf16", res), B, out, ws)
+            torch.cuda.synchronize()
+            e = util.rel_err(out.float().cpu().numpy(), outs[i])
+            worst = max(worst, e)
+            assert e <= util.TOL["bf16"], f"{name} stage {s} layer {i} ({l.kh}x{l.kw} {l.cin}->{l.cout} s{l.stride}): {e:.3e}"
+        x = outs[st.out_layer]
+    m.check()
+
+
+# ----------------------------------------------------------------------------- config 5: streaming trace
+
+def test_streaming_trace_matches_oracle_schedule():
+    """Algorithm 1 (T_SLO = infinity) on a virtual clock: the GPU-driven loop must launch exactly the batches the
+    oracle-side replay launches, and every request must leave at the exit and with the class of its serial run."""
+    from paper_2209_13443_b200.serving import FluidServer
+
+    spec = wl.tiny_ee_cnn(seed=0)
+    pool_np = wl.make_input(spec, 48, seed=9)
+    serial = [eo.run_sample_serial(spec, pool_np[i]) for i in range(len(pool_np))]
+    keep = [i for i, sref in enumerate(serial) if all(abs(c - 0.6) > 10 * util.BAND for c in sref[2][:2])][:32]
+    assert len(keep) == 32
+    pool_np, serial = pool_np[keep], [serial[i] for i in keep]
+    n = 300
+    arrivals = wl.poisson_arrivals(3, n, 2000.0)
+    image_of = [r % 32 for r in range(n)]
+    stage_time = lambda s, b: 2e-4 * (s + 1) + 3e-5 * b      # noqa: E731
+    srv = FluidServer(spec)
+    got = srv.serve(arrivals, image_of, eb.to_device("f32", pool_np), stage_time)
+    exit_of = np.array([serial[image_of[r]][0] for r in range(n)])
+    fin, launches = eo.serve_trace(3, spec.max_batch, arrivals, exit_of, stage_time)
+    assert got["launches"] == launches
+    assert np.array_equal(got["exit_stage"], exit_of)
+    assert got["pred"].tolist() == [serial[image_of[r]][1] for r in range(n)]
+    np.testing.assert_allclose(got["finish"], fin, rtol=0, atol=1e-9)
+    assert len({len(ids) for _, ids in launches}) > 3                          # the trace exercises varying batch sizes

@@ -18,6 +18,12 @@ from paper_2209_13443_b200 import workloads as wl
 # error in ANY fp32 summation order.  FLOOR = 0.05 keeps the bar meaningful for every element that
 # matters and still bounds the small ones in absolute terms (tol * 0.05 * scale).
 TOL = {"f32": 1e-5, "bf16": 1e-2}
+# Whole stages of a bf16 model (10-19 layers, each output rounded to bf16 on both sides) are held to two bf16 ulps in
+# the max-norm, 2^-6: a legitimate last-bit difference early in the chain moves later pre-rounding values across
+# rounding boundaries, so the largest elements of a 10^7-element map end up one to two ulps (2^-7 each at the bottom
+# of a binade) apart in ANY correct implementation.  The 1e-2 bar itself is enforced layer by layer
+# (test_every_layer_of_the_full_size_models), where both sides round the same pre-activation once.
+STAGE_TOL = {"f32": 1e-5, "bf16": 2.0 ** -6}
 FLOOR = 0.05
 BAND = 1e-3   # samples whose oracle confidence is within BAND of the threshold may flip; they are listed and counted
 
@@ -86,12 +92,13 @@ def check_stage(spec, g: dict, o: dict, where="", tol=None, elementwise=False):
     perturbs every downstream pre-rounding value, and each perturbed value that straddles a bf16
     rounding boundary moves by a full ulp (2^-8 relative), so individual elements drift by a few
     percent in any summation order while the max-norm error stays near one ulp."""
-    tol = TOL[spec.dtype] if tol is None else tol
+    if tol is None:
+        tol = TOL[spec.dtype] if elementwise else STAGE_TOL[spec.dtype]
     ferr = rel_err if elementwise else norm_err
     B = len(o["conf"])
     st_thr = o.get("threshold")
     e_z = ferr(g["z"], o["z"])
-    assert e_z <= tol, f"{where}: logits rel err {e_z:.3e} > {tol}"
+    assert e_z <= TOL[spec.dtype], f"{where}: logits rel err {e_z:.3e} > {TOL[spec.dtype]}"
     # softmax top-1 is 1/2-Lipschitz in the max-norm of the logits (d conf = conf (1 - conf) d(z_top - z_k)):
     # the confidence may move by at most half the largest logit difference, plus fp32 rounding of the exp-sum
     dz = np.max(np.abs(g["z"] - o["z"]), axis=1) if B else np.zeros(0)
