@@ -19,6 +19,7 @@
 #pragma once
 #include <cuda.h>
 
+#include <algorithm>
 #include <vector>
 
 #include "common.cuh"
@@ -27,7 +28,6 @@ namespace ee {
 
 constexpr int kTcBM = 128;       // output pixels per CTA (= TMEM lanes)
 constexpr int kTcBK = 64;        // bf16 elements per K block: 128 bytes = one swizzle span
-constexpr int kTcStages = 3;      // 96 KB of tiles at BN = 128: two CTAs per SM, one's epilogue overlaps the other's main loop
 constexpr int kTcThreads = 192;  // producer warp, MMA warp, four epilogue warps
 constexpr long long kTcWaitCycles = 4000000000LL;  // ~2 s at boost clock; far beyond any healthy wait
 
@@ -43,6 +43,7 @@ struct TcParams {
   const bf16* residual;
   bf16* out;
   int* err_flag;
+  int kb_per;           // split-K: K blocks per range (a property of the layer)
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -142,13 +143,15 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 
 // ----------------------------------------------------------------------------- kernel
 
-// Shared-memory plan of one CTA.  Layers with a residual operand keep a dedicated 128 x BN bf16 tile that the
-// producer fills with the residual at kernel start and the epilogue overwrites in place with the output; they run
-// a two-stage operand ring.  Layers without one run three stages and stage their output in ring slot 0 once the
-// main loop has drained it.  Either way 96 KB at BN = 128: two CTAs per SM.
-template <int BN, bool RES>
+// Shared-memory plan of one CTA: a ring of STAGES operand slots (A 16 KB + W BN*128 B each), then, for layers whose
+// residual operand is prefetched (RES), a dedicated 128 x BN bf16 tile that the producer fills with the residual at
+// kernel start and the epilogue overwrites in place with the output.  Without it the output is staged in ring slot
+// 0 once the main loop has drained it.  The shallow variants (3 slots, or 2 + residual tile: 96 KB at BN = 128) let
+// two CTAs share an SM so one's epilogue overlaps the other's main loop; the deep variants (6, or 5 + tile) are
+// used when the grid has at most one CTA per SM anyway and a longer ring hides more TMA latency.
+template <int BN, int STAGES, bool RES>
 struct TcSmem {
-  static constexpr int kStages = RES ? 2 : 3;
+  static constexpr int kStages = STAGES;
   static constexpr int kABytes = kTcBM * kTcBK * 2;
   static constexpr int kBBytes = BN * kTcBK * 2;
   static constexpr int kStage = kABytes + kBBytes;
@@ -158,6 +161,7 @@ struct TcSmem {
   static constexpr int kAfter = kTiles + (RES ? kIoBytes : 0);
   static constexpr int kBytes = kAfter + 2 * BN * 4 + 256 + 1024;  // + scale/bias, barriers, alignment slack
   static_assert(RES || kIoBytes <= kStage, "output staging must fit in ring slot 0");
+  static_assert(kBytes <= 227 * 1024, "exceeds the shared memory of an SM");
 };
 
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int c0, int c1) {
@@ -167,12 +171,19 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src
 
 // tmA: activations (2-D tile map or im2col map), tmW: weights [Cin][taps][Cout], tmR / tmO: residual and output as
 // [rows][Cout] matrices with a 64-column x 32-row box (128-byte swizzle).
-template <int BN, bool RES>
+//
+// SPLIT: the K loop of one output tile is cut into gridDim.z (2, 4 or 8) fixed ranges of p.kb_per K blocks, a
+// property of the layer and never of the batch.  The CTAs of a tile form a thread-block cluster along z: each leaves
+// its fp32 partial tile in its own shared memory, then every CTA reduces one slice of rows by reading all partials
+// through distributed shared memory in ascending range order (a reduce-scatter), applies the epilogue to that
+// slice and stores it.
+template <int BN, int STAGES, bool RES, bool SPLIT>
 __global__ void __launch_bounds__(kTcThreads, 2)
 conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                           const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmO, TcParams p) {
+  static_assert(!(RES && SPLIT), "split-K tiles read their residual with plain loads");
   extern __shared__ uint8_t smem_raw[];
-  using S = TcSmem<BN, RES>;
+  using S = TcSmem<BN, STAGES, RES>;
   constexpr int kStages = S::kStages;
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
@@ -189,7 +200,10 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * kTcBM, n0 = blockIdx.y * BN;
-  const int num_kb = p.taps * p.cblocks;
+  const int num_kb_all = p.taps * p.cblocks;
+  const int kb_begin = SPLIT ? (int)blockIdx.z * p.kb_per : 0;
+  const int kb_end = SPLIT ? min(num_kb_all, kb_begin + p.kb_per) : num_kb_all;
+  const int num_kb = kb_end - kb_begin;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -199,6 +213,12 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
     mbar_init(accum_bar, 1);
     mbar_init(res_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0 && lane == 0) {  // descriptor fetches overlap the rest of the prologue
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmO) : "memory");
+    if (RES) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmR) : "memory");
   }
   if (warp == 1) {  // TMEM: BN fp32 columns x 128 lanes
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN) : "memory");
@@ -233,9 +253,10 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
         cw = (rem - ho * p.Wo) * p.stride - p.pad;
         ch = ho * p.stride - p.pad;
       }
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % kStages;
-        const uint32_t ph = (uint32_t)(kb / kStages) & 1u;
+      for (int i = 0; i < num_kb; ++i) {
+        const int kb = kb_begin + i;
+        const int s = i % kStages;
+        const uint32_t ph = (uint32_t)(i / kStages) & 1u;
         if (!mbar_wait(empty_bar(s), ph ^ 1u, p.err_flag)) break;
         const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
         const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
@@ -253,19 +274,19 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc(BN);
       bool ok = true;
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % kStages;
-        const uint32_t ph = (uint32_t)(kb / kStages) & 1u;
+      for (int i = 0; i < num_kb; ++i) {
+        const int s = i % kStages;
+        const uint32_t ph = (uint32_t)(i / kStages) & 1u;
         ok = mbar_wait(full_bar(s), ph, p.err_flag);
         if (!ok) break;
         tc_fence_after();
         const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
 #pragma unroll
         for (int k = 0; k < kTcBK / 16; ++k)
-          umma_bf16(tmem_base, umma_desc(sa + k * 32), umma_desc(sb + k * 32), idesc, (uint32_t)((kb | k) != 0));
+          umma_bf16(tmem_base, umma_desc(sa + k * 32), umma_desc(sb + k * 32), idesc, (uint32_t)((i | k) != 0));
         umma_commit(empty_bar(s));  // frees the stage once these MMAs have read it
       }
-      if (ok) umma_commit(accum_bar);  // accumulator complete: every MMA has also finished reading the ring
+      if (ok && num_kb > 0) umma_commit(accum_bar);  // accumulator complete: every MMA has also finished reading the ring
     }
   } else {
     const int et = threadIdx.x - 64;  // 0..127
@@ -276,11 +297,33 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");
     // warp-uniform outcomes: tcgen05.ld is a warp-wide instruction
-    bool ok = __all_sync(0xffffffffu, mbar_wait(accum_bar, 0, p.err_flag));
+    bool ok = num_kb > 0 ? __all_sync(0xffffffffu, mbar_wait(accum_bar, 0, p.err_flag)) : true;
     if (RES) ok = __all_sync(0xffffffffu, mbar_wait(res_bar, 0, p.err_flag)) && ok;
     tc_fence_after();
-    if (ok) {
-      const int q = warp & 3;  // TMEM lane quarter this warp may read = rows [32q, 32q + 32) of the tile
+    const int q = warp & 3;  // TMEM lane quarter this warp may read = rows [32q, 32q + 32) of the tile
+    const int row = q * 32 + lane;
+    if (SPLIT) {
+      // fp32 partial tile [128 rows][BN] into the drained ring; 16-byte chunks XOR-swizzled with the row so that
+      // neither these row-wise writes nor the peers' reads pile onto one bank
+      constexpr int CH = BN / 4;
+      float* part = reinterpret_cast<float*>(gen);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        float v[32];
+        if (ok && num_kb > 0) {
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = 0.f;
+        }
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          const int c = (c0 >> 2) + g;
+          *reinterpret_cast<float4*>(part + (size_t)row * BN + ((c ^ (row & (CH - 1))) << 2)) =
+              make_float4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+        }
+      }
+    } else if (ok) {
       uint8_t* io = gen + S::kIoOff;
       const uint32_t io_s = base + S::kIoOff;
       bool stored = false;
@@ -289,13 +332,14 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
         if (n0 + h * 64 >= p.N) break;
         // this thread's 128-byte line of the 64-column half; its eight 16-byte chunks are XOR-swizzled with the
         // row index so that the TMA unit (128-byte swizzle) finds row-major data
-        uint8_t* line = io + h * 16384 + (q * 32 + lane) * 128;
+        uint8_t* line = io + h * 16384 + row * 128;
 #pragma unroll
         for (int sub = 0; sub < 2; ++sub) {
+          const int c0 = h * 64 + sub * 32;
           float v[32];
-          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 64 + sub * 32), v);
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = fmaf(s_scale[h * 64 + sub * 32 + j], v[j], s_bias[h * 64 + sub * 32 + j]);
+          for (int j = 0; j < 32; ++j) v[j] = fmaf(s_scale[c0 + j], v[j], s_bias[c0 + j]);
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
             bf16* chunk = reinterpret_cast<bf16*>(line + (((sub * 4 + g) ^ (lane & 7)) << 4));
@@ -321,6 +365,63 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
       }
       if (stored) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // shared memory is read before the CTA retires
     }
+  }
+  if (SPLIT) {
+    // every thread of every CTA of the cluster passes both barriers, whatever happened above
+    asm volatile("barrier.cluster.arrive.release;\n barrier.cluster.wait.acquire;" ::: "memory");
+    if (warp >= 2) {
+      constexpr int CH = BN / 4, G = BN / 8;     // 16-byte fp32 chunks and 8-column groups per row
+      const int et = threadIdx.x - 64;
+      const int nsplit = (int)gridDim.z;
+      uint32_t rank;
+      asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+      const int rows_per = kTcBM / nsplit;
+      const uint32_t part_s = base;             // same offset in every CTA of the cluster
+      for (int item = et; item < rows_per * G; item += 128) {
+        const int r = item / G, g = item - r * G;
+        const int trow = (int)rank * rows_per + r;
+        const int m = m0 + trow, n = n0 + g * 8;
+        const uint32_t a0 = part_s + (uint32_t)trow * (BN * 4) + (uint32_t)(((2 * g) ^ (trow & (CH - 1))) << 4);
+        const uint32_t a1 = part_s + (uint32_t)trow * (BN * 4) + (uint32_t)(((2 * g + 1) ^ (trow & (CH - 1))) << 4);
+        float v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = 0.f;
+        float4 x0[8], x1[8];
+#pragma unroll
+        for (int z = 0; z < 8; ++z) {             // all remote loads in flight before the first addition
+          if (z < nsplit) {
+            uint32_t ra0, ra1;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra0) : "r"(a0), "r"(z));
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra1) : "r"(a1), "r"(z));
+            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(x0[z].x), "=f"(x0[z].y), "=f"(x0[z].z), "=f"(x0[z].w) : "r"(ra0) : "memory");
+            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(x1[z].x), "=f"(x1[z].y), "=f"(x1[z].z), "=f"(x1[z].w) : "r"(ra1) : "memory");
+          }
+        }
+#pragma unroll
+        for (int z = 0; z < 8; ++z) {             // ascending range order: the grouping of the sum is fixed by the layer
+          if (z < nsplit) {
+            v[0] += x0[z].x; v[1] += x0[z].y; v[2] += x0[z].z; v[3] += x0[z].w;
+            v[4] += x1[z].x; v[5] += x1[z].y; v[6] += x1[z].z; v[7] += x1[z].w;
+          }
+        }
+        if (m < p.M && n < p.N) {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) v[e] = fmaf(s_scale[g * 8 + e], v[e], s_bias[g * 8 + e]);
+          if (p.residual) {
+            Vec16<bf16> rr;
+            rr.load(p.residual + (size_t)m * p.N + n);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[e] += rr.v[e];
+          }
+          Vec16<bf16> o;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) o.v[e] = apply_act(v[e], p.act);
+          o.store(p.out + (size_t)m * p.N + n);
+        }
+      }
+    }
+    // no CTA may retire while a peer still reads its shared memory
+    asm volatile("barrier.cluster.arrive.release;\n barrier.cluster.wait.acquire;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
@@ -401,6 +502,7 @@ struct TcLayer {
   int in_h = 0, in_w = 0, out_h = 0, out_w = 0, max_batch = 0;
   int bn = 128;
   bool im2col = false;
+  int splits = 1, kb_per = 0;    // split-K ranges of this layer (fixed per layer, independent of the batch)
   CUtensorMap tm_w;
   struct Cached {
     const void* ptr;
@@ -420,11 +522,21 @@ inline ee_status_t tc_context_init(TcContext& c) {
   f = nullptr;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f, cudaEnableDefault, &q) != cudaSuccess || !f) return EE_ERR_CUDA;
   c.encode_im2col = (PFN_encodeIm2col)f;
-  if (cudaFuncSetAttribute(conv_igemm_tcgen05_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<64, false>::kBytes) != cudaSuccess ||
-      cudaFuncSetAttribute(conv_igemm_tcgen05_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<64, true>::kBytes) != cudaSuccess ||
-      cudaFuncSetAttribute(conv_igemm_tcgen05_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<128, false>::kBytes) != cudaSuccess ||
-      cudaFuncSetAttribute(conv_igemm_tcgen05_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<128, true>::kBytes) != cudaSuccess)
-    return EE_ERR_CUDA;
+  cudaError_t e = cudaSuccess;
+  auto set = [&](auto kernel, int bytes) {
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  };
+  set(conv_igemm_tcgen05_kernel<64, 3, false, false>, TcSmem<64, 3, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 6, false, false>, TcSmem<64, 6, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 2, true, false>, TcSmem<64, 2, true>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 5, true, false>, TcSmem<64, 5, true>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 6, false, true>, TcSmem<64, 6, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 3, false, false>, TcSmem<128, 3, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 6, false, false>, TcSmem<128, 6, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 2, true, false>, TcSmem<128, 2, true>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 5, true, false>, TcSmem<128, 5, true>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 6, false, true>, TcSmem<128, 6, false>::kBytes);
+  if (e != cudaSuccess) return EE_ERR_CUDA;
   return EE_OK;
 }
 
@@ -444,6 +556,24 @@ inline ee_status_t tc_plan_layer(TcContext& c, const ee_layer_desc_t& d, int in_
   L->in_h = in_h, L->in_w = in_w, L->out_h = out_h, L->out_w = out_w, L->max_batch = max_batch;
   L->bn = d.cout > 64 ? 128 : 64;
   L->im2col = !(d.kh == 1 && d.stride == 1 && d.pad == 0);
+  // Split-K for layers whose grid stays small even at the model's max_batch while their K loop is long (the deep
+  // stages of a small-batch model): a lone CTA cannot pull operands faster than its SM's L2 port, so the K range is
+  // spread over a cluster of 2, 4 or 8 CTAs.  The cut depends on the layer and on max_batch (both fixed at model
+  // creation), never on the batch actually run, so a sample's sums are grouped the same way in every call.
+  {
+    const int num_kb = d.kh * d.kw * cdiv(d.cin, kTcBK);
+    const long tiles = (long)cdiv((long)max_batch * out_h * out_w, kTcBM) * cdiv(d.cout, L->bn);
+    L->splits = 1;
+    L->kb_per = num_kb;
+    for (int sp = 8; sp >= 2; sp >>= 1) {
+      const int per = cdiv(num_kb, sp);
+      if (tiles * sp <= 148 && sp * 4 <= num_kb && (sp - 1) * per < num_kb) {
+        L->splits = sp;
+        L->kb_per = per;
+        break;
+      }
+    }
+  }
   // weights [Cout][taps][Cin] as a 3-D tensor, box = 64 channels x 1 tap x BN filters
   const cuuint64_t dims[3] = {(cuuint64_t)d.cin, (cuuint64_t)(d.kh * d.kw), (cuuint64_t)d.cout};
   const cuuint64_t strides[2] = {(cuuint64_t)d.cin * 2, (cuuint64_t)d.cin * d.kh * d.kw * 2};
@@ -509,20 +639,35 @@ inline ee_status_t tc_buffer_map(const TcContext& c, const TcLayer& L, const voi
   return EE_OK;
 }
 
-template <int BN, bool RES>
+template <int BN, int STAGES, bool RES, bool SPLIT>
 inline cudaError_t tc_launch_t(dim3 grid, cudaStream_t st, const CUtensorMap& a, const CUtensorMap& w, const CUtensorMap& r,
                                const CUtensorMap& o, const TcParams& p) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = dim3(kTcThreads);
-  cfg.dynamicSmemBytes = TcSmem<BN, RES>::kBytes;
+  cfg.dynamicSmemBytes = TcSmem<BN, STAGES, RES>::kBytes;
   cfg.stream = st;
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;  // prologue may overlap the previous kernel's tail
-  attr.val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = &attr;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // prologue may overlap the previous kernel's tail
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_kernel<BN, RES>, a, w, r, o, p);
+  if (SPLIT) {  // the K ranges of one tile form a cluster along z
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = grid.z;
+    cfg.numAttrs = 2;
+  }
+  return cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_kernel<BN, STAGES, RES, SPLIT>, a, w, r, o, p);
+}
+
+template <int BN>
+inline cudaError_t tc_launch_bn(bool deep, bool res, bool split, dim3 grid, cudaStream_t st, const CUtensorMap& a, const CUtensorMap& w,
+                                const CUtensorMap& r, const CUtensorMap& o, const TcParams& p) {
+  if (split) return tc_launch_t<BN, 6, false, true>(grid, st, a, w, r, o, p);  // small grids by construction: deep ring
+  if (res) return deep ? tc_launch_t<BN, 5, true, false>(grid, st, a, w, r, o, p) : tc_launch_t<BN, 2, true, false>(grid, st, a, w, r, o, p);
+  return deep ? tc_launch_t<BN, 6, false, false>(grid, st, a, w, r, o, p) : tc_launch_t<BN, 3, false, false>(grid, st, a, w, r, o, p);
 }
 
 inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, const void* res, void* dst, int B, const float* scale,
@@ -553,12 +698,14 @@ inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, co
   p.residual = (const bf16*)res;
   p.out = (bf16*)dst;
   p.err_flag = err_flag;
-  dim3 grid(cdiv(p.M, kTcBM), cdiv(L.cout, L.bn));
-  cudaError_t e;
-  if (L.bn == 128)
-    e = res ? tc_launch_t<128, true>(grid, st, tmA, L.tm_w, tmR, tmO, p) : tc_launch_t<128, false>(grid, st, tmA, L.tm_w, tmR, tmO, p);
-  else
-    e = res ? tc_launch_t<64, true>(grid, st, tmA, L.tm_w, tmR, tmO, p) : tc_launch_t<64, false>(grid, st, tmA, L.tm_w, tmR, tmO, p);
+  const bool split = L.splits > 1;
+  p.kb_per = L.kb_per;
+  dim3 grid(cdiv(p.M, kTcBM), cdiv(L.cout, L.bn), split ? L.splits : 1);
+  // at most one CTA per SM anyway: take the deep operand ring
+  const bool deep = (long)grid.x * grid.y * grid.z <= 148;
+  const bool tma_res = res && !split;
+  cudaError_t e = L.bn == 128 ? tc_launch_bn<128>(deep, tma_res, split, grid, st, tmA, L.tm_w, tmR, tmO, p)
+                              : tc_launch_bn<64>(deep, tma_res, split, grid, st, tmA, L.tm_w, tmR, tmO, p);
   return e == cudaSuccess ? EE_OK : EE_ERR_CUDA;
 }
 
