@@ -168,7 +168,7 @@ ee_status_t ee_batch_refill(ee_model_t* model, int boundary, void* batch_feat, i
 /* One layer of a stage alone (the same kernel and launch configuration ee_stage_run uses for it): `input` is
  * the layer's input tensor [batch][in_h][in_w][cin], `residual` its residual operand [batch][out_h][out_w][cout]
  * (required iff the layer has one), `output` [batch][out_h][out_w][cout]; all DEVICE, model dtype, 16-byte aligned,
- * caller-owned.  `workspace` as for ee_stage_run (only a packed stem uses it).  For per-layer parity checks and
+ * caller-owned.  `workspace` is reserved (no layer kernel needs scratch today; pass the stage workspace or NULL).  For per-layer parity checks and
  * micro-benchmarks.  Errors: INVALID_ARG, STAGE (stage or layer out of range), CAPACITY, CUDA. */
 ee_status_t ee_layer_run(ee_model_t* model, int stage, int layer, const void* input, const void* residual, int batch,
                          void* output, void* workspace, size_t workspace_bytes, void* cuda_stream);

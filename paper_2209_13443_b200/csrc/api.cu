@@ -26,8 +26,8 @@ thread_local std::string g_cuda_err;
     }                                                                                      \
   } while (0)
 
-enum KernelKind { KK_SIMT = 0, KK_TC = 1, KK_DW = 2, KK_POOL = 3, KK_TC_PACKED = 4 };
-const char* kKernelNames[] = {"conv_igemm_simt", "conv_igemm_tcgen05", "dwconv", "maxpool", "conv_igemm_tcgen05_packed"};
+enum KernelKind { KK_SIMT = 0, KK_TC = 1, KK_DW = 2, KK_POOL = 3, KK_TC_GATHER = 4 };
+const char* kKernelNames[] = {"conv_igemm_simt", "conv_igemm_tcgen05", "dwconv", "maxpool", "conv_igemm_tcgen05_gather"};
 
 struct LayerPlan {
   ee_layer_desc_t d;
@@ -39,16 +39,14 @@ struct LayerPlan {
   void* w_dev = nullptr;
   float* scale_dev = nullptr;
   float* bias_dev = nullptr;
-  TcLayer tc;  // tensor-core plan (valid iff kind == KK_TC or KK_TC_PACKED)
-  int kp = 0, runp = 0;  // KK_TC_PACKED: columns of the packed Toeplitz matrix and of one filter-row run
-  int pack_chunk = 0;    // KK_TC_PACKED: samples packed per launch, so that the packed chunk stays in L2
+  TcLayer tc;  // tensor-core plan (valid iff kind == KK_TC or KK_TC_GATHER)
 };
 
 struct StagePlan {
   std::vector<LayerPlan> layers;
   int in_h, in_w, in_c, out_h, out_w, out_c, out_slot;
   std::vector<size_t> slot_off;  // byte offsets at max_batch
-  size_t head_off = 0, ws_bytes = 0, head_bytes = 0, pack_off = 0;
+  size_t head_off = 0, ws_bytes = 0, head_bytes = 0;
   int n_classes = 0;
   void* fc_w = nullptr;
   float* fc_b = nullptr;
@@ -136,8 +134,7 @@ void record(ee_model* m, StagePlan& sp, cudaStream_t st, const char* name) {
 }
 
 template <typename T>
-ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const void* res, void* dst, void* pack, int B,
-                         cudaStream_t st) {
+ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const void* res, void* dst, int B, cudaStream_t st) {
   ConvGeom g{B, L.in_h, L.in_w, L.d.cin, L.out_h, L.out_w, L.d.cout, L.d.kh, L.d.kw, L.d.stride, L.d.pad, L.d.act};
   constexpr int V = Elem<T>::kVec;
   switch (L.kind) {
@@ -152,26 +149,10 @@ ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const
       if (s != EE_OK) return s;
       break;
     }
-    case KK_TC_PACKED: {
+    case KK_TC_GATHER: {
       if constexpr (sizeof(T) == 2) {
-        // chunk by chunk: pack a few samples' Toeplitz rows (they stay in L2), multiply, next chunk
-        const size_t in_ps = (size_t)L.in_h * L.in_w * L.d.cin, out_ps = (size_t)L.out_h * L.out_w * L.d.cout;
-        for (int b0 = 0; b0 < B; b0 += L.pack_chunk) {
-          const int nb = std::min(L.pack_chunk, B - b0);
-          const long runs = (long)nb * L.out_h * L.out_w * L.d.kh;
-          const int grid = (int)std::min<long>(cdiv(runs, 256), 148L * 64);
-          const bf16* xs = (const bf16*)src + in_ps * b0;
-          if (L.d.cin == 3)
-            im2col_pack_kernel<3><<<grid, 256, 0, st>>>(xs, (bf16*)pack, nb, L.in_h, L.in_w, 3, L.out_h, L.out_w, L.d.kh, L.d.kw,
-                                                         L.d.stride, L.d.pad, L.runp, L.kp);
-          else
-            im2col_pack_kernel<0><<<grid, 256, 0, st>>>(xs, (bf16*)pack, nb, L.in_h, L.in_w, L.d.cin, L.out_h, L.out_w, L.d.kh,
-                                                         L.d.kw, L.d.stride, L.d.pad, L.runp, L.kp);
-          EE_CUDA(cudaGetLastError());
-          const bf16* rs = res ? (const bf16*)res + out_ps * b0 : nullptr;
-          ee_status_t s = tc_launch(m->tc, L.tc, pack, rs, (bf16*)dst + out_ps * b0, nb, L.scale_dev, L.bias_dev, m->err_flag, st);
-          if (s != EE_OK) return s;
-        }
+        ee_status_t s = tc_launch(m->tc, L.tc, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st);
+        if (s != EE_OK) return s;
       } else {
         return EE_ERR_INTERNAL;
       }
@@ -441,7 +422,6 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
     sp.threshold = sd.threshold;
     sp.always_exit = sd.always_exit;
     // uploads and kernel choice
-    size_t pack_bytes = 0;
     for (int i = 0; i < sd.n_layers; ++i) {
       LayerPlan& L = sp.layers[i];
       const ee_layer_desc_t& d = L.d;
@@ -460,31 +440,28 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
         L.kind = KK_TC;
         rc = tc_plan_layer(m->tc, d, L.in_h, L.in_w, L.out_h, L.out_w, desc->max_batch, L.w_dev, &L.tc);
         if (rc != EE_OK) return fail(rc);
-      } else if (desc->dtype == EE_BF16 && d.cout % 8 == 0 && d.kh * d.kw * d.cin <= 512 && d.kw * d.cin <= 64) {
+      } else if (desc->dtype == EE_BF16 && d.cout % 8 == 0 && d.kh * d.kw * d.cin <= 1024) {
         // pixel rows are not 16-byte units (e.g. a 3-channel stem): explicit Toeplitz rows, then the tensor-core GEMM
-        L.kind = KK_TC_PACKED;
+        L.kind = KK_TC_GATHER;
         const int run = d.kw * d.cin;
-        L.runp = cdiv(run, 8) * 8;
-        L.kp = cdiv(d.kh * L.runp, kTcBK) * kTcBK;
-        const size_t per_sample = (size_t)L.out_h * L.out_w * L.kp * 2;
-        L.pack_chunk = (int)std::max<size_t>(1, std::min<size_t>((size_t)desc->max_batch, ((size_t)32 << 20) / per_sample));
+        const int runp = cdiv(run, 8) * 8;
+        const int kp = cdiv(d.kh * runp, kTcBK) * kTcBK;
         void* wp = nullptr;
-        if (cudaMalloc(&wp, (size_t)d.cout * L.kp * 2) != cudaSuccess) return fail(EE_ERR_CUDA);
+        if (cudaMalloc(&wp, (size_t)d.cout * kp * 2) != cudaSuccess) return fail(EE_ERR_CUDA);
         m->owned.push_back(wp);
-        pack_weights_kernel<<<cdiv((long)d.cout * L.kp, 256), 256, 0, st>>>((const bf16*)L.w_dev, (bf16*)wp, d.cout, d.kh, run, L.runp, L.kp);
+        pack_weights_kernel<<<cdiv((long)d.cout * kp, 256), 256, 0, st>>>((const bf16*)L.w_dev, (bf16*)wp, d.cout, d.kh, run, runp, kp);
         if (cudaGetLastError() != cudaSuccess) return fail(EE_ERR_CUDA);
-        ee_layer_desc_t g = d;
-        g.cin = L.kp, g.kh = g.kw = 1, g.stride = 1, g.pad = 0;
-        rc = tc_plan_layer(m->tc, g, L.out_h, L.out_w, L.out_h, L.out_w, L.pack_chunk, wp, &L.tc);
+        ee_layer_desc_t g = d;   // the GEMM view: a 1x1 layer over kp packed columns
+        g.cin = kp, g.kh = g.kw = 1, g.stride = 1, g.pad = 0;
+        rc = tc_plan_layer(m->tc, g, L.out_h, L.out_w, L.out_h, L.out_w, desc->max_batch, wp, &L.tc);
         if (rc != EE_OK) return fail(rc);
-        pack_bytes = std::max(pack_bytes, per_sample * L.pack_chunk);
+        L.tc.gather = true;
+        L.tc.splits = 1, L.tc.kb_per = kp / kTcBK;
+        L.tc.g_h = L.in_h, L.tc.g_w = L.in_w, L.tc.g_cin = d.cin, L.tc.g_kh = d.kh, L.tc.g_kw = d.kw;
+        L.tc.g_stride = d.stride, L.tc.g_pad = d.pad, L.tc.g_runp = runp;
       } else {
         L.kind = KK_SIMT;
       }
-    }
-    if (pack_bytes) {  // the packed matrix lives behind the head scratch
-      sp.pack_off = align_up(sp.ws_bytes, 1024);
-      sp.ws_bytes = sp.pack_off + pack_bytes;
     }
     if ((rc = upload_bytes(m, sd.fc_weight, (size_t)sd.n_classes * sp.out_c * es, ondev, st, &sp.fc_w)) != EE_OK) return fail(rc);
     if ((rc = upload<float>(m, sd.fc_bias, sd.n_classes, ondev, st, &sp.fc_b)) != EE_OK) return fail(rc);
@@ -534,9 +511,8 @@ ee_status_t ee_stage_run(ee_model_t* m, int stage, const ee_stage_in_t* in, void
     const void* src = L.src_slot < 0 ? in->features : ws + sp.slot_off[L.src_slot];
     const void* res = L.res_slot == -2 ? nullptr : (L.res_slot == -1 ? in->features : ws + sp.slot_off[L.res_slot]);
     void* dst = ws + sp.slot_off[L.out_slot];
-    void* pack = ws + sp.pack_off;
-    ee_status_t s = m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, src, res, dst, pack, B, st)
-                                        : launch_layer<float>(m, L, src, res, dst, pack, B, st);
+    ee_status_t s = m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, src, res, dst, B, st)
+                                        : launch_layer<float>(m, L, src, res, dst, B, st);
     if (s != EE_OK) return s;
     record(m, sp, st, kKernelNames[L.kind]);
   }
@@ -567,15 +543,11 @@ ee_status_t ee_layer_run(ee_model_t* m, int stage, int layer, const void* input,
   const bool has_res = L.res_slot != -2;
   if (!input || !output || (has_res && !residual) || ((uintptr_t)input & 15) || ((uintptr_t)output & 15) || ((uintptr_t)residual & 15))
     return EE_ERR_INVALID_ARG;
-  void* pack = nullptr;
-  if (L.kind == KK_TC_PACKED) {
-    if (!workspace || ((uintptr_t)workspace & 255)) return EE_ERR_INVALID_ARG;
-    if (workspace_bytes < sp.ws_bytes) return EE_ERR_CAPACITY;
-    pack = (char*)workspace + sp.pack_off;
-  }
+  (void)workspace;
+  (void)workspace_bytes;
   cudaStream_t st = (cudaStream_t)cuda_stream;
-  return m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, input, has_res ? residual : nullptr, output, pack, batch, st)
-                             : launch_layer<float>(m, L, input, has_res ? residual : nullptr, output, pack, batch, st);
+  return m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, input, has_res ? residual : nullptr, output, batch, st)
+                             : launch_layer<float>(m, L, input, has_res ? residual : nullptr, output, batch, st);
 }
 
 ee_status_t ee_batch_refill(ee_model_t* m, int boundary, void* batch_feat, int32_t* batch_ids, int n_surv, const void* arr_feat,
@@ -725,7 +697,7 @@ ee_status_t ee_model_plan(const ee_model_t* m, int stage, int batch, int cap, ee
     const double in_b = (double)batch * L.in_h * L.in_w * L.d.cin * es, out_b = (double)p.m * p.n * es;
     const double w_b = L.d.op == EE_OP_MAXPOOL ? 0.0 : (double)L.d.cout * p.k * es;
     p.bytes = in_b + out_b + w_b + (L.res_slot != -2 ? out_b : 0.0);
-    p.launches = L.kind == KK_TC_PACKED ? 2 * cdiv(batch, L.pack_chunk) : 1;
+    p.launches = 1;
   }
   return EE_OK;
 }

@@ -44,6 +44,9 @@ struct TcParams {
   bf16* out;
   int* err_flag;
   int kb_per;           // split-K: K blocks per range (a property of the layer)
+  // gather mode (layers whose pixel rows are not 16-byte units, e.g. a 3-channel stem): the epilogue warps build the A tile
+  const bf16* gx;       // input feature map [B][gH][gW][gCin]
+  int gH, gW, gCin, gkh, grun, grunp;  // run = kw*Cin contiguous taps of one filter row, zero-padded to runp columns
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -143,6 +146,81 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 
 // ----------------------------------------------------------------------------- kernel
 
+// Gather-mode row builders (see the GATHER note on the kernel).  Thread `grow` writes row `grow` of the A tile of
+// every K block: 64 bf16 = eight 16-byte chunks, chunk c stored at position c ^ (row & 7) of the 128-byte line, which
+// is where the 128-byte swizzle of the MMA descriptor looks for it.  full barrier of slot s sits at bar0 + 8 s, the
+// empty barrier at bar0 + 8 (STAGES + s).
+template <int STAGES>
+__device__ __forceinline__ void gather_rows_generic(const TcParams& p, const bf16* xb, bool row_in, int hi0, int off0, int row_elems,
+                                                    uint8_t* gen, int stage_bytes, int grow, uint32_t bar0, int num_kb) {
+  const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
+  for (int i = 0; i < num_kb; ++i) {
+    const int s = i % STAGES;
+    const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+    if (!mbar_wait(bar0 + 8u * (STAGES + s), ph ^ 1u, p.err_flag)) break;
+    uint8_t* line = gen + (size_t)s * stage_bytes + grow * 128;
+    int rf = (i * kTcBK) / p.grunp, j = i * kTcBK - rf * p.grunp;   // filter row and column within its run
+#pragma unroll 1
+    for (int c = 0; c < 8; ++c) {
+      __align__(16) bf16 v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int hi = hi0 + rf, off = off0 + j;
+        const bool in = row_in && rf < p.gkh && j < p.grun && hi >= 0 && hi < p.gH && off >= 0 && off < row_elems;
+        v[e] = in ? xb[(size_t)hi * row_elems + off] : zero;
+        if (++j == p.grunp) {
+          j = 0;
+          ++rf;
+        }
+      }
+      *reinterpret_cast<uint4*>(line + ((c ^ (grow & 7)) << 4)) = *reinterpret_cast<const uint4*>(v);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar0 + 8u * s) : "memory");
+  }
+}
+
+// Same with the run geometry known at compile time: every (filter row, column) of every chunk is a constant, a pixel
+// whose taps all lie inside the image row takes the check-free path, and loads carry immediate offsets.
+template <int RUN, int RUNP, int KH, int NUMKB, int STAGES>
+__device__ __forceinline__ void gather_rows_static(const TcParams& p, const bf16* xb, bool row_in, int hi0, int off0, int row_elems,
+                                                   uint8_t* gen, int stage_bytes, int grow, uint32_t bar0) {
+  const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
+  const bool interior = off0 >= 0 && off0 + RUN <= row_elems;
+  unsigned rows_ok = 0;  // bit r: filter row r lies inside the image
+#pragma unroll
+  for (int r = 0; r < KH; ++r)
+    if (row_in && hi0 + r >= 0 && hi0 + r < p.gH) rows_ok |= 1u << r;
+  const bf16* x0 = xb + (long)hi0 * row_elems + off0;  // tap (0, 0); only dereferenced where in range
+#pragma unroll
+  for (int i = 0; i < NUMKB; ++i) {
+    const int s = i % STAGES;
+    const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+    if (!mbar_wait(bar0 + 8u * (STAGES + s), ph ^ 1u, p.err_flag)) break;
+    uint8_t* line = gen + (size_t)s * stage_bytes + grow * 128;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      __align__(16) bf16 v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        constexpr int dummy = 0;
+        (void)dummy;
+        const int k = i * kTcBK + c * 8 + e;
+        const int rf = k / RUNP, j = k % RUNP;     // compile-time after unrolling
+        if (rf < KH && j < RUN) {
+          const bool in = ((rows_ok >> rf) & 1u) && (interior || (off0 + j >= 0 && off0 + j < row_elems));
+          v[e] = in ? x0[(long)rf * row_elems + j] : zero;
+        } else {
+          v[e] = zero;
+        }
+      }
+      *reinterpret_cast<uint4*>(line + ((c ^ (grow & 7)) << 4)) = *reinterpret_cast<const uint4*>(v);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar0 + 8u * s) : "memory");
+  }
+}
+
 // Shared-memory plan of one CTA: a ring of STAGES operand slots (A 16 KB + W BN*128 B each), then, for layers whose
 // residual operand is prefetched (RES), a dedicated 128 x BN bf16 tile that the producer fills with the residual at
 // kernel start and the epilogue overwrites in place with the output.  Without it the output is staged in ring slot
@@ -177,11 +255,18 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src
 // its fp32 partial tile in its own shared memory, then every CTA reduces one slice of rows by reading all partials
 // through distributed shared memory in ascending range order (a reduce-scatter), applies the epilogue to that
 // slice and stores it.
-template <int BN, int STAGES, bool RES, bool SPLIT>
+//
+// GATHER: operand A comes from CUDA cores instead of TMA, for layers whose pixel rows are not whole 16-byte units
+// (a 3-channel stem).  K is laid out as kh runs of runp columns: run r holds the kw*Cin taps of filter row r, which
+// are contiguous in the NHWC input, then zeros; the weights are packed the same way.  While the main loop runs, the
+// four epilogue warps (one thread per tile row) read their pixel's taps and write them into the ring slot at the
+// position the 128-byte swizzle expects; the Toeplitz matrix still never touches global memory.
+template <int BN, int STAGES, bool RES, bool SPLIT, bool GATHER>
 __global__ void __launch_bounds__(kTcThreads, 2)
 conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                           const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmO, TcParams p) {
   static_assert(!(RES && SPLIT), "split-K tiles read their residual with plain loads");
+  static_assert(!GATHER || (!RES && !SPLIT), "gather mode is for plain stem layers");
   extern __shared__ uint8_t smem_raw[];
   using S = TcSmem<BN, STAGES, RES>;
   constexpr int kStages = S::kStages;
@@ -207,7 +292,7 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(full_bar(s), 1);
+      mbar_init(full_bar(s), GATHER ? 129 : 1);  // gather: 128 row writers + the weight tile's expect_tx
       mbar_init(empty_bar(s), 1);
     }
     mbar_init(accum_bar, 1);
@@ -260,8 +345,9 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
         if (!mbar_wait(empty_bar(s), ph ^ 1u, p.err_flag)) break;
         const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
         const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
-        mbar_expect_tx(full_bar(s), S::kStage);
-        if (p.im2col) {
+        mbar_expect_tx(full_bar(s), GATHER ? S::kBBytes : S::kStage);
+        if (GATHER) {
+        } else if (p.im2col) {
           const int r = tap / p.kw;
           tma_load_im2col_4d(sa, &tmA, full_bar(s), cb * kTcBK, cw, ch, cn, (uint16_t)(tap - r * p.kw), (uint16_t)r);
         } else {
@@ -296,6 +382,23 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
       s_bias[i] = (p.bias && in) ? p.bias[n0 + i] : 0.f;
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (GATHER) {
+      const int grow = (warp & 3) * 32 + lane;  // tile row = output pixel built by this thread
+      const int m = m0 + grow;
+      const bool row_in = m < p.M;
+      const int hw = p.Ho * p.Wo;
+      const int b = m / hw, rem = m - b * hw, ho = rem / p.Wo, wo = rem - ho * p.Wo;
+      const int hi0 = ho * p.stride - p.pad;
+      const int off0 = (wo * p.stride - p.pad) * p.gCin;  // flat element offset of tap 0 within an input row (may be negative)
+      const int row_elems = p.gW * p.gCin;
+      const bf16* xb = p.gx + (size_t)(row_in ? b : 0) * p.gH * row_elems;
+      if (p.grun == 21 && p.grunp == 24 && p.gkh == 7 && num_kb == 3)        // 7x7 stem on 3 channels
+        gather_rows_static<21, 24, 7, 3, STAGES>(p, xb, row_in, hi0, off0, row_elems, gen, S::kStage, grow, bar0);
+      else if (p.grun == 9 && p.grunp == 16 && p.gkh == 3 && num_kb == 1)    // 3x3 stem on 3 channels
+        gather_rows_static<9, 16, 3, 1, STAGES>(p, xb, row_in, hi0, off0, row_elems, gen, S::kStage, grow, bar0);
+      else
+        gather_rows_generic<STAGES>(p, xb, row_in, hi0, off0, row_elems, gen, S::kStage, grow, bar0, num_kb);
+    }
     // warp-uniform outcomes: tcgen05.ld is a warp-wide instruction
     bool ok = num_kb > 0 ? __all_sync(0xffffffffu, mbar_wait(accum_bar, 0, p.err_flag)) : true;
     if (RES) ok = __all_sync(0xffffffffu, mbar_wait(res_bar, 0, p.err_flag)) && ok;
@@ -431,48 +534,7 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
   }
 }
 
-// Explicit Toeplitz rows for layers whose pixel rows are not 16-byte units (a 3-channel stem).  Row m of `out`
-// holds, for every filter row r, the kw*Cin taps of output pixel m (contiguous in the NHWC input), zero for
-// padding taps, each run zero-padded to `runp` columns; the row is zero-padded to Kp columns.  One thread writes
-// one run.  The packed matrix then feeds the tensor-core kernel as a 1x1 layer with Kp input channels; the
-// weights are laid out to match by pack_weights_kernel.
-template <int CIN>
-__global__ void __launch_bounds__(256)
-im2col_pack_kernel(const bf16* __restrict__ x, bf16* __restrict__ out, int B, int H, int W, int cin_rt, int Ho, int Wo, int kh, int kw,
-                   int stride, int pad, int runp, int Kp) {
-  const int Cin = CIN > 0 ? CIN : cin_rt;
-  const long total = (long)B * Ho * Wo * kh;
-  const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
-  for (long idx = (long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long)gridDim.x * blockDim.x) {
-    const int r = (int)(idx % kh);
-    const long m = idx / kh;
-    const int wo = (int)(m % Wo);
-    const long q = m / Wo;
-    const int ho = (int)(q % Ho);
-    const long b = q / Ho;
-    const int hi = ho * stride - pad + r;
-    const bool row_in = hi >= 0 && hi < H;
-    const int wi0 = wo * stride - pad;
-    const bf16* xr = x + ((b * H + (row_in ? hi : 0)) * W) * (long)Cin;
-    bf16* orow = out + (size_t)m * Kp + (size_t)r * runp;
-    int j = 0;
-    for (int g = 0; g < runp; g += 8) {
-      __align__(16) bf16 v[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e, ++j) {
-        const int sx = j / Cin, ci = j - sx * Cin;   // CIN is a compile-time constant on the hot instantiation
-        const int wi = wi0 + sx;
-        v[e] = (row_in && sx < kw && wi >= 0 && wi < W) ? xr[(long)wi * Cin + ci] : zero;
-      }
-      *reinterpret_cast<uint4*>(orow + g) = *reinterpret_cast<const uint4*>(v);
-    }
-    if (r == 0) {  // zero tail of the row: the matching weight columns are zero, but 0 * NaN is NaN
-      for (int k = kh * runp; k < Kp; k += 8) *reinterpret_cast<uint4*>(out + (size_t)m * Kp + k) = make_uint4(0, 0, 0, 0);
-    }
-  }
-}
-
-// Weight rows [Cout][kh][kw*Cin] copied into rows [Cout][kh][runp] padded to Kp columns, zeros elsewhere.
+// Gather mode: weight rows [Cout][kh][kw*Cin] copied into rows [Cout][kh][runp] padded to Kp columns, zeros elsewhere.
 __global__ void pack_weights_kernel(const bf16* __restrict__ w, bf16* __restrict__ out, int rows, int kh, int run, int runp, int Kp) {
   const long total = (long)rows * Kp;
   for (long idx = (long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long)gridDim.x * blockDim.x) {
@@ -503,6 +565,9 @@ struct TcLayer {
   int bn = 128;
   bool im2col = false;
   int splits = 1, kb_per = 0;    // split-K ranges of this layer (fixed per layer, independent of the batch)
+  // gather mode: geometry of the real convolution (cin/kh/... above then describe the packed 1x1 GEMM view)
+  bool gather = false;
+  int g_h = 0, g_w = 0, g_cin = 0, g_kh = 0, g_kw = 0, g_stride = 1, g_pad = 0, g_runp = 0;
   CUtensorMap tm_w;
   struct Cached {
     const void* ptr;
@@ -526,16 +591,18 @@ inline ee_status_t tc_context_init(TcContext& c) {
   auto set = [&](auto kernel, int bytes) {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   };
-  set(conv_igemm_tcgen05_kernel<64, 3, false, false>, TcSmem<64, 3, false>::kBytes);
-  set(conv_igemm_tcgen05_kernel<64, 6, false, false>, TcSmem<64, 6, false>::kBytes);
-  set(conv_igemm_tcgen05_kernel<64, 2, true, false>, TcSmem<64, 2, true>::kBytes);
-  set(conv_igemm_tcgen05_kernel<64, 5, true, false>, TcSmem<64, 5, true>::kBytes);
-  set(conv_igemm_tcgen05_kernel<64, 6, false, true>, TcSmem<64, 6, false>::kBytes);
-  set(conv_igemm_tcgen05_kernel<128, 3, false, false>, TcSmem<128, 3, false>::kBytes);
-  set(conv_igemm_tcgen05_kernel<128, 6, false, false>, TcSmem<128, 6, false>::kBytes);
-  set(conv_igemm_tcgen05_kernel<128, 2, true, false>, TcSmem<128, 2, true>::kBytes);
-  set(conv_igemm_tcgen05_kernel<128, 5, true, false>, TcSmem<128, 5, true>::kBytes);
-  set(conv_igemm_tcgen05_kernel<128, 6, false, true>, TcSmem<128, 6, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 3, false, false, true>, TcSmem<64, 3, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 3, false, false, true>, TcSmem<128, 3, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 3, false, false, false>, TcSmem<64, 3, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 6, false, false, false>, TcSmem<64, 6, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 2, true, false, false>, TcSmem<64, 2, true>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 5, true, false, false>, TcSmem<64, 5, true>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 6, false, true, false>, TcSmem<64, 6, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 3, false, false, false>, TcSmem<128, 3, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 6, false, false, false>, TcSmem<128, 6, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 2, true, false, false>, TcSmem<128, 2, true>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 5, true, false, false>, TcSmem<128, 5, true>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 6, false, true, false>, TcSmem<128, 6, false>::kBytes);
   if (e != cudaSuccess) return EE_ERR_CUDA;
   return EE_OK;
 }
@@ -639,7 +706,7 @@ inline ee_status_t tc_buffer_map(const TcContext& c, const TcLayer& L, const voi
   return EE_OK;
 }
 
-template <int BN, int STAGES, bool RES, bool SPLIT>
+template <int BN, int STAGES, bool RES, bool SPLIT, bool GATHER = false>
 inline cudaError_t tc_launch_t(dim3 grid, cudaStream_t st, const CUtensorMap& a, const CUtensorMap& w, const CUtensorMap& r,
                                const CUtensorMap& o, const TcParams& p) {
   cudaLaunchConfig_t cfg = {};
@@ -659,7 +726,7 @@ inline cudaError_t tc_launch_t(dim3 grid, cudaStream_t st, const CUtensorMap& a,
     attr[1].val.clusterDim.z = grid.z;
     cfg.numAttrs = 2;
   }
-  return cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_kernel<BN, STAGES, RES, SPLIT>, a, w, r, o, p);
+  return cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_kernel<BN, STAGES, RES, SPLIT, GATHER>, a, w, r, o, p);
 }
 
 template <int BN>
@@ -675,11 +742,14 @@ inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, co
   if (((uintptr_t)src & 15) || ((uintptr_t)dst & 15) || ((uintptr_t)res & 15)) return EE_ERR_INVALID_ARG;
   // copies: a later lookup may grow the cache and move its entries
   const CUtensorMap* t = nullptr;
-  ee_status_t s = tc_buffer_map(c, L, src, B, 0, &t);
+  ee_status_t s = tc_buffer_map(c, L, dst, B, 1, &t);
   if (s != EE_OK) return s;
-  const CUtensorMap tmA = *t;
-  if ((s = tc_buffer_map(c, L, dst, B, 1, &t)) != EE_OK) return s;
   const CUtensorMap tmO = *t;
+  CUtensorMap tmA = tmO;  // unused in gather mode
+  if (!L.gather) {
+    if ((s = tc_buffer_map(c, L, src, B, 0, &t)) != EE_OK) return s;
+    tmA = *t;
+  }
   CUtensorMap tmR = tmO;
   if (res) {
     if ((s = tc_buffer_map(c, L, res, B, 1, &t)) != EE_OK) return s;
@@ -700,10 +770,19 @@ inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, co
   p.err_flag = err_flag;
   const bool split = L.splits > 1;
   p.kb_per = L.kb_per;
+  p.gx = (const bf16*)src;
+  p.gH = L.g_h, p.gW = L.g_w, p.gCin = L.g_cin, p.gkh = L.g_kh, p.grun = L.g_kw * L.g_cin, p.grunp = L.g_runp;
+  if (L.gather) p.stride = L.g_stride, p.pad = L.g_pad;
   dim3 grid(cdiv(p.M, kTcBM), cdiv(L.cout, L.bn), split ? L.splits : 1);
   // at most one CTA per SM anyway: take the deep operand ring
   const bool deep = (long)grid.x * grid.y * grid.z <= 148;
   const bool tma_res = res && !split;
+  if (L.gather) {
+    if (res || split) return EE_ERR_INTERNAL;
+    cudaError_t ge = L.bn == 128 ? tc_launch_t<128, 3, false, false, true>(grid, st, tmA, L.tm_w, tmR, tmO, p)
+                                 : tc_launch_t<64, 3, false, false, true>(grid, st, tmA, L.tm_w, tmR, tmO, p);
+    return ge == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+  }
   cudaError_t e = L.bn == 128 ? tc_launch_bn<128>(deep, tma_res, split, grid, st, tmA, L.tm_w, tmR, tmO, p)
                               : tc_launch_bn<64>(deep, tma_res, split, grid, st, tmA, L.tm_w, tmR, tmO, p);
   return e == cudaSuccess ? EE_OK : EE_ERR_CUDA;
