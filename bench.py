@@ -191,6 +191,9 @@ def run_ours(args):
     res_host = [dict(conf=torch.empty(B).pin_memory(), pred=torch.empty(B, dtype=torch.int32).pin_memory(),
                      mask=torch.empty(B, dtype=torch.uint8).pin_memory()) for _ in range(nst)]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # larger than the 126 MB L2
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()          # a capturable stream: stages replay as CUDA graphs after their first call
+    torch.cuda.set_stream(side)
     stream = torch.cuda.current_stream()
     sizes_last = []
     def stage_launches(s, n):

@@ -211,6 +211,14 @@ ee_status_t ee_exit_head_static(ee_model_t* model, int stage, const void* x, int
 ee_status_t ee_gather_survivors(const void* feat, size_t bytes_per_sample, const int32_t* survivor_idx,
                                 const int32_t* n_surv_dev, int max_rows, void* feat_out, void* cuda_stream);
 
+/* Stage replay.  On by default: the first ee_stage_run with a given signature (stage, every pointer of in/out, the
+ * workspace, the batch) on a capturable stream (not the legacy default stream, not a stream the caller is already
+ * capturing) records the stage's launches into a CUDA graph; later calls with the same signature replay it.  A server
+ * that keeps its buffers (Section III-B, Overhead: buffers are allocated once at initialisation) therefore pays the
+ * launch cost of a stage once per batch size.  Results are identical either way.  Disabled while per-layer timing is on.
+ * Errors: INVALID_ARG. */
+ee_status_t ee_model_set_graphs(ee_model_t* model, int enabled);
+
 /* Per-layer device timing.  When enabled, ee_stage_run brackets every kernel with CUDA events on the
  * stream it launches on.  ee_model_get_timing synchronises those events and writes, for the last run
  * of `stage`, up to `cap` entries: the layers in order, then the head and the gather kernels.

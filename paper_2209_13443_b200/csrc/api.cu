@@ -42,8 +42,26 @@ struct LayerPlan {
   TcLayer tc;  // tensor-core plan (valid iff kind == KK_TC or KK_TC_GATHER)
 };
 
+struct StageCallKey {  // everything that distinguishes one ee_stage_run call from another
+  ee_stage_in_t in;
+  ee_stage_out_t out;
+  void* ws;
+};
+struct StageGraph {
+  StageCallKey key;
+  cudaGraphExec_t exec;
+};
+inline bool same_call(const StageCallKey& a, const StageCallKey& b) {  // field by field: the structs have padding
+  return a.ws == b.ws && a.in.features == b.in.features && a.in.ids == b.in.ids && a.in.batch == b.in.batch &&
+         a.in.logit_shift == b.in.logit_shift && a.in.shift_class == b.in.shift_class &&
+         a.out.features_out == b.out.features_out && a.out.conf == b.out.conf && a.out.pred == b.out.pred &&
+         a.out.logits == b.out.logits && a.out.exit_mask == b.out.exit_mask && a.out.survivor_idx == b.out.survivor_idx &&
+         a.out.ids_out == b.out.ids_out && a.out.n_surv_dev == b.out.n_surv_dev && a.out.n_surv_host == b.out.n_surv_host;
+}
+
 struct StagePlan {
   std::vector<LayerPlan> layers;
+  std::vector<StageGraph> graphs;  // captured stage executions by call signature
   int in_h, in_w, in_c, out_h, out_w, out_c, out_slot;
   std::vector<size_t> slot_off;  // byte offsets at max_batch
   size_t head_off = 0, ws_bytes = 0, head_bytes = 0;
@@ -100,6 +118,7 @@ struct ee_model {
   std::vector<void*> owned;  // device allocations
   int* err_flag = nullptr;   // device word set by kernels whose bounded waits ran out
   bool timing = false;
+  bool graphs = true;  // replay stages as CUDA graphs on capturable streams
   TcContext tc;
 };
 
@@ -253,6 +272,36 @@ ee_status_t append_launch_t(const void* src, void* dst, size_t bytes, const int3
   return EE_OK;
 }
 
+// Everything one stage launches, in stream order (also the body of a captured graph).
+ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, char* ws, const ee_stage_out_t* out, cudaStream_t st) {
+  const int B = in->batch;
+  sp.ev_used = 0;
+  record(m, sp, st, "begin");
+  for (size_t i = 0; i < sp.layers.size(); ++i) {
+    const LayerPlan& L = sp.layers[i];
+    const void* src = L.src_slot < 0 ? in->features : ws + sp.slot_off[L.src_slot];
+    const void* res = L.res_slot == -2 ? nullptr : (L.res_slot == -1 ? in->features : ws + sp.slot_off[L.res_slot]);
+    void* dst = ws + sp.slot_off[L.out_slot];
+    ee_status_t s = m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, src, res, dst, B, st)
+                                        : launch_layer<float>(m, L, src, res, dst, B, st);
+    if (s != EE_OK) return s;
+    record(m, sp, st, kKernelNames[L.kind]);
+  }
+  const void* so = ws + sp.slot_off[sp.out_slot];
+  const int hw = sp.out_h * sp.out_w;
+  ee_status_t s = m->dtype == EE_BF16
+                      ? launch_head<bf16>(m, sp, so, B, hw, in->logit_shift, in->shift_class, ws + sp.head_off, in, out, st, true)
+                      : launch_head<float>(m, sp, so, B, hw, in->logit_shift, in->shift_class, ws + sp.head_off, in, out, st, true);
+  if (s != EE_OK) return s;
+  if (!sp.always_exit) {
+    s = gather_launch(so, (size_t)hw * sp.out_c * esize(m->dtype), out->survivor_idx, out->n_surv_dev, B, out->features_out, st);
+    if (s != EE_OK) return s;
+    record(m, sp, st, "gather_survivors");
+  }
+  if (out->n_surv_host) EE_CUDA(cudaMemcpyAsync(out->n_surv_host, out->n_surv_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  return EE_OK;
+}
+
 bool valid_out(const ee_stage_out_t* o, bool need_feat) {
   return o && o->exit_mask && o->survivor_idx && o->n_surv_dev && (!need_feat || o->features_out);
 }
@@ -280,8 +329,10 @@ const char* ee_last_cuda_error(void) { return g_cuda_err.c_str(); }
 
 ee_status_t ee_model_destroy(ee_model_t* m) {
   if (!m) return EE_ERR_INVALID_ARG;
-  for (auto& sp : m->stages)
+  for (auto& sp : m->stages) {
     for (auto e : sp.ev) cudaEventDestroy(e);
+    for (auto& g : sp.graphs) cudaGraphExecDestroy(g.exec);
+  }
   for (void* p : m->owned) cudaFree(p);
   delete m;
   return EE_OK;
@@ -503,32 +554,45 @@ ee_status_t ee_stage_run(ee_model_t* m, int stage, const ee_stage_in_t* in, void
   }
   if (!in->features || !workspace || ((uintptr_t)workspace & 255)) return EE_ERR_INVALID_ARG;
   if (workspace_bytes < sp.ws_bytes) return EE_ERR_CAPACITY;
-  char* ws = (char*)workspace;
-  sp.ev_used = 0;
-  record(m, sp, st, "begin");
-  for (size_t i = 0; i < sp.layers.size(); ++i) {
-    const LayerPlan& L = sp.layers[i];
-    const void* src = L.src_slot < 0 ? in->features : ws + sp.slot_off[L.src_slot];
-    const void* res = L.res_slot == -2 ? nullptr : (L.res_slot == -1 ? in->features : ws + sp.slot_off[L.res_slot]);
-    void* dst = ws + sp.slot_off[L.out_slot];
-    ee_status_t s = m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, src, res, dst, B, st)
-                                        : launch_layer<float>(m, L, src, res, dst, B, st);
-    if (s != EE_OK) return s;
-    record(m, sp, st, kKernelNames[L.kind]);
+  // Replay path: the whole stage (every layer, the head, the gather, the count copy) as one CUDA graph, captured the
+  // first time this exact call (same buffers, same batch) is seen on a capturable stream.  It removes the host cost
+  // of ~25 launches per stage and most of the launch latency between the small kernels of a small batch.
+  const bool legacy = st == nullptr || st == cudaStreamLegacy || st == cudaStreamPerThread;
+  if (m->graphs && !m->timing && !legacy) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) == cudaSuccess && cs == cudaStreamCaptureStatusNone) {
+      StageCallKey key;
+      key.in = *in;
+      key.out = *out;
+      key.ws = workspace;
+      for (auto& g : sp.graphs)
+        if (same_call(g.key, key)) {
+          EE_CUDA(cudaGraphLaunch(g.exec, st));
+          return EE_OK;
+        }
+      if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+        ee_status_t es = enqueue_stage(m, sp, in, (char*)workspace, out, st);
+        cudaGraph_t graph = nullptr;
+        cudaError_t ce = cudaStreamEndCapture(st, &graph);
+        cudaGraphExec_t exec = nullptr;
+        if (es == EE_OK && ce == cudaSuccess && graph && cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess) {
+          cudaGraphDestroy(graph);
+          if (sp.graphs.size() >= 96) {  // bounded cache: drop the oldest
+            cudaGraphExecDestroy(sp.graphs.front().exec);
+            sp.graphs.erase(sp.graphs.begin());
+          }
+          sp.graphs.push_back({key, exec});
+          EE_CUDA(cudaGraphLaunch(exec, st));
+          return EE_OK;
+        }
+        if (graph) cudaGraphDestroy(graph);
+        cudaGetLastError();   // capture is not available here: fall back to plain launches from now on
+        m->graphs = false;
+        if (es != EE_OK) return es;
+      }
+    }
   }
-  const void* so = ws + sp.slot_off[sp.out_slot];
-  const int hw = sp.out_h * sp.out_w;
-  ee_status_t s = m->dtype == EE_BF16
-                      ? launch_head<bf16>(m, sp, so, B, hw, in->logit_shift, in->shift_class, ws + sp.head_off, in, out, st, true)
-                      : launch_head<float>(m, sp, so, B, hw, in->logit_shift, in->shift_class, ws + sp.head_off, in, out, st, true);
-  if (s != EE_OK) return s;
-  if (!sp.always_exit) {
-    s = gather_launch(so, (size_t)hw * sp.out_c * esize(m->dtype), out->survivor_idx, out->n_surv_dev, B, out->features_out, st);
-    if (s != EE_OK) return s;
-    record(m, sp, st, "gather_survivors");
-  }
-  if (out->n_surv_host) EE_CUDA(cudaMemcpyAsync(out->n_surv_host, out->n_surv_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-  return EE_OK;
+  return enqueue_stage(m, sp, in, (char*)workspace, out, st);
 }
 
 ee_status_t ee_layer_run(ee_model_t* m, int stage, int layer, const void* input, const void* residual, int batch, void* output,
@@ -654,6 +718,12 @@ ee_status_t ee_gather_survivors(const void* feat, size_t bytes_per_sample, const
                                 int max_rows, void* feat_out, void* cuda_stream) {
   if (!feat || !survivor_idx || !n_surv_dev || !feat_out || max_rows < 0) return EE_ERR_INVALID_ARG;
   return gather_launch(feat, bytes_per_sample, survivor_idx, n_surv_dev, max_rows, feat_out, (cudaStream_t)cuda_stream);
+}
+
+ee_status_t ee_model_set_graphs(ee_model_t* m, int enabled) {
+  if (!m) return EE_ERR_INVALID_ARG;
+  m->graphs = enabled != 0;
+  return EE_OK;
 }
 
 ee_status_t ee_model_set_timing(ee_model_t* m, int enabled) {

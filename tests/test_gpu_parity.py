@@ -410,3 +410,40 @@ def test_streaming_trace_matches_oracle_schedule():
     assert got["pred"].tolist() == [serial[image_of[r]][1] for r in range(n)]
     np.testing.assert_allclose(got["finish"], fin, rtol=0, atol=1e-9)
     assert len({len(ids) for _, ids in launches}) > 3                          # the trace exercises varying batch sizes
+
+
+def test_stage_replay_as_graph_is_bit_identical():
+    """On a side stream a stage is captured into a CUDA graph at its first call and replayed afterwards; the replay,
+    and a replay on new input values in the same buffers, must equal plain launches bit for bit."""
+    spec = wl.resnet50_ee(seed=1, in_hw=64, n_classes=100, max_batch=6)
+    run = util.GpuRunner(spec)
+    m, out, ws = run.m, run.bufs[0], run.ws
+    B = 5
+    xa = eb.to_device("bf16", wl.make_input(spec, B, seed=1))
+    xb = eb.to_device("bf16", wl.make_input(spec, B, seed=2))
+    ids = torch.arange(B, dtype=torch.int32, device="cuda")
+
+    def snapshot():
+        torch.cuda.synchronize()
+        n = int(out.n_surv_host[0])
+        return (n, out.features_out[:n].clone(), out.logits[:B].clone(), out.exit_mask[:B].clone(), out.survivor_idx[:n].clone())
+
+    m.set_graphs(False)
+    m.stage_run(0, xa, B, out, ws, ids)
+    ref_a = snapshot()
+    buf = xa.clone()
+    m.set_graphs(True)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for expect_from in (xa, xa, xb):                     # capture, replay, replay on new values
+            buf.copy_(expect_from)
+            m.stage_run(0, buf, B, out, ws, ids)
+            got = snapshot()
+            if expect_from is xa:
+                assert got[0] == ref_a[0] and all(torch.equal(g, r) for g, r in zip(got[1:], ref_a[1:]))
+        got_b = got
+    m.set_graphs(False)
+    m.stage_run(0, xb, B, out, ws, ids)
+    ref_b = snapshot()
+    assert got_b[0] == ref_b[0] and all(torch.equal(g, r) for g, r in zip(got_b[1:], ref_b[1:]))
+    m.check()
