@@ -129,6 +129,28 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 }
 // 32 consecutive fp32 columns of this thread's TMEM lane.  Load and wait sit in one statement so that no
 // use of the registers can be scheduled before the wait.
+// Issue only; pair with tmem_ld_wait() before the registers are read.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+// The "+r" ties make every later use of the 64 registers depend on the wait.
+__device__ __forceinline__ void tmem_ld_wait(float* a, float* b) {
+  uint32_t* x = reinterpret_cast<uint32_t*>(a);
+  uint32_t* y = reinterpret_cast<uint32_t*>(b);
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) asm volatile("" : "+r"(x[i]), "+r"(y[i]));
+}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
   uint32_t* r = reinterpret_cast<uint32_t*>(v);
   asm volatile(
@@ -534,6 +556,252 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
   }
 }
 
+// ----------------------------------------------------------------------------- persistent variant
+//
+// For grids of several waves (large B*Ho*Wo): one CTA per SM walks output tiles t = blockIdx.x, + gridDim.x, ...
+// (tile t -> M tile t / n_tiles, N tile t % n_tiles, so CTAs running side by side share A rows in L2).  The operand
+// ring keeps streaming across tile boundaries and the accumulator is double-buffered in TMEM: while the epilogue warps
+// drain accumulator j & 1 of tile j, the MMA warp already fills the other one with tile j + 1, and the producer is
+// further ahead still.  A tile then costs max(load, MMA, epilogue) instead of their sum, and the per-CTA prologue
+// (barriers, TMEM allocation, descriptor fetch) is paid once per SM instead of once per tile.
+// Residual tiles and staged outputs alternate between two 128 x BN bf16 buffers; a buffer returns to the producer
+// (io_free) once all four epilogue warps have seen their TMA store finish reading it.
+template <int BN, bool RES>
+struct TcPersistSmem {
+  static constexpr int kStages = BN == 128 ? 4 : 7;
+  static constexpr int kABytes = kTcBM * kTcBK * 2;
+  static constexpr int kBBytes = BN * kTcBK * 2;
+  static constexpr int kStage = kABytes + kBBytes;
+  static constexpr int kTiles = kStages * kStage;
+  static constexpr int kIoBytes = kTcBM * BN * 2;
+  static constexpr int kAfter = kTiles + 2 * kIoBytes;
+  static constexpr int kBytes = kAfter + 4 * 2 * BN * 4 + 256 + 1024;  // + one scale/bias copy per epilogue warp, barriers, slack
+  static_assert(kBytes <= 227 * 1024, "exceeds the shared memory of an SM");
+};
+
+template <int BN, bool RES>
+__global__ void __launch_bounds__(kTcThreads, 1)
+conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+                                     const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmO, TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  using S = TcPersistSmem<BN, RES>;
+  constexpr int kStages = S::kStages;
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - raw);
+  float* s_sb = reinterpret_cast<float*>(gen + S::kAfter);  // [4 epilogue warps][scale BN | bias BN]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kAfter + 8 * BN * 4);
+  const uint32_t bar0 = base + S::kAfter + 8 * BN * 4;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+  auto acc_full = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
+  auto acc_empty = [&](int b) { return bar0 + 8u * (2 * kStages + 2 + b); };
+  auto res_full = [&](int b) { return bar0 + 8u * (2 * kStages + 4 + b); };
+  auto io_free = [&](int b) { return bar0 + 8u * (2 * kStages + 6 + b); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_kb = p.taps * p.cblocks;
+  const int n_tiles = (p.N + BN - 1) / BN;
+  const int m_tiles = (p.M + kTcBM - 1) / kTcBM;
+  const int total = n_tiles * m_tiles;
+  const int my_tiles = (int)blockIdx.x < total ? (total - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(acc_full(b), 1);
+      mbar_init(acc_empty(b), 4);   // lane 0 of each epilogue warp
+      mbar_init(res_full(b), 1);
+      mbar_init(io_free(b), 4);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0 && lane == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmO) : "memory");
+    if (RES) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmR) : "memory");
+  }
+  if (warp == 1) {  // two accumulators of BN fp32 columns
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(2 * BN) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int g = 0;  // K blocks issued so far, across tiles: the ring never drains at a tile boundary
+      bool ok = true;
+      for (int j = 0; j < my_tiles && ok; ++j) {
+        const int t = (int)blockIdx.x + j * (int)gridDim.x;
+        const int m0 = (t / n_tiles) * kTcBM, n0 = (t % n_tiles) * BN;
+        const int b = j & 1;
+        if (RES) {
+          if (j >= 2) ok = mbar_wait(io_free(b), (uint32_t)((j >> 1) - 1) & 1u, p.err_flag);
+          if (!ok) break;
+          mbar_expect_tx(res_full(b), S::kIoBytes);
+#pragma unroll
+          for (int h = 0; h < BN / 64; ++h)
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              tma_load_2d(base + S::kTiles + b * S::kIoBytes + h * 16384 + q * 4096, &tmR, res_full(b), n0 + h * 64, m0 + q * 32);
+        }
+        int cw = 0, ch = 0, cn = 0;
+        if (p.im2col) {
+          const int hw = p.Ho * p.Wo;
+          cn = m0 / hw;
+          const int rem = m0 - cn * hw;
+          const int ho = rem / p.Wo;
+          cw = (rem - ho * p.Wo) * p.stride - p.pad;
+          ch = ho * p.stride - p.pad;
+        }
+        for (int kb = 0; kb < num_kb; ++kb, ++g) {
+          const int s = g % kStages;
+          const uint32_t ph = (uint32_t)(g / kStages) & 1u;
+          ok = mbar_wait(empty_bar(s), ph ^ 1u, p.err_flag);
+          if (!ok) break;
+          const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
+          const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
+          mbar_expect_tx(full_bar(s), S::kStage);
+          if (p.im2col) {
+            const int r = tap / p.kw;
+            tma_load_im2col_4d(sa, &tmA, full_bar(s), cb * kTcBK, cw, ch, cn, (uint16_t)(tap - r * p.kw), (uint16_t)r);
+          } else {
+            tma_load_2d(sa, &tmA, full_bar(s), cb * kTcBK, m0);
+          }
+          tma_load_3d(sb, &tmW, full_bar(s), cb * kTcBK, tap, n0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc(BN);
+      int g = 0;
+      bool ok = true;
+      for (int j = 0; j < my_tiles && ok; ++j) {
+        const int b = j & 1;
+        if (j >= 2) {  // the epilogue must have drained this accumulator (tile j - 2)
+          ok = mbar_wait(acc_empty(b), (uint32_t)((j >> 1) - 1) & 1u, p.err_flag);
+          if (!ok) break;
+          tc_fence_after();
+        }
+        const uint32_t acc = tmem_base + (uint32_t)(b * BN);
+        for (int kb = 0; kb < num_kb; ++kb, ++g) {
+          const int s = g % kStages;
+          const uint32_t ph = (uint32_t)(g / kStages) & 1u;
+          ok = mbar_wait(full_bar(s), ph, p.err_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
+#pragma unroll
+          for (int k = 0; k < kTcBK / 16; ++k)
+            umma_bf16(acc, umma_desc(sa + k * 32), umma_desc(sb + k * 32), idesc, (uint32_t)((kb | k) != 0));
+          umma_commit(empty_bar(s));
+        }
+        if (ok) umma_commit(acc_full(b));
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    float* sc = s_sb + q * 2 * BN;  // this warp's own copy: no barrier across warps inside the tile loop
+    bool ok = true;
+    int sc_n0 = -1;
+    bool pending = false;  // lane 0: a bulk store group of this warp may still be reading shared memory
+    for (int j = 0; j < my_tiles; ++j) {
+      const int t = (int)blockIdx.x + j * (int)gridDim.x;
+      const int m0 = (t / n_tiles) * kTcBM, n0 = (t % n_tiles) * BN;
+      const int b = j & 1;
+      if (n0 != sc_n0) {  // consecutive tiles of a CTA usually share the N tile: reload only on change
+        __syncwarp();
+        for (int i = lane; i < BN; i += 32) {
+          const bool in = n0 + i < p.N;
+          sc[i] = (p.scale && in) ? p.scale[n0 + i] : 1.f;
+          sc[BN + i] = (p.bias && in) ? p.bias[n0 + i] : 0.f;
+        }
+        sc_n0 = n0;
+      }
+      __syncwarp();  // scale/bias of this tile visible to the warp
+      ok = __all_sync(0xffffffffu, mbar_wait(acc_full(b), (uint32_t)(j >> 1) & 1u, p.err_flag));
+      if (RES && ok) ok = __all_sync(0xffffffffu, mbar_wait(res_full(b), (uint32_t)(j >> 1) & 1u, p.err_flag));
+      if (!ok) break;
+      tc_fence_after();
+      uint8_t* io = gen + S::kTiles + b * S::kIoBytes;
+      const uint32_t io_s = base + S::kTiles + b * S::kIoBytes;
+      const uint32_t acc = tmem_base + (uint32_t)(b * BN) + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+      for (int h = 0; h < BN / 64; ++h) {
+        uint8_t* line = io + h * 16384 + row * 128;
+        float va[32], vb[32];  // both 32-column loads of the half in flight before one wait
+        tmem_ld32_issue(acc + (uint32_t)(h * 64), va);
+        tmem_ld32_issue(acc + (uint32_t)(h * 64 + 32), vb);
+        tmem_ld_wait(va, vb);
+        if (h == BN / 64 - 1) {  // the accumulator is in registers: the MMA warp may refill it
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acc_empty(b)) : "memory");
+        }
+#pragma unroll
+        for (int sub = 0; sub < 2; ++sub) {
+          const int c0 = h * 64 + sub * 32;
+          float* v = sub ? vb : va;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = fmaf(sc[c0 + i], v[i], sc[BN + c0 + i]);
+#pragma unroll
+          for (int gq = 0; gq < 4; ++gq) {
+            bf16* chunk = reinterpret_cast<bf16*>(line + (((sub * 4 + gq) ^ (lane & 7)) << 4));
+            if (RES) {
+              Vec16<bf16> r;
+              r.load(chunk);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) v[gq * 8 + e] += r.v[e];
+            }
+            Vec16<bf16> o;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) o.v[e] = apply_act(v[gq * 8 + e], p.act);
+            o.store(chunk);
+          }
+          if (h == 0 && sub == 0 && lane == 0 && pending) {
+            // One chunk into tile j, this warp's store of tile j - 1 has long finished reading its buffer: confirm it
+            // (no stall in the steady state) and hand the buffer back to the producer for the residual of tile j + 1.
+            // It also licenses the next iteration to overwrite that buffer.
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            pending = false;
+            if (RES) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(io_free((j - 1) & 1)) : "memory");
+          }
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) {
+        if (m0 + q * 32 < p.M) {
+#pragma unroll
+          for (int h = 0; h < BN / 64; ++h)
+            if (n0 + h * 64 < p.N) tma_store_2d(&tmO, io_s + h * 16384 + q * 4096, n0 + h * 64, m0 + q * 32);
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");  // possibly empty: keeps the bookkeeping uniform
+        pending = true;
+      }
+    }
+    if (lane == 0 && pending) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * BN) : "memory");
+  }
+}
+
 // Gather mode: weight rows [Cout][kh][kw*Cin] copied into rows [Cout][kh][runp] padded to Kp columns, zeros elsewhere.
 __global__ void pack_weights_kernel(const bf16* __restrict__ w, bf16* __restrict__ out, int rows, int kh, int run, int runp, int Kp) {
   const long total = (long)rows * Kp;
@@ -557,6 +825,7 @@ typedef CUresult (*PFN_encodeIm2col)(CUtensorMap*, CUtensorMapDataType, cuuint32
 struct TcContext {
   PFN_encodeTiled encode_tiled = nullptr;
   PFN_encodeIm2col encode_im2col = nullptr;
+  int sm_count = 148;
 };
 
 struct TcLayer {
@@ -587,6 +856,11 @@ inline ee_status_t tc_context_init(TcContext& c) {
   f = nullptr;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f, cudaEnableDefault, &q) != cudaSuccess || !f) return EE_ERR_CUDA;
   c.encode_im2col = (PFN_encodeIm2col)f;
+  {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+      c.sm_count = sms;
+  }
   cudaError_t e = cudaSuccess;
   auto set = [&](auto kernel, int bytes) {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
@@ -603,6 +877,10 @@ inline ee_status_t tc_context_init(TcContext& c) {
   set(conv_igemm_tcgen05_kernel<128, 2, true, false, false>, TcSmem<128, 2, true>::kBytes);
   set(conv_igemm_tcgen05_kernel<128, 5, true, false, false>, TcSmem<128, 5, true>::kBytes);
   set(conv_igemm_tcgen05_kernel<128, 6, false, true, false>, TcSmem<128, 6, false>::kBytes);
+  set(conv_igemm_tcgen05_persistent_kernel<64, false>, TcPersistSmem<64, false>::kBytes);
+  set(conv_igemm_tcgen05_persistent_kernel<64, true>, TcPersistSmem<64, true>::kBytes);
+  set(conv_igemm_tcgen05_persistent_kernel<128, false>, TcPersistSmem<128, false>::kBytes);
+  set(conv_igemm_tcgen05_persistent_kernel<128, true>, TcPersistSmem<128, true>::kBytes);
   if (e != cudaSuccess) return EE_ERR_CUDA;
   return EE_OK;
 }
@@ -737,6 +1015,22 @@ inline cudaError_t tc_launch_bn(bool deep, bool res, bool split, dim3 grid, cuda
   return deep ? tc_launch_t<BN, 6, false, false>(grid, st, a, w, r, o, p) : tc_launch_t<BN, 3, false, false>(grid, st, a, w, r, o, p);
 }
 
+template <int BN, bool RES>
+inline cudaError_t tc_launch_persistent(int ctas, cudaStream_t st, const CUtensorMap& a, const CUtensorMap& w, const CUtensorMap& r,
+                                        const CUtensorMap& o, const TcParams& p) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(ctas);
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = TcPersistSmem<BN, RES>::kBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_persistent_kernel<BN, RES>, a, w, r, o, p);
+}
+
 inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, const void* res, void* dst, int B, const float* scale,
                              const float* bias, int* err_flag, cudaStream_t st) {
   if (((uintptr_t)src & 15) || ((uintptr_t)dst & 15) || ((uintptr_t)res & 15)) return EE_ERR_INVALID_ARG;
@@ -782,6 +1076,16 @@ inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, co
     cudaError_t ge = L.bn == 128 ? tc_launch_t<128, 3, false, false, true>(grid, st, tmA, L.tm_w, tmR, tmO, p)
                                  : tc_launch_t<64, 3, false, false, true>(grid, st, tmA, L.tm_w, tmR, tmO, p);
     return ge == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+  }
+  const long tiles = (long)grid.x * grid.y;
+  if (!split && !res && L.kh * L.kw == 1 && tiles >= 2 * c.sm_count) {  // several waves of short K loops: one persistent CTA per SM walks the tiles
+    const int ctas = c.sm_count;
+    cudaError_t pe;
+    if (L.bn == 128)
+      pe = res ? tc_launch_persistent<128, true>(ctas, st, tmA, L.tm_w, tmR, tmO, p) : tc_launch_persistent<128, false>(ctas, st, tmA, L.tm_w, tmR, tmO, p);
+    else
+      pe = res ? tc_launch_persistent<64, true>(ctas, st, tmA, L.tm_w, tmR, tmO, p) : tc_launch_persistent<64, false>(ctas, st, tmA, L.tm_w, tmR, tmO, p);
+    return pe == cudaSuccess ? EE_OK : EE_ERR_CUDA;
   }
   cudaError_t e = L.bn == 128 ? tc_launch_bn<128>(deep, tma_res, split, grid, st, tmA, L.tm_w, tmR, tmO, p)
                               : tc_launch_bn<64>(deep, tma_res, split, grid, st, tmA, L.tm_w, tmR, tmO, p);
