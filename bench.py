@@ -198,8 +198,8 @@ def run_ours(args):
     sizes_last = []
     def stage_launches(s, n):
         """Kernels one ee_stage_run launches: the layers' (a packed stem packs and multiplies chunk by chunk),
-        three for the head, one gather."""
-        return sum(pl["launches"] for pl in model.plan(s, n)) + 3 + (0 if spec.stages[s].always_exit else 1)
+        two for the head (pooling; FC with the exit decision in its last CTA), one gather."""
+        return sum(pl["launches"] for pl in model.plan(s, n)) + 2 + (0 if spec.stages[s].always_exit else 1)
 
     def step(e2e: bool):
         """One pass of the whole path.  Returns (#kernel launches, h2d bytes, d2h bytes, per-stage batch)."""
@@ -288,7 +288,7 @@ def run_ours(args):
             ns = int(bufs[s].n_surv_host[0])
             es = 2 if spec.dtype == "bf16" else 4
             fam["head_gap"]["bytes"] += n * info["out_bytes_per_sample"]
-            fam["head_fc"]["bytes"] += info["out_c"] * spec.stages[s].n_classes * es + n * info["out_c"] * 4
+            fam["head_fc_softmax_scan"]["bytes"] += info["out_c"] * spec.stages[s].n_classes * es + n * info["out_c"] * 4
             if "gather_survivors" in fam and not spec.stages[s].always_exit:
                 fam["gather_survivors"]["bytes"] += 2 * ns * info["out_bytes_per_sample"]
             n = ns

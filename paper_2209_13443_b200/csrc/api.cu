@@ -99,7 +99,7 @@ HeadLayout head_layout(int max_batch, int hw, int c, int k, size_t es) {
   h.nchunks = cdiv(hw, h.rows_per_chunk);
   size_t o = 0;
   h.off_cnt = o;
-  o = align_up(o + sizeof(unsigned) * (size_t)max_batch, 256);
+  o = align_up(o + sizeof(unsigned) * ((size_t)max_batch + 1), 256);  // per-sample pooling counters + the FC kernel's
   h.off_partial = o;
   o = align_up(o + sizeof(float) * (size_t)max_batch * h.nchunks * c, 256);
   h.off_gap = o;
@@ -213,7 +213,7 @@ ee_status_t launch_head(ee_model* m, StagePlan& sp, const void* x, int B, int hw
   float* gap = (float*)(scratch + h.off_gap);
   float* z = out->logits ? out->logits : (float*)(scratch + h.off_z);
   constexpr int V = Elem<T>::kVec;
-  EE_CUDA(cudaMemsetAsync(cnt, 0, sizeof(unsigned) * (size_t)B, st));
+  EE_CUDA(cudaMemsetAsync(cnt, 0, sizeof(unsigned) * ((size_t)m->max_batch + 1), st));
   dim3 ggrid(h.nchunks, B);
   if (C % V == 0)
     gap_kernel<T, V><<<ggrid, kGapThreads, 0, st>>>((const T*)x, hw, C, h.rows_per_chunk, partial, gap, cnt);
@@ -221,17 +221,14 @@ ee_status_t launch_head(ee_model* m, StagePlan& sp, const void* x, int B, int hw
     gap_kernel<T, 1><<<ggrid, kGapThreads, 0, st>>>((const T*)x, hw, C, h.rows_per_chunk, partial, gap, cnt);
   EE_CUDA(cudaGetLastError());
   if (timed) record(m, sp, st, "head_gap");
+  DecideArgs da{shift, shift_cls, sp.threshold, sp.always_exit, out->conf, out->pred, out->exit_mask,
+                in_ids ? in_ids->ids : nullptr, out->survivor_idx, out->ids_out, out->n_surv_dev, cnt + m->max_batch};
   if (C % V == 0)
-    fc_kernel<T, V><<<cdiv(K, kFcClasses), kFcWarps * 32, 0, st>>>(gap, (const T*)sp.fc_w, sp.fc_b, B, C, K, z);
+    fc_kernel<T, V><<<cdiv(K, kFcClasses), kFcWarps * 32, 0, st>>>(gap, (const T*)sp.fc_w, sp.fc_b, B, C, K, z, da);
   else
-    fc_kernel<T, 1><<<cdiv(K, kFcClasses), kFcWarps * 32, 0, st>>>(gap, (const T*)sp.fc_w, sp.fc_b, B, C, K, z);
+    fc_kernel<T, 1><<<cdiv(K, kFcClasses), kFcWarps * 32, 0, st>>>(gap, (const T*)sp.fc_w, sp.fc_b, B, C, K, z, da);
   EE_CUDA(cudaGetLastError());
-  if (timed) record(m, sp, st, "head_fc");
-  exit_decide_kernel<<<1, kDecideThreads, 0, st>>>(z, B, K, shift, shift_cls, sp.threshold, sp.always_exit, out->conf,
-                                                   out->pred, out->exit_mask, in_ids ? in_ids->ids : nullptr,
-                                                   out->survivor_idx, out->ids_out, out->n_surv_dev);
-  EE_CUDA(cudaGetLastError());
-  if (timed) record(m, sp, st, "head_softmax_scan");
+  if (timed) record(m, sp, st, "head_fc_softmax_scan");
   return EE_OK;
 }
 

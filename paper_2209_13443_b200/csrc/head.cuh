@@ -97,80 +97,140 @@ gap_kernel(const T* __restrict__ x, int HW, int C, int rows_per_chunk, float* __
   if (tid == 0) counters[b] = 0;
 }
 
+struct DecideArgs {  // everything the exit decision needs besides the logits
+  const float* shift;
+  const int32_t* shift_cls;
+  float thr;
+  int always_exit;
+  float* conf;
+  int32_t* pred;
+  uint8_t* mask;
+  const int32_t* ids;
+  int32_t* surv_idx;
+  int32_t* ids_out;
+  int32_t* n_surv;
+  unsigned* done;  // CTAs of the FC kernel that have written their logits; zero between launches
+};
+
+template <int THREADS>
+__device__ __forceinline__ void exit_decide_block(float* z, int B, int K, const float* __restrict__ shift,
+                                                  const int32_t* __restrict__ shift_cls, float thr, int always_exit,
+                                                  float* __restrict__ conf, int32_t* __restrict__ pred, uint8_t* mask,
+                                                  const int32_t* __restrict__ ids, int32_t* __restrict__ surv_idx,
+                                                  int32_t* __restrict__ ids_out, int32_t* __restrict__ n_surv);
+
 constexpr int kFcWarps = 8, kFcClassesPerWarp = 2, kFcSamples = 16, kFcChunk = 256;
 constexpr int kFcClasses = kFcWarps * kFcClassesPerWarp;
 
 // z[b][k] = bfc[k] + sum_c wfc[k][c] * gap[b][c].  A CTA owns 16 classes (two per warp) and walks the samples in
 // tiles of 16; the tile's pooled vectors are staged in shared memory 256 channels at a time, so the pooled matrix
 // crosses L2 once per CTA.  Per (b, k): every lane adds its channels in ascending order, then a shuffle tree;
-// the order does not depend on the batch size.
+// the order does not depend on the batch size.  The CTA that finishes last (a counter, no waiting) goes on to the
+// exit decision for the whole batch: softmax top-1, threshold, stable scan of the survivors.
 template <typename T, int VEC>
 __global__ void __launch_bounds__(kFcWarps * 32)
 fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float* __restrict__ bfc, int B, int C, int K,
-          float* __restrict__ z) {
+          float* z, DecideArgs d) {
   __shared__ __align__(16) float gs[kFcSamples][kFcChunk];
+  __shared__ bool last_cta;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int k0 = blockIdx.x * kFcClasses + warp * kFcClassesPerWarp;
-  constexpr int PER = kFcChunk / 32;  // channels per lane per chunk (8)
-  for (int b0 = 0; b0 < B; b0 += kFcSamples) {
-    float acc[kFcClassesPerWarp][kFcSamples];
+  constexpr int PER = kFcChunk / 32;                              // channels per lane per chunk (8)
+  constexpr int STG = kFcSamples * kFcChunk / (kFcWarps * 32);    // staged floats per thread per step (16)
+  const int nchunk = (C + kFcChunk - 1) / kFcChunk;
+  const int nstep = ((B + kFcSamples - 1) / kFcSamples) * nchunk; // (sample tile, channel chunk) pairs, tile-major
+
+  // One step ahead in registers: the pooled values this thread stages and the weight vectors of its two classes, so
+  // that the global-load latency of step i + 1 hides behind the arithmetic of step i.
+  float pre[STG];
+  float wnext[kFcClassesPerWarp][PER];
+  auto fetch = [&](int step) {
+    const int b0 = (step / nchunk) * kFcSamples, c0 = (step % nchunk) * kFcChunk;
 #pragma unroll
-    for (int q = 0; q < kFcClassesPerWarp; ++q)
-#pragma unroll
-      for (int s = 0; s < kFcSamples; ++s) acc[q][s] = 0.f;
-    for (int c0 = 0; c0 < C; c0 += kFcChunk) {
-      __syncthreads();
-      for (int i = threadIdx.x; i < kFcSamples * kFcChunk; i += kFcWarps * 32) {
-        const int s = i / kFcChunk, c = i - s * kFcChunk;
-        gs[s][c] = (b0 + s < B && c0 + c < C) ? gap[(size_t)(b0 + s) * C + c0 + c] : 0.f;
-      }
-      __syncthreads();
-      const int c = c0 + lane * PER;
-      float wv[kFcClassesPerWarp][PER];
-#pragma unroll
-      for (int q = 0; q < kFcClassesPerWarp; ++q) {
-        const int k = k0 + q;
-#pragma unroll
-        for (int e = 0; e < PER; ++e) wv[q][e] = 0.f;
-        if (k < K) {
-          if constexpr (VEC == 8) {
-            if (c + PER <= C) {
-              Vec16<T> t;
-              t.load(wfc + (size_t)k * C + c);
-#pragma unroll
-              for (int e = 0; e < PER; ++e) wv[q][e] = t.v[e];
-            }
-          } else {
-#pragma unroll
-            for (int e = 0; e < PER; ++e)
-              if (c + e < C) wv[q][e] = Elem<T>::ld(wfc + (size_t)k * C + c + e);
-          }
-        }
-      }
-#pragma unroll
-      for (int s = 0; s < kFcSamples; ++s) {
-        const float4 g0 = *reinterpret_cast<const float4*>(&gs[s][lane * PER]);
-        const float4 g1 = *reinterpret_cast<const float4*>(&gs[s][lane * PER + 4]);
-        const float gv[PER] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-#pragma unroll
-        for (int q = 0; q < kFcClassesPerWarp; ++q)
-#pragma unroll
-          for (int e = 0; e < PER; ++e) acc[q][s] = fmaf(wv[q][e], gv[e], acc[q][s]);
-      }
+    for (int u = 0; u < STG; ++u) {
+      const int i = threadIdx.x + u * (kFcWarps * 32);
+      const int sidx = i / kFcChunk, c = i - sidx * kFcChunk;
+      pre[u] = (b0 + sidx < B && c0 + c < C) ? gap[(size_t)(b0 + sidx) * C + c0 + c] : 0.f;
     }
+    const int c = c0 + lane * PER;
 #pragma unroll
     for (int q = 0; q < kFcClassesPerWarp; ++q) {
       const int k = k0 + q;
-      const float bk = (bfc && k < K) ? bfc[k] : 0.f;
 #pragma unroll
-      for (int s = 0; s < kFcSamples; ++s) {
-        float v = acc[q][s];
+      for (int e = 0; e < PER; ++e) wnext[q][e] = 0.f;
+      if (k < K) {
+        if constexpr (VEC == 8) {
+          if (c + PER <= C) {
+            Vec16<T> t;
+            t.load(wfc + (size_t)k * C + c);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0 && k < K && b0 + s < B) z[(size_t)(b0 + s) * K + k] = v + bk;
+            for (int e = 0; e < PER; ++e) wnext[q][e] = t.v[e];
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < PER; ++e)
+            if (c + e < C) wnext[q][e] = Elem<T>::ld(wfc + (size_t)k * C + c + e);
+        }
+      }
+    }
+  };
+  float acc[kFcClassesPerWarp][kFcSamples];
+  if (nstep > 0) fetch(0);
+  for (int step = 0; step < nstep; ++step) {
+    const int b0 = (step / nchunk) * kFcSamples, ci = step % nchunk;
+    if (ci == 0) {
+#pragma unroll
+      for (int q = 0; q < kFcClassesPerWarp; ++q)
+#pragma unroll
+        for (int s2 = 0; s2 < kFcSamples; ++s2) acc[q][s2] = 0.f;
+    }
+    __syncthreads();  // everyone is done reading the previous step's tile
+#pragma unroll
+    for (int u = 0; u < STG; ++u) {
+      const int i = threadIdx.x + u * (kFcWarps * 32);
+      (&gs[0][0])[i] = pre[u];
+    }
+    float wv[kFcClassesPerWarp][PER];
+#pragma unroll
+    for (int q = 0; q < kFcClassesPerWarp; ++q)
+#pragma unroll
+      for (int e = 0; e < PER; ++e) wv[q][e] = wnext[q][e];
+    __syncthreads();
+    if (step + 1 < nstep) fetch(step + 1);
+#pragma unroll
+    for (int s2 = 0; s2 < kFcSamples; ++s2) {
+      const float4 g0 = *reinterpret_cast<const float4*>(&gs[s2][lane * PER]);
+      const float4 g1 = *reinterpret_cast<const float4*>(&gs[s2][lane * PER + 4]);
+      const float gv[PER] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+      for (int q = 0; q < kFcClassesPerWarp; ++q)
+#pragma unroll
+        for (int e = 0; e < PER; ++e) acc[q][s2] = fmaf(wv[q][e], gv[e], acc[q][s2]);
+    }
+    if (ci == nchunk - 1) {
+#pragma unroll
+      for (int q = 0; q < kFcClassesPerWarp; ++q) {
+        const int k = k0 + q;
+        const float bk = (bfc && k < K) ? bfc[k] : 0.f;
+#pragma unroll
+        for (int s2 = 0; s2 < kFcSamples; ++s2) {
+          float v = acc[q][s2];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+          if (lane == 0 && k < K && b0 + s2 < B) z[(size_t)(b0 + s2) * K + k] = v + bk;
+        }
       }
     }
   }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) last_cta = atomicAdd(d.done, 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (!last_cta) return;
+  __threadfence();
+  if (threadIdx.x == 0) *d.done = 0;
+  exit_decide_block<kFcWarps * 32>(z, B, K, d.shift, d.shift_cls, d.thr, d.always_exit, d.conf, d.pred, d.mask, d.ids, d.surv_idx,
+                                   d.ids_out, d.n_surv);
 }
 
 constexpr int kDecideThreads = 1024;
@@ -178,16 +238,17 @@ constexpr int kDecideThreads = 1024;
 // One CTA.  Per sample (one warp each): optional logit shift, max / lowest argmax, conf = 1 / sum exp(z - max),
 // exit = always || conf >= thr (NaN never exits).  Then a ballot + prefix-sum scan over the not-exit flags
 // gives the ascending survivor list, the survivors' ids and their count.
-__global__ void __launch_bounds__(kDecideThreads)
-exit_decide_kernel(float* __restrict__ z, int B, int K, const float* __restrict__ shift, const int32_t* __restrict__ shift_cls,
-                   float thr, int always_exit, float* __restrict__ conf, int32_t* __restrict__ pred,
-                   uint8_t* __restrict__ mask, const int32_t* __restrict__ ids, int32_t* __restrict__ surv_idx,
-                   int32_t* __restrict__ ids_out, int32_t* __restrict__ n_surv) {
+template <int THREADS>
+__device__ __forceinline__ void exit_decide_block(float* z, int B, int K, const float* __restrict__ shift,
+                                                  const int32_t* __restrict__ shift_cls, float thr, int always_exit,
+                                                  float* __restrict__ conf, int32_t* __restrict__ pred, uint8_t* mask,
+                                                  const int32_t* __restrict__ ids, int32_t* __restrict__ surv_idx,
+                                                  int32_t* __restrict__ ids_out, int32_t* __restrict__ n_surv) {
   __shared__ int warp_tot[32];
   __shared__ int pass_total;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int kRegs = 32;  // logits per lane held in registers: one pass over memory for K <= 1024
-  for (int b = warp; b < B; b += kDecideThreads / 32) {
+  for (int b = warp; b < B; b += THREADS / 32) {
     float* zb = z + (size_t)b * K;
     const int cls = (shift && shift_cls) ? shift_cls[b] : -1;
     const float sh = cls >= 0 && cls < K ? shift[b] : 0.f;
@@ -197,7 +258,7 @@ exit_decide_kernel(float* __restrict__ z, int B, int K, const float* __restrict_
 #pragma unroll
     for (int i = 0; i < kRegs; ++i) {
       const int k = lane + 32 * i;
-      zr[i] = k < K ? zb[k] : -INFINITY;
+      zr[i] = k < K ? __ldcg(zb + k) : -INFINITY;   // logits may come from other CTAs: read through L2
     }
 #pragma unroll
     for (int i = 0; i < kRegs; ++i) {
@@ -212,7 +273,7 @@ exit_decide_kernel(float* __restrict__ z, int B, int K, const float* __restrict_
       }
     }
     for (int k = lane + 32 * kRegs; k < K; k += 32) {  // classes past the register window
-      float v = zb[k];
+      float v = __ldcg(zb + k);
       if (k == cls) {
         v += sh;
         zb[k] = v;
@@ -236,7 +297,7 @@ exit_decide_kernel(float* __restrict__ z, int B, int K, const float* __restrict_
 #pragma unroll
     for (int i = 0; i < kRegs; ++i)
       if (lane + 32 * i < K) s += expf(zr[i] - m);
-    for (int k = lane + 32 * kRegs; k < K; k += 32) s += expf(zb[k] - m);
+    for (int k = lane + 32 * kRegs; k < K; k += 32) s += expf(__ldcg(zb + k) - m);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     if (lane == 0) {
@@ -248,7 +309,7 @@ exit_decide_kernel(float* __restrict__ z, int B, int K, const float* __restrict_
   }
   __syncthreads();
   int base = 0;  // identical in every thread
-  for (int p0 = 0; p0 < B; p0 += kDecideThreads) {
+  for (int p0 = 0; p0 < B; p0 += THREADS) {
     const int b = p0 + tid;
     const bool keep = b < B && mask[b] == 0;
     const unsigned bal = __ballot_sync(0xffffffffu, keep);
@@ -256,7 +317,7 @@ exit_decide_kernel(float* __restrict__ z, int B, int K, const float* __restrict_
     if (lane == 0) warp_tot[warp] = __popc(bal);
     __syncthreads();
     if (warp == 0) {
-      const int t = warp_tot[lane];
+      const int t = lane < THREADS / 32 ? warp_tot[lane] : 0;
       int inc = t;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -276,6 +337,14 @@ exit_decide_kernel(float* __restrict__ z, int B, int K, const float* __restrict_
     __syncthreads();
   }
   if (tid == 0) n_surv[0] = base;
+}
+
+__global__ void __launch_bounds__(kDecideThreads)
+exit_decide_kernel(float* z, int B, int K, const float* __restrict__ shift, const int32_t* __restrict__ shift_cls, float thr,
+                   int always_exit, float* __restrict__ conf, int32_t* __restrict__ pred, uint8_t* mask,
+                   const int32_t* __restrict__ ids, int32_t* __restrict__ surv_idx, int32_t* __restrict__ ids_out,
+                   int32_t* __restrict__ n_surv) {
+  exit_decide_block<kDecideThreads>(z, B, K, shift, shift_cls, thr, always_exit, conf, pred, mask, ids, surv_idx, ids_out, n_surv);
 }
 
 constexpr int kCopyThreads = 256, kCopyUnroll = 8;
