@@ -43,11 +43,13 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "tf_burst": 1590.0, "tf_sustained": 1400.0, "source": "fallback"}
 
 
-def make_spec(workload: str, batch: int):
+def make_spec(workload: str, batch: int, flat_heads: bool = False):
     from paper_2209_13443_b200 import workloads as wl
 
     if workload == "resnet50":
-        return wl.resnet50_ee(seed=1, max_batch=batch), 1
+        # flat_heads: FC weights scaled down so that unshifted confidences sit near 1/1000 and only the forced
+        # Bernoulli logit shifts of the exit-rate sweep decide who leaves
+        return wl.resnet50_ee(seed=1, max_batch=batch, alphas=[0.01] * 4 if flat_heads else None), 1
     if workload == "mobilenetv2":
         return wl.mobilenetv2_ee(seed=2, max_batch=batch), 2
     if workload == "tiny":
@@ -55,8 +57,9 @@ def make_spec(workload: str, batch: int):
     raise SystemExit(f"unknown workload {workload}")
 
 
-def workload_name(spec, batch):
-    return f"{spec.name} {spec.dtype} B={batch} {spec.in_h}x{spec.in_w}x{spec.in_c}, {len(spec.stages)} exits, calibrated exit rates"
+def workload_name(spec, batch, exit_rate=None):
+    rates = "calibrated exit rates" if exit_rate is None else f"forced exit rate p={exit_rate} per exit (seeded Bernoulli logit shifts)"
+    return f"{spec.name} {spec.dtype} B={batch} {spec.in_h}x{spec.in_w}x{spec.in_c}, {len(spec.stages)} exits, {rates}"
 
 
 class ClockSampler:
@@ -175,7 +178,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     peaks = load_peaks()
     B, K, W = args.batch, args.steps, max(args.warmup, 3)
-    spec, seed = make_spec(args.workload, B)
+    spec, seed = make_spec(args.workload, B, flat_heads=args.exit_rate is not None)
     model = eb.EEModel(spec)
     nst = model.n_stages
     bufs = [eb.StageBuffers(model, s, with_logits=False) for s in range(nst)]
@@ -196,6 +199,23 @@ def run_ours(args):
     torch.cuda.set_stream(side)
     stream = torch.cuda.current_stream()
     sizes_last = []
+    # exit-rate sweep: per (sample id, exit) one seeded Bernoulli(p) draw forces the exit through a logit shift; the
+    # survivors of every stage are known in advance, so the per-stage shift vectors are laid out in batch order here
+    forced = [None] * nst
+    if args.exit_rate is not None:
+        draws, shifts, cls = wl.bernoulli_exit_shifts(4, world * B, nst - 1, args.exit_rate, spec.stages[0].n_classes)
+        alive = np.arange(first_id, first_id + B)
+        for s in range(nst - 1):
+            forced[s] = (torch.from_numpy(shifts[s][alive]).cuda(), torch.from_numpy(cls[alive]).cuda())
+            alive = alive[draws[s][alive] == 0]
+
+    def run_stage(s, feat, n, ids):
+        if forced[s] is not None:
+            assert n == forced[s][0].numel(), "survivors must follow the forced draws"
+            model.stage_run(s, feat, n, bufs[s], ws, ids, forced[s][0], forced[s][1])
+        else:
+            model.stage_run(s, feat, n, bufs[s], ws, ids)
+
     def stage_launches(s, n):
         """Kernels one ee_stage_run launches: the layers' (a packed stem packs and multiplies chunk by chunk),
         two for the head (pooling; FC with the exit decision in its last CTA), one gather."""
@@ -214,7 +234,7 @@ def run_ours(args):
         sizes = []
         for s in range(nst):
             sizes.append(n)
-            model.stage_run(s, feat, n, bufs[s], ws, ids)
+            run_stage(s, feat, n, ids)
             nl += stage_launches(s, n)
             if e2e:
                 res_host[s]["conf"][:n].copy_(bufs[s].conf[:n], non_blocking=True)
@@ -271,7 +291,7 @@ def run_ours(args):
         model.batch_refill(0, batch0, ids0, 0, x_dev, ids_dev, B)
         feat, ids, n = batch0, ids0, B
         for s in range(nst):
-            model.stage_run(s, feat, n, bufs[s], ws, ids)
+            run_stage(s, feat, n, ids)
             stream.synchronize()
             plan = model.plan(s, n)
             tm = model.get_timing(s)
@@ -338,7 +358,7 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": spec.dtype, "data": "synthetic",
-        "config": {"workload": workload_name(spec, B), "global_batch": world * B, "parallelism": f"replicas x{world}",
+        "config": {"workload": workload_name(spec, B, args.exit_rate), "global_batch": world * B, "parallelism": f"replicas x{world}",
                    "l2": "flushed between timed steps (256 MB write)", "batch_per_stage": sizes_last},
         "clocks": clocks,
         "e2e": {"value": replicas.job_throughput(world, B, K, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -363,6 +383,44 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_trace(args):
+    """Streaming fluid-batch trace: seeded Poisson arrivals served by the exit-aware preemptive loop (Algorithm 1,
+    T_SLO = infinity) on the wall clock; request r carries image r mod 256 of a fixed pool."""
+    import torch
+
+    from paper_2209_13443_b200 import binding as eb
+    from paper_2209_13443_b200 import workloads as wl
+    from paper_2209_13443_b200.serving import FluidServer
+
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    spec, seed = make_spec(args.workload, args.batch)
+    pool = eb.to_device(spec.dtype, wl.make_input(spec, 256, seed=seed))
+    n = args.trace_requests
+    image_of = [r % 256 for r in range(n)]
+    side = torch.cuda.Stream()
+    torch.cuda.set_stream(side)
+    srv = FluidServer(spec)
+    warm = wl.poisson_arrivals(5, 300, 1e5)                 # a burst: touches every batch size once before timing
+    srv.serve(warm, image_of[:300], pool)
+    arrivals = wl.poisson_arrivals(3, n, args.trace_rate)
+    out = srv.serve(arrivals, image_of, pool)
+    lat = (out["finish"] - arrivals) * 1e3
+    span = float(out["finish"].max() - arrivals[0])
+    sizes = [len(ids) for _, ids in out["launches"]]
+    exits = np.bincount(out["exit_stage"], minlength=len(spec.stages)).tolist()
+    print(json.dumps({
+        "metric": METRIC, "value": n / span, "unit": UNIT, "n_gpus": 1, "steps": n, "warmup": 300, "ms_per_step": span / n * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": spec.dtype, "data": "synthetic",
+        "config": {"workload": f"{spec.name} {spec.dtype} streaming trace, {n} requests, Poisson {args.trace_rate:g} req/s, B_max={args.batch}, "
+                               "Algorithm 1 with T_SLO=inf, wall clock"},
+        "latency_ms": {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99)), "mean": float(lat.mean())},
+        "stage_launches": len(sizes), "mean_batch": float(np.mean(sizes)), "max_batch_seen": int(max(sizes)),
+        "exits_per_stage": exits,
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -371,11 +429,18 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=64)
     ap.add_argument("--workload", default="resnet50", choices=["resnet50", "mobilenetv2", "tiny"])
+    ap.add_argument("--exit-rate", type=float, default=None,
+                    help="exit-rate sweep: force this fraction of the samples reaching each early exit to leave (resnet50 only)")
+    ap.add_argument("--trace-rate", type=float, default=None,
+                    help="streaming trace instead of fixed batches: Poisson arrivals at this many requests/s, Algorithm 1 with T_SLO = inf")
+    ap.add_argument("--trace-requests", type=int, default=2000)
     ap.add_argument("--cpu-samples", type=int, default=16)
     ap.add_argument("--report-layers", action="store_true", help="add a per-layer table (time, TFLOP/s, GB/s, roofline bound) to the JSON line")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.trace_rate is not None:
+        run_trace(args)
     else:
         run_ours(args)
 
