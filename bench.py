@@ -73,7 +73,7 @@ class ClockSampler:
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "20",
                                           "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._pump, daemon=True).start()
         except Exception:
@@ -424,7 +424,7 @@ def run_trace(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=64)
@@ -434,7 +434,7 @@ def main():
     ap.add_argument("--trace-rate", type=float, default=None,
                     help="streaming trace instead of fixed batches: Poisson arrivals at this many requests/s, Algorithm 1 with T_SLO = inf")
     ap.add_argument("--trace-requests", type=int, default=2000)
-    ap.add_argument("--cpu-samples", type=int, default=16)
+    ap.add_argument("--cpu-samples", type=int, default=64)
     ap.add_argument("--report-layers", action="store_true", help="add a per-layer table (time, TFLOP/s, GB/s, roofline bound) to the JSON line")
     args = ap.parse_args()
     if args.impl == "reference":
