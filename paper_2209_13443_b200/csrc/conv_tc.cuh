@@ -28,6 +28,7 @@ namespace ee {
 
 constexpr int kTcBM = 128;       // output pixels per CTA (= TMEM lanes)
 constexpr int kTcBK = 64;        // bf16 elements per K block: 128 bytes = one swizzle span
+constexpr int kTcSplitMaxCtas = 296;  // split-K only while tiles x ranges at max_batch stay within two CTAs per SM
 constexpr int kTcThreads = 192;  // producer warp, MMA warp, four epilogue warps
 constexpr long long kTcWaitCycles = 4000000000LL;  // ~2 s at boost clock; far beyond any healthy wait
 
@@ -872,11 +873,13 @@ inline ee_status_t tc_context_init(TcContext& c) {
   set(conv_igemm_tcgen05_kernel<64, 2, true, false, false>, TcSmem<64, 2, true>::kBytes);
   set(conv_igemm_tcgen05_kernel<64, 5, true, false, false>, TcSmem<64, 5, true>::kBytes);
   set(conv_igemm_tcgen05_kernel<64, 6, false, true, false>, TcSmem<64, 6, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 3, false, true, false>, TcSmem<64, 3, false>::kBytes);
   set(conv_igemm_tcgen05_kernel<128, 3, false, false, false>, TcSmem<128, 3, false>::kBytes);
   set(conv_igemm_tcgen05_kernel<128, 6, false, false, false>, TcSmem<128, 6, false>::kBytes);
   set(conv_igemm_tcgen05_kernel<128, 2, true, false, false>, TcSmem<128, 2, true>::kBytes);
   set(conv_igemm_tcgen05_kernel<128, 5, true, false, false>, TcSmem<128, 5, true>::kBytes);
   set(conv_igemm_tcgen05_kernel<128, 6, false, true, false>, TcSmem<128, 6, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 3, false, true, false>, TcSmem<128, 3, false>::kBytes);
   set(conv_igemm_tcgen05_persistent_kernel<64, false>, TcPersistSmem<64, false>::kBytes);
   set(conv_igemm_tcgen05_persistent_kernel<64, true>, TcPersistSmem<64, true>::kBytes);
   set(conv_igemm_tcgen05_persistent_kernel<128, false>, TcPersistSmem<128, false>::kBytes);
@@ -912,7 +915,7 @@ inline ee_status_t tc_plan_layer(TcContext& c, const ee_layer_desc_t& d, int in_
     L->kb_per = num_kb;
     for (int sp = 8; sp >= 2; sp >>= 1) {
       const int per = cdiv(num_kb, sp);
-      if (tiles * sp <= 148 && sp * 4 <= num_kb && (sp - 1) * per < num_kb) {
+      if (tiles * sp <= kTcSplitMaxCtas && sp * 8 <= num_kb && (sp - 1) * per < num_kb) {
         L->splits = sp;
         L->kb_per = per;
         break;
@@ -1010,7 +1013,7 @@ inline cudaError_t tc_launch_t(dim3 grid, cudaStream_t st, const CUtensorMap& a,
 template <int BN>
 inline cudaError_t tc_launch_bn(bool deep, bool res, bool split, dim3 grid, cudaStream_t st, const CUtensorMap& a, const CUtensorMap& w,
                                 const CUtensorMap& r, const CUtensorMap& o, const TcParams& p) {
-  if (split) return tc_launch_t<BN, 6, false, true>(grid, st, a, w, r, o, p);  // small grids by construction: deep ring
+  if (split) return deep ? tc_launch_t<BN, 6, false, true>(grid, st, a, w, r, o, p) : tc_launch_t<BN, 3, false, true>(grid, st, a, w, r, o, p);
   if (res) return deep ? tc_launch_t<BN, 5, true, false>(grid, st, a, w, r, o, p) : tc_launch_t<BN, 2, true, false>(grid, st, a, w, r, o, p);
   return deep ? tc_launch_t<BN, 6, false, false>(grid, st, a, w, r, o, p) : tc_launch_t<BN, 3, false, false>(grid, st, a, w, r, o, p);
 }
