@@ -565,17 +565,22 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
 // drain accumulator j & 1 of tile j, the MMA warp already fills the other one with tile j + 1, and the producer is
 // further ahead still.  A tile then costs max(load, MMA, epilogue) instead of their sum, and the per-CTA prologue
 // (barriers, TMEM allocation, descriptor fetch) is paid once per SM instead of once per tile.
-// Residual tiles and staged outputs alternate between two 128 x BN bf16 buffers; a buffer returns to the producer
-// (io_free) once all four epilogue warps have seen their TMA store finish reading it.
+// Staged outputs leave through TMA stores; a staging tile is rewritten only after the warp has seen its previous store
+// finish reading it.  Residual tiles are prefetched by the producer into two buffers of their own, which return to it
+// (res_free) as soon as all four epilogue warps have read them.
 template <int BN, bool RES>
 struct TcPersistSmem {
-  static constexpr int kStages = BN == 128 ? 4 : 7;
+  // without a residual: a longer ring and two output staging tiles; with one: two residual tiles the producer
+  // prefetches (free again as soon as the epilogue has read them) and a single staging tile
+  static constexpr int kStages = RES ? (BN == 128 ? 3 : 5) : (BN == 128 ? 4 : 7);
   static constexpr int kABytes = kTcBM * kTcBK * 2;
   static constexpr int kBBytes = BN * kTcBK * 2;
   static constexpr int kStage = kABytes + kBBytes;
   static constexpr int kTiles = kStages * kStage;
   static constexpr int kIoBytes = kTcBM * BN * 2;
-  static constexpr int kAfter = kTiles + 2 * kIoBytes;
+  static constexpr int kROff = kTiles;
+  static constexpr int kOOff = kTiles + (RES ? 2 * kIoBytes : 0);
+  static constexpr int kAfter = kOOff + (RES ? 1 : 2) * kIoBytes;
   static constexpr int kBytes = kAfter + 4 * 2 * BN * 4 + 256 + 1024;  // + one scale/bias copy per epilogue warp, barriers, slack
   static_assert(kBytes <= 227 * 1024, "exceeds the shared memory of an SM");
 };
@@ -598,7 +603,7 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
   auto acc_full = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
   auto acc_empty = [&](int b) { return bar0 + 8u * (2 * kStages + 2 + b); };
   auto res_full = [&](int b) { return bar0 + 8u * (2 * kStages + 4 + b); };
-  auto io_free = [&](int b) { return bar0 + 8u * (2 * kStages + 6 + b); };
+  auto res_free = [&](int b) { return bar0 + 8u * (2 * kStages + 6 + b); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -617,7 +622,7 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
       mbar_init(acc_full(b), 1);
       mbar_init(acc_empty(b), 4);   // lane 0 of each epilogue warp
       mbar_init(res_full(b), 1);
-      mbar_init(io_free(b), 4);
+      mbar_init(res_free(b), 4);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -647,14 +652,14 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
         const int m0 = (t / n_tiles) * kTcBM, n0 = (t % n_tiles) * BN;
         const int b = j & 1;
         if (RES) {
-          if (j >= 2) ok = mbar_wait(io_free(b), (uint32_t)((j >> 1) - 1) & 1u, p.err_flag);
+          if (j >= 2) ok = mbar_wait(res_free(b), (uint32_t)((j >> 1) - 1) & 1u, p.err_flag);
           if (!ok) break;
           mbar_expect_tx(res_full(b), S::kIoBytes);
 #pragma unroll
           for (int h = 0; h < BN / 64; ++h)
 #pragma unroll
             for (int q = 0; q < 4; ++q)
-              tma_load_2d(base + S::kTiles + b * S::kIoBytes + h * 16384 + q * 4096, &tmR, res_full(b), n0 + h * 64, m0 + q * 32);
+              tma_load_2d(base + S::kROff + b * S::kIoBytes + h * 16384 + q * 4096, &tmR, res_full(b), n0 + h * 64, m0 + q * 32);
         }
         int cw = 0, ch = 0, cn = 0;
         if (p.im2col) {
@@ -736,12 +741,13 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
       if (RES && ok) ok = __all_sync(0xffffffffu, mbar_wait(res_full(b), (uint32_t)(j >> 1) & 1u, p.err_flag));
       if (!ok) break;
       tc_fence_after();
-      uint8_t* io = gen + S::kTiles + b * S::kIoBytes;
-      const uint32_t io_s = base + S::kTiles + b * S::kIoBytes;
+      const int ob = RES ? 0 : b;  // output staging tile of this tile
+      uint8_t* io = gen + S::kOOff + ob * S::kIoBytes;
+      const uint32_t io_s = base + S::kOOff + ob * S::kIoBytes;
+      const uint8_t* rin = gen + S::kROff + b * S::kIoBytes;
       const uint32_t acc = tmem_base + (uint32_t)(b * BN) + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
       for (int h = 0; h < BN / 64; ++h) {
-        uint8_t* line = io + h * 16384 + row * 128;
         float va[32], vb[32];  // both 32-column loads of the half in flight before one wait
         tmem_ld32_issue(acc + (uint32_t)(h * 64), va);
         tmem_ld32_issue(acc + (uint32_t)(h * 64 + 32), vb);
@@ -751,6 +757,13 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
           __syncwarp();
           if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acc_empty(b)) : "memory");
         }
+        if (RES && h == 0) {  // single staging tile: this warp's previous store must have finished reading it
+          if (lane == 0 && pending) {
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            pending = false;
+          }
+          __syncwarp();
+        }
 #pragma unroll
         for (int sub = 0; sub < 2; ++sub) {
           const int c0 = h * 64 + sub * 32;
@@ -759,27 +772,29 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
           for (int i = 0; i < 32; ++i) v[i] = fmaf(sc[c0 + i], v[i], sc[BN + c0 + i]);
 #pragma unroll
           for (int gq = 0; gq < 4; ++gq) {
-            bf16* chunk = reinterpret_cast<bf16*>(line + (((sub * 4 + gq) ^ (lane & 7)) << 4));
+            const int off = h * 16384 + row * 128 + (((sub * 4 + gq) ^ (lane & 7)) << 4);
             if (RES) {
               Vec16<bf16> r;
-              r.load(chunk);
+              r.load(reinterpret_cast<const bf16*>(rin + off));
 #pragma unroll
               for (int e = 0; e < 8; ++e) v[gq * 8 + e] += r.v[e];
             }
             Vec16<bf16> o;
 #pragma unroll
             for (int e = 0; e < 8; ++e) o.v[e] = apply_act(v[gq * 8 + e], p.act);
-            o.store(chunk);
+            o.store(reinterpret_cast<bf16*>(io + off));
           }
-          if (h == 0 && sub == 0 && lane == 0 && pending) {
-            // One chunk into tile j, this warp's store of tile j - 1 has long finished reading its buffer: confirm it
-            // (no stall in the steady state) and hand the buffer back to the producer for the residual of tile j + 1.
-            // It also licenses the next iteration to overwrite that buffer.
+          if (!RES && h == 0 && sub == 0 && lane == 0 && pending) {
+            // One chunk into tile j, this warp's store of tile j - 1 has long finished reading its staging tile:
+            // confirm it (no stall in the steady state); it licenses the next iteration to overwrite that tile.
             asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             pending = false;
-            if (RES) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(io_free((j - 1) & 1)) : "memory");
           }
         }
+      }
+      if (RES) {  // the residual tile is consumed: the producer may prefetch the one of tile j + 2 into it
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(res_free(b)) : "memory");
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
@@ -1081,7 +1096,7 @@ inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, co
     return ge == cudaSuccess ? EE_OK : EE_ERR_CUDA;
   }
   const long tiles = (long)grid.x * grid.y;
-  if (!split && !res && L.kh * L.kw == 1 && tiles >= 2 * c.sm_count) {  // several waves of short K loops: one persistent CTA per SM walks the tiles
+  if (!split && L.kh * L.kw == 1 && tiles >= 2 * c.sm_count) {  // several waves of short K loops: one persistent CTA per SM walks the tiles
     const int ctas = c.sm_count;
     cudaError_t pe;
     if (L.bn == 128)
