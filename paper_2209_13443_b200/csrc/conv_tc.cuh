@@ -572,6 +572,8 @@ template <int BN, bool RES>
 struct TcPersistSmem {
   // without a residual: a longer ring and two output staging tiles; with one: two residual tiles the producer
   // prefetches (free again as soon as the epilogue has read them) and a single staging tile
+  static constexpr int kEpiWarps = BN == 128 ? 8 : 4;   // at BN = 128 two warps share a TMEM lane quarter, one per 64-column half
+  static constexpr int kThreads = 64 + 32 * kEpiWarps;
   static constexpr int kStages = RES ? (BN == 128 ? 3 : 5) : (BN == 128 ? 4 : 7);
   static constexpr int kABytes = kTcBM * kTcBK * 2;
   static constexpr int kBBytes = BN * kTcBK * 2;
@@ -581,12 +583,12 @@ struct TcPersistSmem {
   static constexpr int kROff = kTiles;
   static constexpr int kOOff = kTiles + (RES ? 2 * kIoBytes : 0);
   static constexpr int kAfter = kOOff + (RES ? 1 : 2) * kIoBytes;
-  static constexpr int kBytes = kAfter + 4 * 2 * BN * 4 + 256 + 1024;  // + one scale/bias copy per epilogue warp, barriers, slack
+  static constexpr int kBytes = kAfter + kEpiWarps * 2 * BN * 4 + 256 + 1024;  // + one scale/bias copy per epilogue warp, barriers, slack
   static_assert(kBytes <= 227 * 1024, "exceeds the shared memory of an SM");
 };
 
 template <int BN, bool RES>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(TcPersistSmem<BN, RES>::kThreads, 1)
 conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                                      const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmO, TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -595,9 +597,9 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
-  float* s_sb = reinterpret_cast<float*>(gen + S::kAfter);  // [4 epilogue warps][scale BN | bias BN]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kAfter + 8 * BN * 4);
-  const uint32_t bar0 = base + S::kAfter + 8 * BN * 4;
+  float* s_sb = reinterpret_cast<float*>(gen + S::kAfter);  // [epilogue warps][scale BN | bias BN]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kAfter + S::kEpiWarps * 2 * BN * 4);
+  const uint32_t bar0 = base + S::kAfter + S::kEpiWarps * 2 * BN * 4;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
   auto acc_full = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
@@ -620,9 +622,9 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(acc_full(b), 1);
-      mbar_init(acc_empty(b), 4);   // lane 0 of each epilogue warp
+      mbar_init(acc_empty(b), S::kEpiWarps);   // lane 0 of each epilogue warp
       mbar_init(res_full(b), 1);
-      mbar_init(res_free(b), 4);
+      mbar_init(res_free(b), S::kEpiWarps);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -719,7 +721,9 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
   } else {
     const int q = warp & 3;
     const int row = q * 32 + lane;
-    float* sc = s_sb + q * 2 * BN;  // this warp's own copy: no barrier across warps inside the tile loop
+    const int ew = warp - 2;
+    const int h0 = BN == 128 ? (ew >> 2) : 0, h1 = h0 + 1;  // the 64-column half (halves) this warp owns
+    float* sc = s_sb + ew * 2 * BN;  // this warp's own copy: no barrier across warps inside the tile loop
     bool ok = true;
     int sc_n0 = -1;
     bool pending = false;  // lane 0: a bulk store group of this warp may still be reading shared memory
@@ -747,17 +751,17 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
       const uint8_t* rin = gen + S::kROff + b * S::kIoBytes;
       const uint32_t acc = tmem_base + (uint32_t)(b * BN) + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
-      for (int h = 0; h < BN / 64; ++h) {
+      for (int h = h0; h < h1; ++h) {
         float va[32], vb[32];  // both 32-column loads of the half in flight before one wait
         tmem_ld32_issue(acc + (uint32_t)(h * 64), va);
         tmem_ld32_issue(acc + (uint32_t)(h * 64 + 32), vb);
         tmem_ld_wait(va, vb);
-        if (h == BN / 64 - 1) {  // the accumulator is in registers: the MMA warp may refill it
+        if (h == h1 - 1) {  // this warp's share of the accumulator is in registers: the MMA warp may refill it
           tc_fence_before();
           __syncwarp();
           if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acc_empty(b)) : "memory");
         }
-        if (RES && h == 0) {  // single staging tile: this warp's previous store must have finished reading it
+        if (RES && h == h0) {  // single staging tile: this warp's previous store must have finished reading it
           if (lane == 0 && pending) {
             asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             pending = false;
@@ -784,7 +788,7 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
             for (int e = 0; e < 8; ++e) o.v[e] = apply_act(v[gq * 8 + e], p.act);
             o.store(reinterpret_cast<bf16*>(io + off));
           }
-          if (!RES && h == 0 && sub == 0 && lane == 0 && pending) {
+          if (!RES && h == h0 && sub == 0 && lane == 0 && pending) {
             // One chunk into tile j, this warp's store of tile j - 1 has long finished reading its staging tile:
             // confirm it (no stall in the steady state); it licenses the next iteration to overwrite that tile.
             asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -800,8 +804,7 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
       __syncwarp();
       if (lane == 0) {
         if (m0 + q * 32 < p.M) {
-#pragma unroll
-          for (int h = 0; h < BN / 64; ++h)
+          for (int h = h0; h < h1; ++h)
             if (n0 + h * 64 < p.N) tma_store_2d(&tmO, io_s + h * 16384 + q * 4096, n0 + h * 64, m0 + q * 32);
         }
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");  // possibly empty: keeps the bookkeeping uniform
@@ -1038,7 +1041,7 @@ inline cudaError_t tc_launch_persistent(int ctas, cudaStream_t st, const CUtenso
                                         const CUtensorMap& o, const TcParams& p) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(ctas);
-  cfg.blockDim = dim3(kTcThreads);
+  cfg.blockDim = dim3(TcPersistSmem<BN, RES>::kThreads);
   cfg.dynamicSmemBytes = TcPersistSmem<BN, RES>::kBytes;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
