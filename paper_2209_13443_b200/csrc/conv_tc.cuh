@@ -7,12 +7,14 @@
 // K block, zero fill for the padding halo), or reads it as a plain 2-D tile for 1x1 stride-1
 // layers.  Batching appends samples along M, so one weight tile serves every sample of the batch.
 //
-// One CTA computes one 128 x BN output tile.  Warp roles: warp 0 issues TMA loads into a ring of
-// shared-memory stages, warp 1 owns the TMEM allocation and issues the MMAs (one thread), warps
-// 2-5 run the epilogue: tcgen05.ld of the fp32 accumulator, folded-BN scale/bias, residual add (the
-// residual tile was brought into shared memory by TMA while the main loop ran), activation, one
-// rounding to bf16, then a TMA store of the tile from shared memory.  The K loop visits (tap, channel block) in a
-// fixed order that does not depend on the batch size.
+// One CTA computes one 128 x BN output tile (or, in the persistent variant, walks many).  Warp roles: warp 0 issues
+// TMA loads into a ring of shared-memory slots, warp 1 owns the TMEM allocation and issues the MMAs (one thread),
+// the remaining warps run the epilogue: tcgen05.ld of the fp32 accumulator, folded-BN scale/bias, residual add (the
+// residual tile was brought into shared memory by TMA while the main loop ran), activation, one rounding to bf16,
+// then a TMA store of the tile from shared memory.  The K loop visits (tap, channel block) in a fixed order that
+// does not depend on the batch size.  Variants (chosen per launch from the grid size, see tc_launch): shallow or
+// deep ring, cluster split-K with a reduce-scatter through distributed shared memory, gather-mode A operand for
+// 3-channel stems, and a persistent kernel with double-buffered TMEM accumulators for multi-wave 1x1 layers.
 //
 // Every wait on an mbarrier is bounded by a clock: on expiry the thread records EE_ERR_TIMEOUT in
 // the model's error word and falls through to the common exit, which frees the TMEM columns.
@@ -226,8 +228,6 @@ __device__ __forceinline__ void gather_rows_static(const TcParams& p, const bf16
       __align__(16) bf16 v[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
-        constexpr int dummy = 0;
-        (void)dummy;
         const int k = i * kTcBK + c * 8 + e;
         const int rf = k / RUNP, j = k % RUNP;     // compile-time after unrolling
         if (rf < KH && j < RUN) {
