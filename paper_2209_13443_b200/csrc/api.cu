@@ -9,6 +9,7 @@
 #include "common.cuh"
 #include "conv_simt.cuh"
 #include "conv_tc.cuh"
+#include "conv_stem.cuh"
 #include "head.cuh"
 
 using namespace ee;
@@ -170,7 +171,8 @@ ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const
     }
     case KK_TC_GATHER: {
       if constexpr (sizeof(T) == 2) {
-        ee_status_t s = tc_launch(m->tc, L.tc, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st);
+        ee_status_t s = L.tc.stem7 ? stem_launch(m->tc, L.tc, src, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st)
+                                   : tc_launch(m->tc, L.tc, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st);
         if (s != EE_OK) return s;
       } else {
         return EE_ERR_INTERNAL;
@@ -363,6 +365,7 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
     if (cudaMemsetAsync(p, 0, 256, st) != cudaSuccess) return fail(EE_ERR_CUDA);
   }
   rc = tc_context_init(m->tc);
+  if (rc == EE_OK) rc = stem_context_init();
   if (rc != EE_OK) return fail(rc);
 
   int h = desc->in_h, w = desc->in_w, c = desc->in_c;
@@ -491,19 +494,24 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
       } else if (desc->dtype == EE_BF16 && d.cout % 8 == 0 && d.kh * d.kw * d.cin <= 1024) {
         // pixel rows are not 16-byte units (e.g. a 3-channel stem): explicit Toeplitz rows, then the tensor-core GEMM
         L.kind = KK_TC_GATHER;
+        const bool stem7 = stem_supported(d, L.in_h, L.in_w, L.out_w) && d.residual_from == EE_NO_RESIDUAL;
         const int run = d.kw * d.cin;
         const int runp = cdiv(run, 8) * 8;
         const int kp = cdiv(d.kh * runp, kTcBK) * kTcBK;
         void* wp = nullptr;
         if (cudaMalloc(&wp, (size_t)d.cout * kp * 2) != cudaSuccess) return fail(EE_ERR_CUDA);
         m->owned.push_back(wp);
-        pack_weights_kernel<<<cdiv((long)d.cout * kp, 256), 256, 0, st>>>((const bf16*)L.w_dev, (bf16*)wp, d.cout, d.kh, run, runp, kp);
+        if (stem7)
+          pack_stem_weights_kernel<<<cdiv((long)d.cout * kp, 256), 256, 0, st>>>((const bf16*)L.w_dev, (bf16*)wp, d.cout);
+        else
+          pack_weights_kernel<<<cdiv((long)d.cout * kp, 256), 256, 0, st>>>((const bf16*)L.w_dev, (bf16*)wp, d.cout, d.kh, run, runp, kp);
         if (cudaGetLastError() != cudaSuccess) return fail(EE_ERR_CUDA);
         ee_layer_desc_t g = d;   // the GEMM view: a 1x1 layer over kp packed columns
         g.cin = kp, g.kh = g.kw = 1, g.stride = 1, g.pad = 0;
         rc = tc_plan_layer(m->tc, g, L.out_h, L.out_w, L.out_h, L.out_w, desc->max_batch, wp, &L.tc);
         if (rc != EE_OK) return fail(rc);
         L.tc.gather = true;
+        L.tc.stem7 = stem7;
         L.tc.splits = 1, L.tc.kb_per = kp / kTcBK;
         L.tc.g_h = L.in_h, L.tc.g_w = L.in_w, L.tc.g_cin = d.cin, L.tc.g_kh = d.kh, L.tc.g_kw = d.kw;
         L.tc.g_stride = d.stride, L.tc.g_pad = d.pad, L.tc.g_runp = runp;

@@ -855,12 +855,13 @@ struct TcLayer {
   int splits = 1, kb_per = 0;    // split-K ranges of this layer (fixed per layer, independent of the batch)
   // gather mode: geometry of the real convolution (cin/kh/... above then describe the packed 1x1 GEMM view)
   bool gather = false;
+  bool stem7 = false;   // the 7x7/2 stem kernel of conv_stem.cuh takes this layer
   int g_h = 0, g_w = 0, g_cin = 0, g_kh = 0, g_kw = 0, g_stride = 1, g_pad = 0, g_runp = 0;
   CUtensorMap tm_w;
   struct Cached {
     const void* ptr;
     int batch;
-    int kind;  // 0: operand A, 1: residual / output matrix
+    int kind;  // 0: operand A, 1: residual / output matrix, 2: stem input rows, 3: stem output rows
     CUtensorMap tm;
   };
   mutable std::vector<Cached> a_maps;  // tensor maps of caller buffers by (pointer, batch, kind)
@@ -966,7 +967,25 @@ inline ee_status_t tc_buffer_map(const TcContext& c, const TcLayer& L, const voi
   e.batch = batch;
   e.kind = kind;
   CUresult r;
-  if (kind == 1) {
+  if (kind == 2) {
+    // stem input as (W*Cin, H, B): one 256-element piece of an image row per load, zero fill outside
+    const cuuint64_t dims[3] = {(cuuint64_t)L.g_w * L.g_cin, (cuuint64_t)L.g_h, (cuuint64_t)batch};
+    const cuuint64_t strides[2] = {(cuuint64_t)L.g_w * L.g_cin * 2, (cuuint64_t)L.g_w * L.g_cin * 2 * L.g_h};
+    const cuuint32_t box[3] = {256, 1, 1};
+    const cuuint32_t es[3] = {1, 1, 1};
+    r = c.encode_tiled(&e.tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else if (kind == 3) {
+    // stem output as (Cout, Wo, B*Ho): a tile is one output row, pixels past Wo are clipped
+    const cuuint64_t dims[3] = {(cuuint64_t)L.cout, (cuuint64_t)L.out_w, (cuuint64_t)batch * L.out_h};
+    const cuuint64_t strides[2] = {(cuuint64_t)L.cout * 2, (cuuint64_t)L.cout * 2 * L.out_w};
+    const cuuint32_t box[3] = {64, 32, 1};
+    const cuuint32_t es[3] = {1, 1, 1};
+    r = c.encode_tiled(&e.tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else if (kind == 1) {
     const cuuint64_t dims[2] = {(cuuint64_t)L.cout, (cuuint64_t)batch * L.out_h * L.out_w};
     const cuuint64_t strides[1] = {(cuuint64_t)L.cout * 2};
     const cuuint32_t box[2] = {64, 32};
