@@ -304,6 +304,14 @@ def run_ours(args):
                     pl = per_layer.setdefault((s, i), {"kernel": name, "m": plan[i]["m"], "n": plan[i]["n"], "k": plan[i]["k"],
                                                        "ms": 0.0, "flops": plan[i]["flops"], "bytes": plan[i]["bytes"]})
                     pl["ms"] += ms / K
+                else:   # head and compaction kernels of the stage follow its layers
+                    info_s = model.query(s)
+                    es_ = 2 if spec.dtype == "bf16" else 4
+                    byt = {"head_gap": n * info_s["out_bytes_per_sample"],
+                           "head_fc_softmax_scan": info_s["out_c"] * spec.stages[s].n_classes * es_ + n * info_s["out_c"] * 4}.get(name, 0)
+                    pl = per_layer.setdefault((s, i), {"kernel": name, "m": n, "n": spec.stages[s].n_classes, "k": info_s["out_c"],
+                                                       "ms": 0.0, "flops": 0.0, "bytes": float(byt)})
+                    pl["ms"] += ms / K
             info = model.query(s)
             ns = int(bufs[s].n_surv_host[0])
             es = 2 if spec.dtype == "bf16" else 4

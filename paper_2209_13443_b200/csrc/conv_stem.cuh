@@ -11,8 +11,8 @@
 //
 // K layout: K = 7 runs (filter rows) of 24 columns: column 0 is a dummy, columns 1..21 are the kw*Cin = 21 taps of
 // the filter row (contiguous in NHWC), columns 22..23 are padding; 168 columns padded to three K blocks of 64.  The
-// dummy column makes every run start on a 4-byte boundary of the patch: with 16 elements of lead-in before the
-// image row, pixel ox starts at element 6 ox + 6.  Weights are packed the same way, with zeros in the dummy and
+// dummy column makes every run start on a 4-byte boundary of the patch: the run of pixel ox begins at element
+// 6 ox - 10 of the image row, and the patch boxes begin at multiples of 8 elements (16 before the row for the first).  Weights are packed the same way, with zeros in the dummy and
 // padding columns; the gather warps zero those columns of A as well, so nothing but real taps enters a sum.
 #pragma once
 #include "conv_tc.cuh"
@@ -32,12 +32,18 @@ constexpr int kStemThreads = 320;      // producer, MMA, 4 gather warps, 4 epilo
 constexpr int kStemKh = 7, kStemKw = 7, kStemCin = 3, kStemStride = 2, kStemPad = 3;
 constexpr int kStemRunWords = 12;      // 24 bf16 columns per filter row
 constexpr int kStemLead = 16;          // zero elements in front of each patch row (a TMA load may start at x = -16)
-constexpr int kStemRowElems = 768;     // three 256-element TMA boxes per patch row
-constexpr int kStemRowBytes = kStemRowElems * 2;
-constexpr int kStemPatchBytes = kStemKh * kStemRowBytes;
+// The patch is three TMA boxes of 7 rows x 256 elements whose first columns sit kStemBoxStep elements apart: they
+// overlap by 32 elements, more than one pixel's 24-column run, so every pixel finds its whole run inside one box
+// and addresses it with constant offsets.
+constexpr int kStemBoxElems = 256, kStemBoxes = 3, kStemBoxStep = 224;
+constexpr int kStemBoxRowBytes = kStemBoxElems * 2;
+constexpr int kStemBoxBytes = kStemKh * kStemBoxRowBytes;
+constexpr int kStemPatchBytes = kStemBoxes * kStemBoxBytes;
 constexpr int kStemKBlocks = 3;
-// last word a pixel reads: 3 (Wo - 1) + 3 + 10 must stay inside the row
-constexpr int kStemMaxWo = (kStemRowElems / 2 - 14) / 3 + 1 > 128 ? 128 : (kStemRowElems / 2 - 14) / 3 + 1;
+// image elements (before the lead-in shift) the boxes cover: [-kStemLead, kStemCover)
+constexpr int kStemCover = (kStemBoxes - 1) * kStemBoxStep + kStemBoxElems - kStemLead;
+// the run of pixel ox spans elements [6 ox - 10, 6 ox + 13] of the image row
+constexpr int kStemMaxWo = (kStemCover - 14) / (kStemStride * kStemCin) + 1;
 
 struct StemSmem {
   static constexpr int kABytes = kTcBM * kTcBK * 2;        // one K block of A
@@ -59,7 +65,7 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t src
                : "memory");
 }
 
-// tmX: input as (W*3, H, B) with a 256 x 1 x 1 box, no swizzle; tmW: packed weights (192, 1, Cout) with a 64 x 1 x 64
+// tmX: input as (W*3, H, B) with a 256 x 7 x 1 box, no swizzle; tmW: packed weights (192, 1, Cout) with a 64 x 1 x 64
 // box, 128-byte swizzle; tmO: output as (Cout, Wo, B*Ho) with a 64 x 32 x 1 box, 128-byte swizzle, so that pixels past
 // Wo are clipped by the TMA unit.
 __global__ void __launch_bounds__(kStemThreads, 2)
@@ -127,10 +133,8 @@ conv_stem7x7_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
         mbar_expect_tx(patch_full(b), kStemPatchBytes);
         const uint32_t dst = base + S::kPatchOff + b * kStemPatchBytes;
 #pragma unroll
-        for (int r = 0; r < kStemKh; ++r)
-#pragma unroll
-          for (int c = 0; c < 3; ++c)   // rows outside the image and columns outside the row arrive as zeros
-            tma_load_3d(dst + r * kStemRowBytes + c * 512, &tmX, patch_full(b), c * 256 - kStemLead, oy * kStemStride - kStemPad + r, n);
+        for (int c = 0; c < kStemBoxes; ++c)   // rows outside the image and columns outside the row arrive as zeros
+          tma_load_3d(dst + c * kStemBoxBytes, &tmX, patch_full(b), c * kStemBoxStep - kStemLead, oy * kStemStride - kStemPad, n);
       }
     }
   } else if (warp == 1) {
@@ -162,7 +166,13 @@ conv_stem7x7_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
     // gather warps: thread r builds row r (output pixel ox = r) of every K block of A
     const int r = (int)threadIdx.x - 64;
     const int ox = min(r, p.Wo - 1);   // rows past Wo repeat the last pixel; the store clips them
-    const uint32_t* prow = reinterpret_cast<const uint32_t*>(gen + S::kPatchOff) + (kStemStride * kStemCin * ox + (kStemLead - kStemPad * kStemCin - 1)) / 2;
+    const int e0 = kStemStride * kStemCin * ox - kStemPad * kStemCin - 1;   // image-row element of column 0 of the run (even)
+    int box = 0;                                                            // first box that holds the whole run
+#pragma unroll
+    for (int c = 1; c < kStemBoxes; ++c)
+      if (e0 + 2 * kStemRunWords - 1 > (c - 1) * kStemBoxStep - kStemLead + kStemBoxElems - 1) box = c;
+    const uint32_t* prow =
+        reinterpret_cast<const uint32_t*>(gen + S::kPatchOff + box * kStemBoxBytes) + (e0 - (box * kStemBoxStep - kStemLead)) / 2;
     uint8_t* aline = gen + S::kAOff + r * 128;
     bool ok = true;
     for (int j = 0; j < my_tiles && ok; ++j) {
@@ -181,9 +191,9 @@ conv_stem7x7_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
           if (rf >= kStemKh || jw == kStemRunWords - 1)
             w[q] = 0u;                                          // K padding, columns 22..23
           else if (jw == 0)
-            w[q] = pw[rf * (kStemRowBytes / 4)] & 0xFFFF0000u;  // dummy column 0 | first tap
+            w[q] = pw[rf * (kStemBoxRowBytes / 4)] & 0xFFFF0000u;  // dummy column 0 | first tap
           else
-            w[q] = pw[rf * (kStemRowBytes / 4) + jw];
+            w[q] = pw[rf * (kStemBoxRowBytes / 4) + jw];
         }
         uint8_t* line = aline + i * S::kABytes;
 #pragma unroll
@@ -232,8 +242,7 @@ conv_stem7x7_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
 #pragma unroll
       for (int sub = 0; sub < 2; ++sub) {
         float* v = sub ? vb : va;
-#pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = fmaf(s_scale[sub * 32 + i], v[i], s_bias[sub * 32 + i]);
+        scale_bias<32>(v, s_scale + sub * 32, s_bias + sub * 32);
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           Vec16<bf16> o;
@@ -277,7 +286,7 @@ __global__ void pack_stem_weights_kernel(const bf16* __restrict__ w, bf16* __res
 inline bool stem_supported(const ee_layer_desc_t& d, int in_h, int in_w, int out_w) {
   (void)in_h;
   return d.op == EE_OP_CONV && d.cin == kStemCin && d.kh == kStemKh && d.kw == kStemKw && d.stride == kStemStride && d.pad == kStemPad &&
-         d.cout % 8 == 0 && d.cout <= 64 && in_w % 8 == 0 && in_w * kStemCin + kStemLead <= kStemRowElems && out_w <= kStemMaxWo;
+         d.cout % 8 == 0 && d.cout <= 64 && in_w % 8 == 0 && out_w <= kStemMaxWo;
 }
 
 inline ee_status_t stem_context_init() {

@@ -169,6 +169,22 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
       : "memory");
 }
 
+// v[i] = scale[i] * v[i] + bias[i] over N columns (a multiple of 4).  scale and bias are 16-byte aligned rows in shared
+// memory that every lane reads at the same address: as float4 a load is one broadcast wavefront for four columns.
+template <int N>
+__device__ __forceinline__ void scale_bias(float* v, const float* scale, const float* bias) {
+  const float4* s4 = reinterpret_cast<const float4*>(scale);
+  const float4* b4 = reinterpret_cast<const float4*>(bias);
+#pragma unroll
+  for (int i = 0; i < N / 4; ++i) {
+    const float4 s = s4[i], b = b4[i];
+    v[4 * i] = fmaf(s.x, v[4 * i], b.x);
+    v[4 * i + 1] = fmaf(s.y, v[4 * i + 1], b.y);
+    v[4 * i + 2] = fmaf(s.z, v[4 * i + 2], b.z);
+    v[4 * i + 3] = fmaf(s.w, v[4 * i + 3], b.w);
+  }
+}
+
 // ----------------------------------------------------------------------------- kernel
 
 // Gather-mode row builders (see the GATHER note on the kernel).  Thread `grow` writes row `grow` of the A tile of
@@ -464,8 +480,7 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
           const int c0 = h * 64 + sub * 32;
           float v[32];
           tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = fmaf(s_scale[c0 + j], v[j], s_bias[c0 + j]);
+          scale_bias<32>(v, s_scale + c0, s_bias + c0);
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
             bf16* chunk = reinterpret_cast<bf16*>(line + (((sub * 4 + g) ^ (lane & 7)) << 4));
@@ -531,8 +546,7 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
           }
         }
         if (m < p.M && n < p.N) {
-#pragma unroll
-          for (int e = 0; e < 8; ++e) v[e] = fmaf(s_scale[g * 8 + e], v[e], s_bias[g * 8 + e]);
+          scale_bias<8>(v, s_scale + g * 8, s_bias + g * 8);
           if (p.residual) {
             Vec16<bf16> rr;
             rr.load(p.residual + (size_t)m * p.N + n);
@@ -772,8 +786,7 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
         for (int sub = 0; sub < 2; ++sub) {
           const int c0 = h * 64 + sub * 32;
           float* v = sub ? vb : va;
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = fmaf(sc[c0 + i], v[i], sc[BN + c0 + i]);
+          scale_bias<32>(v, sc + c0, sc + BN + c0);
 #pragma unroll
           for (int gq = 0; gq < 4; ++gq) {
             const int off = h * 16384 + row * 128 + (((sub * 4 + gq) ^ (lane & 7)) << 4);
@@ -968,10 +981,10 @@ inline ee_status_t tc_buffer_map(const TcContext& c, const TcLayer& L, const voi
   e.kind = kind;
   CUresult r;
   if (kind == 2) {
-    // stem input as (W*Cin, H, B): one 256-element piece of an image row per load, zero fill outside
+    // stem input as (W*Cin, H, B): 256 elements of 7 consecutive image rows per load, zero fill outside
     const cuuint64_t dims[3] = {(cuuint64_t)L.g_w * L.g_cin, (cuuint64_t)L.g_h, (cuuint64_t)batch};
     const cuuint64_t strides[2] = {(cuuint64_t)L.g_w * L.g_cin * 2, (cuuint64_t)L.g_w * L.g_cin * 2 * L.g_h};
-    const cuuint32_t box[3] = {256, 1, 1};
+    const cuuint32_t box[3] = {256, 7, 1};
     const cuuint32_t es[3] = {1, 1, 1};
     r = c.encode_tiled(&e.tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
