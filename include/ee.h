@@ -188,11 +188,11 @@ size_t ee_exit_head_scratch_bytes(const ee_model_t* model, int stage);
  * decision: code living inside a host application that hands out all device memory at start-up and forbids
  * later cudaMalloc calls (inference-server plug-ins, engines running under a fixed memory budget), and latency-bound
  * serving threads, for which an allocation's implicit synchronisation and unpredictable duration are not
- * acceptable.  Same arguments, results and errors as ee_exit_head, minus `scratch`: the partial sums, pooled vectors,
+ * acceptable.  Same arguments, results and errors as ee_exit_head, minus `scratch`: the pooled vectors,
  * logits (when out->logits is NULL) and counters go to an array of EE_STATIC_HEAD_SCRATCH_BYTES bytes that is part of
  * the library image (each GPU that loads the library holds it until the process exits).
  *   - A model/shape whose head needs more than EE_STATIC_HEAD_SCRATCH_BYTES (what ee_exit_head_scratch_bytes reports
- *     for the stage's own hw) is refused with EE_ERR_CAPACITY and an explanatory ee_last_cuda_error() text.
+ *     for the stage) is refused with EE_ERR_CAPACITY and an explanatory ee_last_cuda_error() text.
  *   - The first call on a device resolves the array's device address (the calling thread's current device must be the
  *     one the model lives on); make that first call outside any stream capture.
  *   - No cudaMalloc / cudaFree or allocating library routine is called.

@@ -80,35 +80,38 @@ struct StagePlan {
 
 size_t esize(int dtype) { return dtype == EE_BF16 ? 2 : 4; }
 
-// Rows of a sample's [HW][C] map summed by one CTA of the pooling kernel: a function of the
-// shape only (never of the batch), about 32 KB of input per CTA.
-int gap_rows_per_chunk(int hw, int c, size_t es) {
-  long rows = (32 * 1024) / ((long)c * (long)es);
-  if (rows < 1) rows = 1;
-  if (rows > hw) rows = hw;
-  return (int)rows;
-}
-
 struct HeadLayout {
-  int rows_per_chunk, nchunks;
-  size_t off_partial, off_gap, off_z, off_cnt, bytes;
+  size_t off_gap, off_z, off_cnt, bytes;
 };
 
-HeadLayout head_layout(int max_batch, int hw, int c, int k, size_t es) {
+HeadLayout head_layout(int max_batch, int c, int k) {
   HeadLayout h;
-  h.rows_per_chunk = gap_rows_per_chunk(hw, c, es);
-  h.nchunks = cdiv(hw, h.rows_per_chunk);
   size_t o = 0;
   h.off_cnt = o;
-  o = align_up(o + sizeof(unsigned) * ((size_t)max_batch + 1), 256);  // per-sample pooling counters + the FC kernel's
-  h.off_partial = o;
-  o = align_up(o + sizeof(float) * (size_t)max_batch * h.nchunks * c, 256);
+  o = align_up(o + sizeof(unsigned) * ((size_t)max_batch + 1), 256);  // the FC kernel's per-tile counters, then its tile count
   h.off_gap = o;
   o = align_up(o + sizeof(float) * (size_t)max_batch * c, 256);
   h.off_z = o;
   o = align_up(o + sizeof(float) * (size_t)max_batch * k, 256);
   h.bytes = o;
   return h;
+}
+
+// Launch with programmatic stream serialization: the kernel may start while its predecessor in the stream drains
+// and calls griddepcontrol.wait before it touches that kernel's results.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
 }  // namespace
@@ -209,27 +212,27 @@ ee_status_t launch_head(ee_model* m, StagePlan& sp, const void* x, int B, int hw
                         const int32_t* shift_cls, char* scratch, const ee_stage_in_t* in_ids, const ee_stage_out_t* out,
                         cudaStream_t st, bool timed) {
   const int C = sp.out_c, K = sp.n_classes;
-  HeadLayout h = head_layout(m->max_batch, hw, C, K, sizeof(T));
+  HeadLayout h = head_layout(m->max_batch, C, K);
   unsigned* cnt = (unsigned*)(scratch + h.off_cnt);
-  float* partial = (float*)(scratch + h.off_partial);
   float* gap = (float*)(scratch + h.off_gap);
   float* z = out->logits ? out->logits : (float*)(scratch + h.off_z);
   constexpr int V = Elem<T>::kVec;
-  EE_CUDA(cudaMemsetAsync(cnt, 0, sizeof(unsigned) * ((size_t)m->max_batch + 1), st));
-  dim3 ggrid(h.nchunks, B);
-  if (C % V == 0)
-    gap_kernel<T, V><<<ggrid, kGapThreads, 0, st>>>((const T*)x, hw, C, h.rows_per_chunk, partial, gap, cnt);
+  const bool vec = C % V == 0 && ((uintptr_t)x & 15) == 0;
+  const int lanes = gap_lanes(hw);
+  const int n_zero = m->max_batch + 1;   // the pooling kernel leaves the FC kernel's counters at zero
+  dim3 ggrid(cdiv(vec ? C / V : C, lanes), B);
+  if (vec)
+    EE_CUDA(launch_pdl(gap_kernel<T, V>, ggrid, dim3(kGapThreads), st, (const T*)x, hw, C, lanes, gap, cnt, n_zero));
   else
-    gap_kernel<T, 1><<<ggrid, kGapThreads, 0, st>>>((const T*)x, hw, C, h.rows_per_chunk, partial, gap, cnt);
-  EE_CUDA(cudaGetLastError());
+    EE_CUDA(launch_pdl(gap_kernel<T, 1>, ggrid, dim3(kGapThreads), st, (const T*)x, hw, C, lanes, gap, cnt, n_zero));
   if (timed) record(m, sp, st, "head_gap");
   DecideArgs da{shift, shift_cls, sp.threshold, sp.always_exit, out->conf, out->pred, out->exit_mask,
-                in_ids ? in_ids->ids : nullptr, out->survivor_idx, out->ids_out, out->n_surv_dev, cnt + m->max_batch};
-  if (C % V == 0)
-    fc_kernel<T, V><<<cdiv(K, kFcClasses), kFcWarps * 32, 0, st>>>(gap, (const T*)sp.fc_w, sp.fc_b, B, C, K, z, da);
+                in_ids ? in_ids->ids : nullptr, out->survivor_idx, out->ids_out, out->n_surv_dev, cnt, cnt + m->max_batch};
+  dim3 fgrid(cdiv(K, kFcClasses), cdiv(B, kFcSamples));
+  if (C % V == 0 && ((uintptr_t)sp.fc_w & 15) == 0)
+    EE_CUDA(launch_pdl(fc_kernel<T, true>, fgrid, dim3(kFcThreads), st, (const float*)gap, (const T*)sp.fc_w, (const float*)sp.fc_b, B, C, K, z, da));
   else
-    fc_kernel<T, 1><<<cdiv(K, kFcClasses), kFcWarps * 32, 0, st>>>(gap, (const T*)sp.fc_w, sp.fc_b, B, C, K, z, da);
-  EE_CUDA(cudaGetLastError());
+    EE_CUDA(launch_pdl(fc_kernel<T, false>, fgrid, dim3(kFcThreads), st, (const float*)gap, (const T*)sp.fc_w, (const float*)sp.fc_b, B, C, K, z, da));
   if (timed) record(m, sp, st, "head_fc_softmax_scan");
   return EE_OK;
 }
@@ -465,7 +468,7 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
     sp.out_h = oh[out_layer];
     sp.out_w = ow[out_layer];
     sp.out_c = oc[out_layer];
-    HeadLayout hl = head_layout(desc->max_batch, sp.out_h * sp.out_w, sp.out_c, sd.n_classes, es);
+    HeadLayout hl = head_layout(desc->max_batch, sp.out_c, sd.n_classes);
     sp.head_off = align_up(off, 1024);
     sp.head_bytes = hl.bytes;
     sp.ws_bytes = sp.head_off + hl.bytes;
@@ -667,8 +670,7 @@ ee_status_t ee_exit_head(ee_model_t* m, int stage, const void* x, int batch, int
     return EE_OK;
   }
   if (!x || !scratch || ((uintptr_t)scratch & 255)) return EE_ERR_INVALID_ARG;
-  // the pooling chunks follow hw, so the scratch need is re-derived for the hw given
-  HeadLayout hl = head_layout(m->max_batch, hw, sp.out_c, sp.n_classes, esize(m->dtype));
+  HeadLayout hl = head_layout(m->max_batch, sp.out_c, sp.n_classes);
   if (scratch_bytes < hl.bytes) return EE_ERR_CAPACITY;
   return m->dtype == EE_BF16
              ? launch_head<bf16>(m, sp, x, batch, hw, logit_shift, shift_class, (char*)scratch, nullptr, out, st, false)
@@ -691,7 +693,7 @@ ee_status_t ee_exit_head_static(ee_model_t* m, int stage, const void* x, int bat
   if (logit_shift && !shift_class) return EE_ERR_INVALID_ARG;
   StagePlan& sp = m->stages[stage];
   if (batch > m->max_batch) return EE_ERR_CAPACITY;
-  HeadLayout hl = head_layout(m->max_batch, hw, sp.out_c, sp.n_classes, esize(m->dtype));
+  HeadLayout hl = head_layout(m->max_batch, sp.out_c, sp.n_classes);
   if (hl.bytes > (size_t)EE_STATIC_HEAD_SCRATCH_BYTES) {
     g_cuda_err = "ee_exit_head_static: this model/shape needs " + std::to_string(hl.bytes) + " scratch bytes, the built-in array holds " +
                  std::to_string((size_t)EE_STATIC_HEAD_SCRATCH_BYTES);
@@ -713,7 +715,7 @@ ee_status_t ee_exit_head_static(ee_model_t* m, int stage, const void* x, int bat
   }
   if (!x) return EE_ERR_INVALID_ARG;
   char* scratch = (char*)g_static_head_ptr[dev];
-  // launch_head zeroes the per-sample counters it needs; everything else in the array is overwritten before it is read
+  // the pooling kernel zeroes the counters the FC kernel needs; everything else in the array is overwritten before it is read
   return m->dtype == EE_BF16
              ? launch_head<bf16>(m, sp, x, batch, hw, logit_shift, shift_class, scratch, nullptr, out, st, false)
              : launch_head<float>(m, sp, x, batch, hw, logit_shift, shift_class, scratch, nullptr, out, st, false);

@@ -17,84 +17,75 @@ namespace ee {
 
 constexpr int kGapThreads = 256;
 
-// Partial column sums of one sample's [HW][C] map over rows [chunk*rows_per_chunk, ...), written to
-// partial[b][chunk][C]; the last CTA to finish a sample adds the chunks in ascending order and
-// writes gap[b][c] = sum / HW.  counters[b] must be zero on entry and is zero again on exit.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// gap[b][c] = mean over the HW rows of sample b's [HW][C] map, in one pass.  A CTA owns one sample and a slab of
+// `lanes` channel vectors: its 256 threads form 256 / lanes row groups, group g adds rows g, g + groups, ... in
+// ascending order (eight loads in flight), then the first lanes * VEC threads add the group sums in ascending group
+// order.  `lanes` depends on the layer shape only (few rows: wide slabs; many rows: many row groups), so the
+// grouping of a sample's sum is the same in every batch.  Block (0, 0) also zeroes the n_zero counters that the
+// FC kernel behind it in the stream relies on.  Launched with programmatic stream serialization.
 template <typename T, int VEC>
 __global__ void __launch_bounds__(kGapThreads)
-gap_kernel(const T* __restrict__ x, int HW, int C, int rows_per_chunk, float* __restrict__ partial,
-           float* __restrict__ gap, unsigned* __restrict__ counters) {
+gap_kernel(const T* __restrict__ x, int HW, int C, int lanes, float* __restrict__ gap, unsigned* __restrict__ zero_me, int n_zero) {
   __shared__ float red[kGapThreads * VEC];
-  __shared__ bool is_last;
-  const int tid = threadIdx.x, b = blockIdx.y, chunk = blockIdx.x, nchunks = gridDim.x;
+  const int tid = threadIdx.x, b = blockIdx.y;
   const int cv = C / VEC;
-  const int per = cv < kGapThreads ? cv : kGapThreads;
-  const int groups = kGapThreads / per;
-  const int grp = tid / per, lv = tid - grp * per;
-  const bool active = grp < groups;
-  const int r0 = chunk * rows_per_chunk;
-  const int r1 = min(HW, r0 + rows_per_chunk);
-  const T* xb = x + (size_t)b * HW * C;
-  float* pout = partial + ((size_t)b * nchunks + chunk) * C;
-  for (int vb = 0; vb < cv; vb += per) {
-    const int v = vb + lv;
-    float acc[VEC];
+  const int groups = kGapThreads / lanes;
+  const int grp = tid / lanes, lv = tid - grp * lanes;
+  const int v = blockIdx.x * lanes + lv;
+  pdl_wait();
+  pdl_launch_dependents();
+  if (blockIdx.x == 0 && blockIdx.y == 0)
+    for (int i = tid; i < n_zero; i += kGapThreads) zero_me[i] = 0u;
+  float acc[VEC];
 #pragma unroll
-    for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
-    if (active && v < cv) {
-      const T* p0 = xb + (size_t)v * VEC;
-      int r = r0 + grp;
+  for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+  if (v < cv) {
+    const T* p0 = x + (size_t)b * HW * C + (size_t)v * VEC;
+    int r = grp;
+    if constexpr (VEC > 1) {
+      for (; r + 7 * groups < HW; r += 8 * groups) {
+        Vec16<T> t[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) t[u].load(p0 + (size_t)(r + u * groups) * C);
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+#pragma unroll
+          for (int e = 0; e < VEC; ++e) acc[e] += t[u].v[e];
+      }
+    }
+    for (; r < HW; r += groups) {
+      const T* p = p0 + (size_t)r * C;
       if constexpr (VEC > 1) {
-        // four independent 16-byte loads in flight; the additions keep the ascending row order
-        for (; r + 3 * groups < r1; r += 4 * groups) {
-          Vec16<T> t0, t1, t2, t3;
-          t0.load(p0 + (size_t)r * C);
-          t1.load(p0 + (size_t)(r + groups) * C);
-          t2.load(p0 + (size_t)(r + 2 * groups) * C);
-          t3.load(p0 + (size_t)(r + 3 * groups) * C);
+        Vec16<T> t;
+        t.load(p);
 #pragma unroll
-          for (int e = 0; e < VEC; ++e) acc[e] = (((acc[e] + t0.v[e]) + t1.v[e]) + t2.v[e]) + t3.v[e];
-        }
-      }
-      for (; r < r1; r += groups) {
-        const T* p = p0 + (size_t)r * C;
-        if constexpr (VEC > 1) {
-          Vec16<T> t;
-          t.load(p);
-#pragma unroll
-          for (int e = 0; e < VEC; ++e) acc[e] += t.v[e];
-        } else {
-          acc[0] += Elem<T>::ld(p);
-        }
-      }
-#pragma unroll
-      for (int e = 0; e < VEC; ++e) red[(grp * per + lv) * VEC + e] = acc[e];
-    }
-    __syncthreads();
-    if (grp == 0 && v < cv) {
-#pragma unroll
-      for (int e = 0; e < VEC; ++e) {
-        float s = 0.f;
-        for (int q = 0; q < groups; ++q) s += red[(q * per + lv) * VEC + e];
-        pout[v * VEC + e] = s;
+        for (int e = 0; e < VEC; ++e) acc[e] += t.v[e];
+      } else {
+        acc[0] += Elem<T>::ld(p);
       }
     }
-    __syncthreads();
   }
-  __threadfence();
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) red[(grp * lanes + lv) * VEC + e] = acc[e];
   __syncthreads();
-  if (tid == 0) is_last = atomicAdd(&counters[b], 1u) == (unsigned)(nchunks - 1);
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-  const float inv = 1.0f / (float)HW;
-  const float* pb = partial + (size_t)b * nchunks * C;
-  for (int c = tid; c < C; c += kGapThreads) {
-    float s = 0.f;
-    for (int q = 0; q < nchunks; ++q) s += __ldcg(pb + (size_t)q * C + c);
-    gap[(size_t)b * C + c] = s * inv;
+  if (tid < lanes * VEC) {
+    const int c = blockIdx.x * lanes * VEC + tid;   // red[q][lv][e] with lv * VEC + e == tid
+    if (c < cv * VEC) {
+      float sum = 0.f;
+      for (int q = 0; q < groups; ++q) sum += red[q * lanes * VEC + tid];
+      gap[(size_t)b * C + c] = sum * (1.0f / (float)HW);
+    }
   }
-  if (tid == 0) counters[b] = 0;
+}
+
+// Channel vectors per CTA of gap_kernel for a [HW][C] map: about 16 rows per thread, between 8 and 64 row groups.
+inline int gap_lanes(int hw) {
+  int groups = 8;
+  while (groups < 64 && groups * 16 < hw) groups *= 2;
+  return kGapThreads / groups;
 }
 
 struct DecideArgs {  // everything the exit decision needs besides the logits
@@ -109,156 +100,35 @@ struct DecideArgs {  // everything the exit decision needs besides the logits
   int32_t* surv_idx;
   int32_t* ids_out;
   int32_t* n_surv;
-  unsigned* done;  // CTAs of the FC kernel that have written their logits; zero between launches
+  unsigned* tile_done;  // per sample tile: CTAs of the FC kernel that have written its logits; zero between launches
+  unsigned* done;       // sample tiles whose exit decisions are written; zero between launches
 };
 
-template <int THREADS>
-__device__ __forceinline__ void exit_decide_block(float* z, int B, int K, const float* __restrict__ shift,
-                                                  const int32_t* __restrict__ shift_cls, float thr, int always_exit,
-                                                  float* __restrict__ conf, int32_t* __restrict__ pred, uint8_t* mask,
-                                                  const int32_t* __restrict__ ids, int32_t* __restrict__ surv_idx,
-                                                  int32_t* __restrict__ ids_out, int32_t* __restrict__ n_surv);
-
-constexpr int kFcWarps = 8, kFcClassesPerWarp = 2, kFcSamples = 16, kFcChunk = 256;
-constexpr int kFcClasses = kFcWarps * kFcClassesPerWarp;
-
-// z[b][k] = bfc[k] + sum_c wfc[k][c] * gap[b][c].  A CTA owns 16 classes (two per warp) and walks the samples in
-// tiles of 16; the tile's pooled vectors are staged in shared memory 256 channels at a time, so the pooled matrix
-// crosses L2 once per CTA.  Per (b, k): every lane adds its channels in ascending order, then a shuffle tree;
-// the order does not depend on the batch size.  The CTA that finishes last (a counter, no waiting) goes on to the
-// exit decision for the whole batch: softmax top-1, threshold, stable scan of the survivors.
-template <typename T, int VEC>
-__global__ void __launch_bounds__(kFcWarps * 32)
-fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float* __restrict__ bfc, int B, int C, int K,
-          float* z, DecideArgs d) {
-  __shared__ __align__(16) float gs[kFcSamples][kFcChunk];
-  __shared__ bool last_cta;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int k0 = blockIdx.x * kFcClasses + warp * kFcClassesPerWarp;
-  constexpr int PER = kFcChunk / 32;                              // channels per lane per chunk (8)
-  constexpr int STG = kFcSamples * kFcChunk / (kFcWarps * 32);    // staged floats per thread per step (16)
-  const int nchunk = (C + kFcChunk - 1) / kFcChunk;
-  const int nstep = ((B + kFcSamples - 1) / kFcSamples) * nchunk; // (sample tile, channel chunk) pairs, tile-major
-
-  // One step ahead in registers: the pooled values this thread stages and the weight vectors of its two classes, so
-  // that the global-load latency of step i + 1 hides behind the arithmetic of step i.
-  float pre[STG];
-  float wnext[kFcClassesPerWarp][PER];
-  auto fetch = [&](int step) {
-    const int b0 = (step / nchunk) * kFcSamples, c0 = (step % nchunk) * kFcChunk;
-#pragma unroll
-    for (int u = 0; u < STG; ++u) {
-      const int i = threadIdx.x + u * (kFcWarps * 32);
-      const int sidx = i / kFcChunk, c = i - sidx * kFcChunk;
-      pre[u] = (b0 + sidx < B && c0 + c < C) ? gap[(size_t)(b0 + sidx) * C + c0 + c] : 0.f;
-    }
-    const int c = c0 + lane * PER;
-#pragma unroll
-    for (int q = 0; q < kFcClassesPerWarp; ++q) {
-      const int k = k0 + q;
-#pragma unroll
-      for (int e = 0; e < PER; ++e) wnext[q][e] = 0.f;
-      if (k < K) {
-        if constexpr (VEC == 8) {
-          if (c + PER <= C) {
-            Vec16<T> t;
-            t.load(wfc + (size_t)k * C + c);
-#pragma unroll
-            for (int e = 0; e < PER; ++e) wnext[q][e] = t.v[e];
-          }
-        } else {
-#pragma unroll
-          for (int e = 0; e < PER; ++e)
-            if (c + e < C) wnext[q][e] = Elem<T>::ld(wfc + (size_t)k * C + c + e);
-        }
-      }
-    }
-  };
-  float acc[kFcClassesPerWarp][kFcSamples];
-  if (nstep > 0) fetch(0);
-  for (int step = 0; step < nstep; ++step) {
-    const int b0 = (step / nchunk) * kFcSamples, ci = step % nchunk;
-    if (ci == 0) {
-#pragma unroll
-      for (int q = 0; q < kFcClassesPerWarp; ++q)
-#pragma unroll
-        for (int s2 = 0; s2 < kFcSamples; ++s2) acc[q][s2] = 0.f;
-    }
-    __syncthreads();  // everyone is done reading the previous step's tile
-#pragma unroll
-    for (int u = 0; u < STG; ++u) {
-      const int i = threadIdx.x + u * (kFcWarps * 32);
-      (&gs[0][0])[i] = pre[u];
-    }
-    float wv[kFcClassesPerWarp][PER];
-#pragma unroll
-    for (int q = 0; q < kFcClassesPerWarp; ++q)
-#pragma unroll
-      for (int e = 0; e < PER; ++e) wv[q][e] = wnext[q][e];
-    __syncthreads();
-    if (step + 1 < nstep) fetch(step + 1);
-#pragma unroll
-    for (int s2 = 0; s2 < kFcSamples; ++s2) {
-      const float4 g0 = *reinterpret_cast<const float4*>(&gs[s2][lane * PER]);
-      const float4 g1 = *reinterpret_cast<const float4*>(&gs[s2][lane * PER + 4]);
-      const float gv[PER] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-#pragma unroll
-      for (int q = 0; q < kFcClassesPerWarp; ++q)
-#pragma unroll
-        for (int e = 0; e < PER; ++e) acc[q][s2] = fmaf(wv[q][e], gv[e], acc[q][s2]);
-    }
-    if (ci == nchunk - 1) {
-#pragma unroll
-      for (int q = 0; q < kFcClassesPerWarp; ++q) {
-        const int k = k0 + q;
-        const float bk = (bfc && k < K) ? bfc[k] : 0.f;
-#pragma unroll
-        for (int s2 = 0; s2 < kFcSamples; ++s2) {
-          float v = acc[q][s2];
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-          if (lane == 0 && k < K && b0 + s2 < B) z[(size_t)(b0 + s2) * K + k] = v + bk;
-        }
-      }
-    }
-  }
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) last_cta = atomicAdd(d.done, 1u) == gridDim.x - 1;
-  __syncthreads();
-  if (!last_cta) return;
-  __threadfence();
-  if (threadIdx.x == 0) *d.done = 0;
-  exit_decide_block<kFcWarps * 32>(z, B, K, d.shift, d.shift_cls, d.thr, d.always_exit, d.conf, d.pred, d.mask, d.ids, d.surv_idx,
-                                   d.ids_out, d.n_surv);
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, int src_bytes) {  // bytes past src_bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc), "r"(src_bytes)
+               : "memory");
 }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-constexpr int kDecideThreads = 1024;
-
-// One CTA.  Per sample (one warp each): optional logit shift, max / lowest argmax, conf = 1 / sum exp(z - max),
-// exit = always || conf >= thr (NaN never exits).  Then a ballot + prefix-sum scan over the not-exit flags
-// gives the ascending survivor list, the survivors' ids and their count.
-template <int THREADS>
-__device__ __forceinline__ void exit_decide_block(float* z, int B, int K, const float* __restrict__ shift,
-                                                  const int32_t* __restrict__ shift_cls, float thr, int always_exit,
-                                                  float* __restrict__ conf, int32_t* __restrict__ pred, uint8_t* mask,
-                                                  const int32_t* __restrict__ ids, int32_t* __restrict__ surv_idx,
-                                                  int32_t* __restrict__ ids_out, int32_t* __restrict__ n_surv) {
-  __shared__ int warp_tot[32];
-  __shared__ int pass_total;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+// Exit decision of samples [b_lo, b_hi), one warp per sample (warp w of nwarps takes b_lo + w, b_lo + w + nwarps, ...):
+// optional logit shift, max / lowest argmax, conf = 1 / sum exp(z - max), exit = always || conf >= thr (NaN never
+// exits).  The logits may have been written by other CTAs and are read through L2.
+__device__ __forceinline__ void exit_decide_samples(float* z, int b_lo, int b_hi, int K, int warp, int nwarps, const DecideArgs& d) {
+  const int lane = threadIdx.x & 31;
   constexpr int kRegs = 32;  // logits per lane held in registers: one pass over memory for K <= 1024
-  for (int b = warp; b < B; b += THREADS / 32) {
+  for (int b = b_lo + warp; b < b_hi; b += nwarps) {
     float* zb = z + (size_t)b * K;
-    const int cls = (shift && shift_cls) ? shift_cls[b] : -1;
-    const float sh = cls >= 0 && cls < K ? shift[b] : 0.f;
+    const int cls = (d.shift && d.shift_cls) ? d.shift_cls[b] : -1;
+    const float sh = cls >= 0 && cls < K ? d.shift[b] : 0.f;
     float m = -INFINITY;
     int arg = 0x7fffffff;
     float zr[kRegs];
 #pragma unroll
     for (int i = 0; i < kRegs; ++i) {
       const int k = lane + 32 * i;
-      zr[i] = k < K ? __ldcg(zb + k) : -INFINITY;   // logits may come from other CTAs: read through L2
+      zr[i] = k < K ? __ldcg(zb + k) : -INFINITY;
     }
 #pragma unroll
     for (int i = 0; i < kRegs; ++i) {
@@ -302,16 +172,24 @@ __device__ __forceinline__ void exit_decide_block(float* z, int B, int K, const 
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     if (lane == 0) {
       const float cf = 1.0f / s;
-      if (conf) conf[b] = cf;
-      if (pred) pred[b] = arg == 0x7fffffff ? 0 : arg;
-      mask[b] = (uint8_t)((always_exit || cf >= thr) ? 1 : 0);
+      if (d.conf) d.conf[b] = cf;
+      if (d.pred) d.pred[b] = arg == 0x7fffffff ? 0 : arg;
+      d.mask[b] = (uint8_t)((d.always_exit || cf >= d.thr) ? 1 : 0);
     }
   }
-  __syncthreads();
+}
+
+// One CTA of THREADS threads: ballot + prefix-sum scan over the not-exit flags of samples [0, B) gives the ascending
+// survivor list, the survivors' ids and their count (B_rem).  The flags may have been written by other CTAs.
+template <int THREADS>
+__device__ __forceinline__ void exit_scan(int B, const DecideArgs& d) {
+  __shared__ int warp_tot[32];
+  __shared__ int pass_total;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   int base = 0;  // identical in every thread
   for (int p0 = 0; p0 < B; p0 += THREADS) {
     const int b = p0 + tid;
-    const bool keep = b < B && mask[b] == 0;
+    const bool keep = b < B && __ldcg(d.mask + b) == 0;
     const unsigned bal = __ballot_sync(0xffffffffu, keep);
     const int pre = __popc(bal & ((1u << lane) - 1u));
     if (lane == 0) warp_tot[warp] = __popc(bal);
@@ -330,21 +208,141 @@ __device__ __forceinline__ void exit_decide_block(float* z, int B, int K, const 
     __syncthreads();
     if (keep) {
       const int pos = base + warp_tot[warp] + pre;
-      surv_idx[pos] = b;
-      if (ids && ids_out) ids_out[pos] = ids[b];
+      d.surv_idx[pos] = b;
+      if (d.ids && d.ids_out) d.ids_out[pos] = d.ids[b];
     }
     base += pass_total;
     __syncthreads();
   }
-  if (tid == 0) n_surv[0] = base;
+  if (tid == 0) d.n_surv[0] = base;
 }
 
-__global__ void __launch_bounds__(kDecideThreads)
-exit_decide_kernel(float* z, int B, int K, const float* __restrict__ shift, const int32_t* __restrict__ shift_cls, float thr,
-                   int always_exit, float* __restrict__ conf, int32_t* __restrict__ pred, uint8_t* mask,
-                   const int32_t* __restrict__ ids, int32_t* __restrict__ surv_idx, int32_t* __restrict__ ids_out,
-                   int32_t* __restrict__ n_surv) {
-  exit_decide_block<kDecideThreads>(z, B, K, shift, shift_cls, thr, always_exit, conf, pred, mask, ids, surv_idx, ids_out, n_surv);
+constexpr int kFcWarps = 8, kFcClassesPerWarp = 2, kFcSamples = 16, kFcChunk = 128;
+constexpr int kFcClasses = kFcWarps * kFcClassesPerWarp;
+constexpr int kFcThreads = kFcWarps * 32;
+
+// z[b][k] = bfc[k] + sum_c wfc[k][c] * gap[b][c].  CTA (x, y) owns 16 classes (two per warp) of the 16 samples of
+// tile y and walks the channels 128 at a time: the tile's pooled values and the classes' weights of a chunk arrive
+// in shared memory through cp.async, two chunks ahead of the arithmetic (ALIGNED; rows that are not whole 16-byte
+// vectors take plain loads, one chunk at a time).  Per (b, k): every lane adds its four channels of each chunk in
+// ascending order, then a shuffle tree; the order does not depend on the batch size or the sample's position.
+//
+// No CTA waits for another.  The CTA that completes a sample tile's logits (a counter per tile) takes that tile's
+// exit decisions: softmax top-1 and threshold.  The CTA that completes the last tile's decisions (a second
+// counter) runs the stable scan of the survivors over the whole batch and leaves all counters at zero.
+// Launched with programmatic stream serialization.
+template <typename T, bool ALIGNED>
+__global__ void __launch_bounds__(kFcThreads)
+fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float* __restrict__ bfc, int B, int C, int K, float* z,
+          DecideArgs d) {
+  constexpr int STAGES = ALIGNED ? (sizeof(T) == 2 ? 3 : 2) : 1;
+  constexpr int PER = kFcChunk / 32;  // channels per lane per chunk (4)
+  __shared__ __align__(16) float gs[STAGES][kFcSamples][kFcChunk];
+  __shared__ __align__(16) T wsm[STAGES][kFcClasses][kFcChunk];
+  __shared__ bool last_flag;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int k0 = blockIdx.x * kFcClasses, b0 = blockIdx.y * kFcSamples;
+  const int nchunk = (C + kFcChunk - 1) / kFcChunk;
+
+  auto stage_load = [&](int chunk, int buf) {
+    const int c0 = chunk * kFcChunk;
+    if constexpr (ALIGNED) {
+      constexpr int WV = 16 / (int)sizeof(T);       // weight elements per 16-byte vector
+      constexpr int WPC = kFcChunk / WV;            // vectors per class
+      for (int i = tid; i < kFcSamples * (kFcChunk / 4); i += kFcThreads) {
+        const int sidx = i / (kFcChunk / 4), c = (i % (kFcChunk / 4)) * 4;
+        const bool in = b0 + sidx < B && c0 + c < C;
+        cp_async16(&gs[buf][sidx][c], in ? gap + (size_t)(b0 + sidx) * C + c0 + c : gap, in ? 16 : 0);
+      }
+      for (int i = tid; i < kFcClasses * WPC; i += kFcThreads) {
+        const int cls = i / WPC, c = (i % WPC) * WV;
+        const bool in = k0 + cls < K && c0 + c < C;
+        cp_async16(&wsm[buf][cls][c], in ? wfc + (size_t)(k0 + cls) * C + c0 + c : wfc, in ? 16 : 0);
+      }
+    } else {
+      for (int i = tid; i < kFcSamples * kFcChunk; i += kFcThreads) {
+        const int sidx = i / kFcChunk, c = i % kFcChunk;
+        gs[buf][sidx][c] = (b0 + sidx < B && c0 + c < C) ? gap[(size_t)(b0 + sidx) * C + c0 + c] : 0.f;
+      }
+      for (int i = tid; i < kFcClasses * kFcChunk; i += kFcThreads) {
+        const int cls = i / kFcChunk, c = i % kFcChunk;
+        Elem<T>::st(&wsm[buf][cls][c], (k0 + cls < K && c0 + c < C) ? Elem<T>::ld(wfc + (size_t)(k0 + cls) * C + c0 + c) : 0.f);
+      }
+    }
+  };
+
+  pdl_wait();
+  pdl_launch_dependents();
+  float acc[kFcClassesPerWarp][kFcSamples];
+#pragma unroll
+  for (int q = 0; q < kFcClassesPerWarp; ++q)
+#pragma unroll
+    for (int s2 = 0; s2 < kFcSamples; ++s2) acc[q][s2] = 0.f;
+  if constexpr (ALIGNED) {
+#pragma unroll
+    for (int s0 = 0; s0 < STAGES - 1; ++s0) {
+      if (s0 < nchunk) stage_load(s0, s0);
+      cp_async_commit();   // one group per chunk, possibly empty: the wait below counts groups
+    }
+  }
+  for (int chunk = 0; chunk < nchunk; ++chunk) {
+    const int buf = chunk % STAGES;
+    if constexpr (ALIGNED) {
+      cp_async_wait<STAGES - 2>();
+      __syncthreads();   // chunk landed for every thread; the buffer refilled below was read one iteration ago
+      const int next = chunk + STAGES - 1;
+      if (next < nchunk) stage_load(next, next % STAGES);
+      cp_async_commit();
+    } else {
+      __syncthreads();
+      stage_load(chunk, 0);
+      __syncthreads();
+    }
+    float wv[kFcClassesPerWarp][PER];
+#pragma unroll
+    for (int q = 0; q < kFcClassesPerWarp; ++q)
+#pragma unroll
+      for (int e = 0; e < PER; ++e) wv[q][e] = Elem<T>::ld(&wsm[buf][warp * kFcClassesPerWarp + q][lane * PER + e]);
+#pragma unroll
+    for (int s2 = 0; s2 < kFcSamples; ++s2) {
+      const float4 g = *reinterpret_cast<const float4*>(&gs[buf][s2][lane * PER]);
+      const float gv[PER] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+      for (int q = 0; q < kFcClassesPerWarp; ++q)
+#pragma unroll
+        for (int e = 0; e < PER; ++e) acc[q][s2] = fmaf(wv[q][e], gv[e], acc[q][s2]);
+    }
+  }
+#pragma unroll
+  for (int q = 0; q < kFcClassesPerWarp; ++q) {
+    const int k = k0 + warp * kFcClassesPerWarp + q;
+    const float bk = (bfc && k < K) ? bfc[k] : 0.f;
+#pragma unroll
+    for (int s2 = 0; s2 < kFcSamples; ++s2) {
+      float v = acc[q][s2];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0 && k < K && b0 + s2 < B) z[(size_t)(b0 + s2) * K + k] = v + bk;
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) last_flag = atomicAdd(d.tile_done + blockIdx.y, 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (!last_flag) return;
+  __threadfence();
+  exit_decide_samples(z, b0, min(B, b0 + kFcSamples), K, warp, kFcWarps, d);
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    d.tile_done[blockIdx.y] = 0;
+    last_flag = atomicAdd(d.done, 1u) == gridDim.y - 1;
+  }
+  __syncthreads();
+  if (!last_flag) return;
+  __threadfence();
+  if (tid == 0) *d.done = 0;
+  exit_scan<kFcThreads>(B, d);
 }
 
 constexpr int kCopyThreads = 256, kCopyUnroll = 8;

@@ -55,11 +55,11 @@ def test_static_scratch_head_matches_caller_scratch_head_twice(dtype, HW, C, K):
 
 
 def test_static_scratch_head_refuses_what_does_not_fit():
-    # 8 MiB array: 64 samples x 98 pooling chunks x 2048 channels of fp32 partial sums alone need 51 MB
-    spec = _head_model("bf16", 784, 2048, 10, max_batch=64)
+    # 8 MiB array: the pooled vectors of 1100 samples x 2048 channels in fp32 alone need 9 MB
+    spec = _head_model("bf16", 4, 2048, 10, max_batch=1100)
     m = eb.EEModel(spec)
     out = eb.StageBuffers(m, 0)
-    x = torch.zeros((1, 784, 2048), dtype=torch.bfloat16, device="cuda")
+    x = torch.zeros((1, 4, 2048), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(eb.EEError) as e:
-        m.exit_head_static(0, x, 1, 784, out)
+        m.exit_head_static(0, x, 1, 4, out)
     assert e.value.status == 3 and "scratch bytes" in str(e.value)
