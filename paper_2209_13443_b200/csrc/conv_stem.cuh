@@ -118,13 +118,15 @@ conv_stem7x7_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (warp == 0 && lane == 0) {   // the whole weight matrix stays resident; no kernel writes it, so it need not wait
+    mbar_expect_tx(w_bar, kStemKBlocks * S::kWBytes);
+    for (int i = 0; i < kStemKBlocks; ++i) tma_load_3d(base + S::kWOff + i * S::kWBytes, &tmW, w_bar, i * kTcBK, 0, 0);
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == 0) {
     if (lane == 0) {
-      mbar_expect_tx(w_bar, kStemKBlocks * S::kWBytes);   // the whole weight matrix stays resident
-      for (int i = 0; i < kStemKBlocks; ++i) tma_load_3d(base + S::kWOff + i * S::kWBytes, &tmW, w_bar, i * kTcBK, 0, 0);
       for (int j = 0; j < my_tiles; ++j) {
         const int t = (int)blockIdx.x + j * (int)gridDim.x;
         const int n = t / p.Ho, oy = t - n * p.Ho;

@@ -352,9 +352,18 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // Programmatic dependent launch: everything above overlapped the tail of the previous kernel in the stream.
-  // From here on this kernel touches activations, so it waits for that kernel's memory; the next kernel in
-  // the stream may begin its own prologue now.
+  // Programmatic dependent launch: everything above overlapped the tail of the previous kernel in the stream, and
+  // so do the weight tiles of the first ring slots, which no kernel writes.  From the wait on this kernel touches
+  // activations, so it needs that kernel's memory; the next kernel in the stream may begin its own prologue now.
+  const int w_ahead = min(num_kb, kStages);
+  if (warp == 0 && lane == 0) {
+    for (int i = 0; i < w_ahead; ++i) {   // the slots start out empty
+      const int kb = kb_begin + i;
+      const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
+      mbar_expect_tx(full_bar(i), GATHER ? S::kBBytes : S::kStage);
+      tma_load_3d(base + (uint32_t)i * S::kStage + S::kABytes, &tmW, full_bar(i), cb * kTcBK, tap, n0);
+    }
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
@@ -381,10 +390,13 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
         const int kb = kb_begin + i;
         const int s = i % kStages;
         const uint32_t ph = (uint32_t)(i / kStages) & 1u;
-        if (!mbar_wait(empty_bar(s), ph ^ 1u, p.err_flag)) break;
         const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
         const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
-        mbar_expect_tx(full_bar(s), GATHER ? S::kBBytes : S::kStage);
+        if (i >= w_ahead) {   // earlier slots: armed and their weight tile requested before the dependency wait
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, p.err_flag)) break;
+          mbar_expect_tx(full_bar(s), GATHER ? S::kBBytes : S::kStage);
+          tma_load_3d(sb, &tmW, full_bar(s), cb * kTcBK, tap, n0);
+        }
         if (GATHER) {
         } else if (p.im2col) {
           const int r = tap / p.kw;
@@ -392,7 +404,6 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
         } else {
           tma_load_2d(sa, &tmA, full_bar(s), cb * kTcBK, m0);
         }
-        tma_load_3d(sb, &tmW, full_bar(s), cb * kTcBK, tap, n0);
       }
     }
   } else if (warp == 1) {
@@ -656,6 +667,17 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // weight tiles of the first ring slots (first tile of this CTA) are requested before the dependency wait: no
+  // kernel writes them
+  const int w_ahead = my_tiles > 0 ? min(num_kb, kStages) : 0;
+  if (warp == 0 && lane == 0) {
+    const int n0 = ((int)blockIdx.x % n_tiles) * BN;
+    for (int i = 0; i < w_ahead; ++i) {
+      const int tap = i / p.cblocks, cb = i - tap * p.cblocks;
+      mbar_expect_tx(full_bar(i), S::kStage);
+      tma_load_3d(base + (uint32_t)i * S::kStage + S::kABytes, &tmW, full_bar(i), cb * kTcBK, tap, n0);
+    }
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
@@ -689,18 +711,20 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
         for (int kb = 0; kb < num_kb; ++kb, ++g) {
           const int s = g % kStages;
           const uint32_t ph = (uint32_t)(g / kStages) & 1u;
-          ok = mbar_wait(empty_bar(s), ph ^ 1u, p.err_flag);
-          if (!ok) break;
           const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
           const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
-          mbar_expect_tx(full_bar(s), S::kStage);
+          if (g >= w_ahead) {   // earlier slots were armed before the dependency wait
+            ok = mbar_wait(empty_bar(s), ph ^ 1u, p.err_flag);
+            if (!ok) break;
+            mbar_expect_tx(full_bar(s), S::kStage);
+            tma_load_3d(sb, &tmW, full_bar(s), cb * kTcBK, tap, n0);
+          }
           if (p.im2col) {
             const int r = tap / p.kw;
             tma_load_im2col_4d(sa, &tmA, full_bar(s), cb * kTcBK, cw, ch, cn, (uint16_t)(tap - r * p.kw), (uint16_t)r);
           } else {
             tma_load_2d(sa, &tmA, full_bar(s), cb * kTcBK, m0);
           }
-          tma_load_3d(sb, &tmW, full_bar(s), cb * kTcBK, tap, n0);
         }
       }
     }
