@@ -30,7 +30,6 @@ namespace ee {
 
 constexpr int kTcBM = 128;       // output pixels per CTA (= TMEM lanes)
 constexpr int kTcBK = 64;        // bf16 elements per K block: 128 bytes = one swizzle span
-constexpr int kTcSplitMaxCtas = 296;  // split-K only while tiles x ranges at max_batch stay within two CTAs per SM
 constexpr int kTcThreads = 192;  // producer warp, MMA warp, four epilogue warps
 constexpr long long kTcWaitCycles = 4000000000LL;  // ~2 s at boost clock; far beyond any healthy wait
 
@@ -289,11 +288,12 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src
 // tmA: activations (2-D tile map or im2col map), tmW: weights [Cin][taps][Cout], tmR / tmO: residual and output as
 // [rows][Cout] matrices with a 64-column x 32-row box (128-byte swizzle).
 //
-// SPLIT: the K loop of one output tile is cut into gridDim.z (2, 4 or 8) fixed ranges of p.kb_per K blocks, a
-// property of the layer and never of the batch.  The CTAs of a tile form a thread-block cluster along z: each leaves
-// its fp32 partial tile in its own shared memory, then every CTA reduces one slice of rows by reading all partials
-// through distributed shared memory in ascending range order (a reduce-scatter), applies the epilogue to that
-// slice and stores it.
+// SPLIT: the K loop of one output tile is cut into gridDim.z (2 to 8) fixed ranges of p.kb_per K blocks, a
+// property of the layer and never of the batch.  The CTAs of a tile form a thread-block cluster along z.  CTA z owns
+// a slice of the tile's rows: once every CTA has drained its ring (first cluster barrier), each thread sends its row
+// of the fp32 partial tile to the owner's shared memory through distributed shared memory; after the second
+// barrier every CTA adds the partials of its rows in ascending range order, all from its own shared memory (a
+// reduce-scatter), applies the epilogue to that slice and stores it.
 //
 // GATHER: operand A comes from CUDA cores instead of TMA, for layers whose pixel rows are not whole 16-byte units
 // (a 3-channel stem).  K is laid out as kh runs of runp columns: run r holds the kw*Cin taps of filter row r, which
@@ -456,10 +456,21 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
     const int q = warp & 3;  // TMEM lane quarter this warp may read = rows [32q, 32q + 32) of the tile
     const int row = q * 32 + lane;
     if (SPLIT) {
-      // fp32 partial tile [128 rows][BN] into the drained ring; 16-byte chunks XOR-swizzled with the row so that
-      // neither these row-wise writes nor the peers' reads pile onto one bank
+      // Reduce-scatter, push side.  CTA z of the cluster owns tile rows [z * rows_per, (z + 1) * rows_per); this thread
+      // sends its row of the fp32 partial tile to the owner's shared memory (slot `rank` of the owner's receive
+      // buffer, which overlays the drained ring), 16-byte chunks XOR-swizzled with the row so that neither these
+      // row-wise stores nor the owner's reads pile onto one bank.  The first cluster barrier guarantees that every
+      // peer has finished with its ring before anybody writes into it.
       constexpr int CH = BN / 4;
-      float* part = reinterpret_cast<float*>(gen);
+      const int nsplit = (int)gridDim.z;
+      const int rows_per = (kTcBM + nsplit - 1) / nsplit;
+      uint32_t rank;
+      asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+      const int owner = row / rows_per, rloc = row - owner * rows_per;
+      uint32_t dst;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(base + (uint32_t)(((int)rank * rows_per + rloc) * (BN * 4))), "r"(owner));
+      asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+      bool waited = false;
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
         float v[32];
@@ -469,11 +480,16 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = 0.f;
         }
+        if (!waited) {
+          asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+          waited = true;
+        }
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
           const int c = (c0 >> 2) + g;
-          *reinterpret_cast<float4*>(part + (size_t)row * BN + ((c ^ (row & (CH - 1))) << 2)) =
-              make_float4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+          asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)((c ^ (rloc & (CH - 1))) << 4)), "f"(v[4 * g]),
+                       "f"(v[4 * g + 1]), "f"(v[4 * g + 2]), "f"(v[4 * g + 3])
+                       : "memory");
         }
       }
     } else if (ok) {
@@ -519,42 +535,36 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
     }
   }
   if (SPLIT) {
-    // every thread of every CTA of the cluster passes both barriers, whatever happened above
+    // Every thread of every CTA of the cluster passes both barriers, whatever happened above: the first one before
+    // any remote store (epilogue threads took it inside their push loop), the second once all partials have landed.
+    if (warp < 2) asm volatile("barrier.cluster.arrive.release;\n barrier.cluster.wait.acquire;" ::: "memory");
     asm volatile("barrier.cluster.arrive.release;\n barrier.cluster.wait.acquire;" ::: "memory");
     if (warp >= 2) {
+      // Pull side, all local: this CTA adds the nsplit partials of its rows in ascending range order (the grouping
+      // of the sum is fixed by the layer), applies the epilogue and stores.
       constexpr int CH = BN / 4, G = BN / 8;     // 16-byte fp32 chunks and 8-column groups per row
       const int et = threadIdx.x - 64;
       const int nsplit = (int)gridDim.z;
+      const int rows_per = (kTcBM + nsplit - 1) / nsplit;
       uint32_t rank;
       asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
-      const int rows_per = kTcBM / nsplit;
-      const uint32_t part_s = base;             // same offset in every CTA of the cluster
+      const float* part = reinterpret_cast<const float*>(gen);
       for (int item = et; item < rows_per * G; item += 128) {
         const int r = item / G, g = item - r * G;
         const int trow = (int)rank * rows_per + r;
+        if (trow >= kTcBM) break;
         const int m = m0 + trow, n = n0 + g * 8;
-        const uint32_t a0 = part_s + (uint32_t)trow * (BN * 4) + (uint32_t)(((2 * g) ^ (trow & (CH - 1))) << 4);
-        const uint32_t a1 = part_s + (uint32_t)trow * (BN * 4) + (uint32_t)(((2 * g + 1) ^ (trow & (CH - 1))) << 4);
+        const int o0 = ((2 * g) ^ (r & (CH - 1))) << 2, o1 = ((2 * g + 1) ^ (r & (CH - 1))) << 2;
         float v[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) v[e] = 0.f;
-        float4 x0[8], x1[8];
-#pragma unroll
-        for (int z = 0; z < 8; ++z) {             // all remote loads in flight before the first addition
-          if (z < nsplit) {
-            uint32_t ra0, ra1;
-            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra0) : "r"(a0), "r"(z));
-            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra1) : "r"(a1), "r"(z));
-            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(x0[z].x), "=f"(x0[z].y), "=f"(x0[z].z), "=f"(x0[z].w) : "r"(ra0) : "memory");
-            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(x1[z].x), "=f"(x1[z].y), "=f"(x1[z].z), "=f"(x1[z].w) : "r"(ra1) : "memory");
-          }
-        }
-#pragma unroll
-        for (int z = 0; z < 8; ++z) {             // ascending range order: the grouping of the sum is fixed by the layer
-          if (z < nsplit) {
-            v[0] += x0[z].x; v[1] += x0[z].y; v[2] += x0[z].z; v[3] += x0[z].w;
-            v[4] += x1[z].x; v[5] += x1[z].y; v[6] += x1[z].z; v[7] += x1[z].w;
-          }
+#pragma unroll 4
+        for (int z = 0; z < nsplit; ++z) {
+          const float* pr = part + (size_t)(z * rows_per + r) * BN;
+          const float4 x0 = *reinterpret_cast<const float4*>(pr + o0);
+          const float4 x1 = *reinterpret_cast<const float4*>(pr + o1);
+          v[0] += x0.x; v[1] += x0.y; v[2] += x0.z; v[3] += x0.w;
+          v[4] += x1.x; v[5] += x1.y; v[6] += x1.z; v[7] += x1.w;
         }
         if (m < p.M && n < p.N) {
           scale_bias<8>(v, s_scale + g * 8, s_bias + g * 8);
@@ -571,8 +581,6 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
         }
       }
     }
-    // no CTA may retire while a peer still reads its shared memory
-    asm volatile("barrier.cluster.arrive.release;\n barrier.cluster.wait.acquire;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
@@ -960,21 +968,39 @@ inline ee_status_t tc_plan_layer(TcContext& c, const ee_layer_desc_t& d, int in_
   L->in_h = in_h, L->in_w = in_w, L->out_h = out_h, L->out_w = out_w, L->max_batch = max_batch;
   L->bn = d.cout > 64 ? 128 : 64;
   L->im2col = !(d.kh == 1 && d.stride == 1 && d.pad == 0);
-  // Split-K for layers whose grid stays small even at the model's max_batch while their K loop is long (the deep
-  // stages of a small-batch model): a lone CTA cannot pull operands faster than its SM's L2 port, so the K range is
-  // spread over a cluster of 2, 4 or 8 CTAs.  The cut depends on the layer and on max_batch (both fixed at model
-  // creation), never on the batch actually run, so a sample's sums are grouped the same way in every call.
+  // Split-K: a lone CTA cannot pull operands faster than its SM's L2 port (about 126 GB/s: a 32 KB K block of a
+  // 128x128 tile takes 0.26 us in tile mode and 0.36 us in im2col mode, against 0.13 us of MMA time), so a layer
+  // whose grid leaves SMs idle spreads the K range of a tile over a cluster of 2..4 CTAs.  A split costs about
+  // 4.5 us (cluster launch, two cluster barriers, the reduce-scatter), larger clusters gain nothing measurable, and
+  // grids of more than two CTAs per SM lose to the unsplit kernel, hence the bounds.  The number of ranges is chosen
+  // once per layer by this cost model summed over the batch sizes the model will see (max_batch, 3/4, 1/2 and 1/4
+  // of it: the batch shrinks at every exit), the analogue of the per-layer objective sum_b w_b T(b) of the paper's
+  // design-space exploration (Eq. 2).  It depends on the layer and on max_batch, never on the batch actually run,
+  // so a sample's sums are grouped the same way in every call.
   {
     const int num_kb = d.kh * d.kw * cdiv(d.cin, kTcBK);
-    const long tiles = (long)cdiv((long)max_batch * out_h * out_w, kTcBM) * cdiv(d.cout, L->bn);
+    const int n_tiles = cdiv(d.cout, L->bn);
+    const double t_block = (L->im2col ? 0.36 : 0.26) * (16384.0 + L->bn * 128.0) / 32768.0;   // us per K block per SM
+    const long tiles_max = (long)cdiv((long)max_batch * out_h * out_w, kTcBM) * n_tiles;
+    double best = 0;
     L->splits = 1;
     L->kb_per = num_kb;
-    for (int sp = 8; sp >= 2; sp >>= 1) {
+    for (int sp = 1; sp <= 4; ++sp) {
       const int per = cdiv(num_kb, sp);
-      if (tiles * sp <= kTcSplitMaxCtas && sp * 8 <= num_kb && (sp - 1) * per < num_kb) {
+      if (sp > 1 && (per < 4 || (sp - 1) * per >= num_kb || tiles_max * sp > 2 * c.sm_count + 4)) continue;
+      double cost = 0;
+      for (int f = 4; f >= 1; --f) {
+        const int b = std::max(1, (max_batch * f + 3) / 4);
+        const long tiles = (long)cdiv((long)b * out_h * out_w, kTcBM) * n_tiles;
+        const long share = cdiv(tiles * sp, c.sm_count);   // CTAs that share the L2 port of the busiest SM
+        cost += 2.4 + (sp > 1 ? 4.5 : 0.0) + (double)share * per * t_block + 0.8 * cdiv(tiles, c.sm_count);
+      }
+      if (sp == 1) {
+        best = cost;
+      } else if (cost < best) {
+        best = cost;
         L->splits = sp;
         L->kb_per = per;
-        break;
       }
     }
   }
