@@ -10,6 +10,7 @@
 #include "conv_simt.cuh"
 #include "conv_tc.cuh"
 #include "conv_stem.cuh"
+#include "conv_halo.cuh"
 #include "head.cuh"
 
 using namespace ee;
@@ -168,7 +169,8 @@ ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const
       break;
     }
     case KK_TC: {
-      ee_status_t s = tc_launch(m->tc, L.tc, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st);
+      ee_status_t s = L.tc.halo ? halo_launch(m->tc, L.tc, src, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st)
+                                : tc_launch(m->tc, L.tc, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st);
       if (s != EE_OK) return s;
       break;
     }
@@ -369,6 +371,7 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
   }
   rc = tc_context_init(m->tc);
   if (rc == EE_OK) rc = stem_context_init();
+  if (rc == EE_OK) rc = halo_context_init();
   if (rc != EE_OK) return fail(rc);
 
   int h = desc->in_h, w = desc->in_w, c = desc->in_c;
@@ -494,6 +497,7 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
         L.kind = KK_TC;
         rc = tc_plan_layer(m->tc, d, L.in_h, L.in_w, L.out_h, L.out_w, desc->max_batch, L.w_dev, &L.tc);
         if (rc != EE_OK) return fail(rc);
+        L.tc.halo = halo_supported(d, L.in_w);
       } else if (desc->dtype == EE_BF16 && d.cout % 8 == 0 && d.kh * d.kw * d.cin <= 1024) {
         // pixel rows are not 16-byte units (e.g. a 3-channel stem): explicit Toeplitz rows, then the tensor-core GEMM
         L.kind = KK_TC_GATHER;

@@ -901,12 +901,13 @@ struct TcLayer {
   // gather mode: geometry of the real convolution (cin/kh/... above then describe the packed 1x1 GEMM view)
   bool gather = false;
   bool stem7 = false;   // the 7x7/2 stem kernel of conv_stem.cuh takes this layer
+  bool halo = false;    // the 3x3 halo-block kernel of conv_halo.cuh takes this layer
   int g_h = 0, g_w = 0, g_cin = 0, g_kh = 0, g_kw = 0, g_stride = 1, g_pad = 0, g_runp = 0;
   CUtensorMap tm_w;
   struct Cached {
     const void* ptr;
     int batch;
-    int kind;  // 0: operand A, 1: residual / output matrix, 2: stem input rows, 3: stem output rows
+    int kind;  // 0: operand A, 1: residual / output matrix, 2: stem input rows, 3: stem output rows, 4: halo blocks
     CUtensorMap tm;
   };
   mutable std::vector<Cached> a_maps;  // tensor maps of caller buffers by (pointer, batch, kind)
@@ -1030,7 +1031,17 @@ inline ee_status_t tc_buffer_map(const TcContext& c, const TcLayer& L, const voi
   e.batch = batch;
   e.kind = kind;
   CUresult r;
-  if (kind == 2) {
+  if (kind == 4) {
+    // NHWC as (C, W, H, B); a box is the R + 2 rows of W + 2 pixels one output tile of R rows touches (zero fill outside)
+    const int wp = L.in_w + 2, rows = kTcBM / wp + 2;
+    const cuuint64_t dims[4] = {(cuuint64_t)L.cin, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)batch};
+    const cuuint64_t strides[3] = {(cuuint64_t)L.cin * 2, (cuuint64_t)L.cin * 2 * L.in_w, (cuuint64_t)L.cin * 2 * L.in_w * L.in_h};
+    const cuuint32_t box[4] = {kTcBK, (cuuint32_t)wp, (cuuint32_t)rows, 1};
+    const cuuint32_t es[4] = {1, 1, 1, 1};
+    r = c.encode_tiled(&e.tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, es,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else if (kind == 2) {
     // stem input as (W*Cin, H, B): 256 elements of 7 consecutive image rows per load, zero fill outside
     const cuuint64_t dims[3] = {(cuuint64_t)L.g_w * L.g_cin, (cuuint64_t)L.g_h, (cuuint64_t)batch};
     const cuuint64_t strides[2] = {(cuuint64_t)L.g_w * L.g_cin * 2, (cuuint64_t)L.g_w * L.g_cin * 2 * L.g_h};

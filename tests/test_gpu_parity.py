@@ -116,6 +116,30 @@ def test_conv_layer(dtype, geom):
         assert g["n_surv"] == B
 
 
+# 3x3 / 64-channel bf16 layers, which the halo-block kernel takes: one tile per image, several tiles per image with a
+# ragged last one, a tile of one image row, the benchmark's 56x56 map, fewer than 64 filters, a one-pixel-wide image
+HALO_GEOMS = [
+    (7, 7, 64, 64, wl.ACT_RELU),
+    (23, 19, 64, 64, wl.ACT_RELU),
+    (5, 61, 64, 40, wl.ACT_NONE),
+    (56, 56, 64, 64, wl.ACT_RELU),
+    (3, 1, 64, 8, wl.ACT_RELU6),
+]
+
+
+@pytest.mark.parametrize("geom", HALO_GEOMS)
+def test_conv3x3_halo_layer(geom):
+    H, W, cin, cout, act = geom
+    spec = util.single_layer_model("bf16", H, W, cin, cout, 3, 1, 1, act, False, seed=hash(geom) % 1000, max_batch=5)
+    run = util.GpuRunner(spec)
+    for B in (1, 5):
+        x = wl.random_features((B, H, W, cin), seed=B, bf16=True, relu=False)
+        o = util.oracle_stage(spec, 0, x)
+        g = run.stage(0, x)
+        util.check_stage(spec, g, o, f"halo {geom} B={B}", elementwise=True)
+        assert g["n_surv"] == B
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("C,stride,H,W", [(32, 1, 9, 9), (96, 2, 10, 7), (144, 1, 6, 6), (12, 2, 8, 8)])
 def test_depthwise_layer(dtype, C, stride, H, W):
