@@ -185,6 +185,12 @@ ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const
       break;
     }
     case KK_DW: {
+      if constexpr (sizeof(T) == 2) {
+        if (dwconv3x3_supported(g, src, L.w_dev, dst)) {
+          EE_CUDA(dwconv3x3_launch((const bf16*)src, (const bf16*)L.w_dev, L.scale_dev, L.bias_dev, (bf16*)dst, g, st));
+          break;
+        }
+      }
       const bool vec = L.d.cin % V == 0;
       const long total = (long)B * L.out_h * L.out_w * (vec ? L.d.cin / V : L.d.cin);
       const int grid = (int)std::min<long>(cdiv(total, 256), 148L * 32);

@@ -156,6 +156,125 @@ dwconv_kernel(const T* __restrict__ x, const T* __restrict__ w, const float* __r
   }
 }
 
+// Depthwise 3x3 pad-1 convolution on bf16, stride 1 or 2: the layers of the inverted-residual blocks.  The kernel
+// above issues one 2-byte load per (tap, channel) for the weights and one 16-byte load per tap for the input: 81
+// loads for 72 FMAs, which makes the load/store units, not memory, the bound.  Here a thread owns one vector of
+// eight channels for its whole life: it reads that vector's 72 weights once (144 contiguous bytes of the
+// [C][3][3] array) and keeps them in registers as stored, then walks items of kDwStrip consecutive output pixels of one
+// output row.  Per item it requests all 3 x ((kDwStrip - 1) * STRIDE + 3) input vectors up front (enough bytes in
+// flight per SM to cover the memory latency) and uses each for every output it overlaps.  Every output still sums its nine taps in ascending (r, s) with fp32 FMAs.
+// Block (x, y): x runs over channel vectors (adjacent threads read adjacent 16-byte vectors), y over items.
+constexpr int kDwStrip = 4;
+
+template <int STRIDE>
+__global__ void __launch_bounds__(256)
+dwconv3x3_bf16_kernel(const bf16* __restrict__ x, const bf16* __restrict__ w, const float* __restrict__ scale,
+                      const float* __restrict__ bias, bf16* __restrict__ y, ConvGeom g, int strips) {
+  constexpr int P = kDwStrip, COLS = (P - 1) * STRIDE + 3;
+  const int cv = g.Cin / 8;
+  const int c8 = blockIdx.y * blockDim.x + threadIdx.x;
+  if (c8 >= cv) return;
+  const int c = c8 * 8;
+  uint32_t raw[36];   // the vector's 72 weights as stored: element e = channel e / 9, tap e % 9
+  {
+    const uint4* wp = reinterpret_cast<const uint4*>(w + (size_t)c * 9);   // 9 x 16 bytes, 16-byte aligned
+#pragma unroll
+    for (int i = 0; i < 9; ++i) {
+      const uint4 v = __ldg(wp + i);
+      raw[4 * i] = v.x, raw[4 * i + 1] = v.y, raw[4 * i + 2] = v.z, raw[4 * i + 3] = v.w;
+    }
+  }
+  auto weight = [&](int tap, int ch) {   // indices are compile-time constants after unrolling
+    const int e = ch * 9 + tap;
+    return (e & 1) ? __uint_as_float(raw[e >> 1] & 0xffff0000u) : __uint_as_float(raw[e >> 1] << 16);
+  };
+  float sc[8], bi[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    sc[e] = scale ? scale[c + e] : 1.f;
+    bi[e] = bias ? bias[c + e] : 0.f;
+  }
+  const long items = (long)g.B * g.Ho * strips;
+  for (long item = (long)blockIdx.x * blockDim.y + threadIdx.y; item < items; item += (long)gridDim.x * blockDim.y) {
+    const int st = (int)(item % strips);
+    const long t = item / strips;
+    const int ho = (int)(t % g.Ho);
+    const long b = t / g.Ho;
+    const int wo0 = st * P;
+    const int hi0 = ho * STRIDE - 1, wi0 = wo0 * STRIDE - 1;
+    float acc[P][8];
+#pragma unroll
+    for (int pp = 0; pp < P; ++pp)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[pp][e] = 0.f;
+    uint4 v[3][COLS];   // every input vector of the item is requested before the first FMA
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+      const int hi = hi0 + r;
+      const bool row_in = hi >= 0 && hi < g.H;
+      const bf16* row = x + ((b * g.H + (row_in ? hi : 0)) * g.W) * (long)g.Cin + c;
+#pragma unroll
+      for (int j = 0; j < COLS; ++j) {
+        const int wi = wi0 + j;
+        v[r][j] = (row_in && wi >= 0 && wi < g.W) ? __ldg(reinterpret_cast<const uint4*>(row + (long)wi * g.Cin)) : make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+#pragma unroll
+      for (int j = 0; j < COLS; ++j) {
+        const uint32_t wd[4] = {v[r][j].x, v[r][j].y, v[r][j].z, v[r][j].w};
+        float f[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          f[2 * i] = __uint_as_float(wd[i] << 16);
+          f[2 * i + 1] = __uint_as_float(wd[i] & 0xffff0000u);
+        }
+#pragma unroll
+        for (int pp = 0; pp < P; ++pp) {
+          const int s = j - pp * STRIDE;   // compile-time after unrolling
+          if (s >= 0 && s < 3) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[pp][e] = fmaf(f[e], weight(r * 3 + s, e), acc[pp][e]);
+          }
+        }
+      }
+    }
+    bf16* yp = y + ((b * g.Ho + ho) * g.Wo + wo0) * (long)g.Cout + c;
+#pragma unroll
+    for (int pp = 0; pp < P; ++pp) {
+      if (wo0 + pp < g.Wo) {
+        Vec16<bf16> o;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) o.v[e] = apply_act(fmaf(sc[e], acc[pp][e], bi[e]), g.act);
+        o.store(yp + (long)pp * g.Cout);
+      }
+    }
+  }
+}
+
+inline bool dwconv3x3_supported(const ConvGeom& g, const void* x, const void* w, const void* y) {
+  return g.kh == 3 && g.kw == 3 && g.pad == 1 && (g.stride == 1 || g.stride == 2) && g.Cin % 8 == 0 && g.Cin == g.Cout &&
+         (((uintptr_t)x | (uintptr_t)w | (uintptr_t)y) & 15) == 0;
+}
+
+inline cudaError_t dwconv3x3_launch(const bf16* x, const bf16* w, const float* scale, const float* bias, bf16* y, const ConvGeom& g,
+                                    cudaStream_t st) {
+  const int cv = g.Cin / 8;
+  const int bx = cv < 128 ? cv : 128;
+  const int by = 256 / bx > 0 ? 256 / bx : 1;
+  const int strips = (g.Wo + kDwStrip - 1) / kDwStrip;
+  const long items = (long)g.B * g.Ho * strips;
+  const long want = (items + by - 1) / by;
+  dim3 grid((unsigned)(want < 148L * 16 ? want : 148L * 16), (unsigned)((cv + bx - 1) / bx));
+  dim3 block(bx, by);
+  if (g.stride == 1)
+    dwconv3x3_bf16_kernel<1><<<grid, block, 0, st>>>(x, w, scale, bias, y, g, strips);
+  else
+    dwconv3x3_bf16_kernel<2><<<grid, block, 0, st>>>(x, w, scale, bias, y, g, strips);
+  return cudaGetLastError();
+}
+
 // Window maximum over in-range taps, NHWC, one thread per (output pixel, channel vector).
 template <typename T, int VEC>
 __global__ void __launch_bounds__(256)
