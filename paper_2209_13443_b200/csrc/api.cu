@@ -11,6 +11,7 @@
 #include "conv_tc.cuh"
 #include "conv_stem.cuh"
 #include "conv_halo.cuh"
+#include "conv_dw.cuh"
 #include "head.cuh"
 
 using namespace ee;
@@ -186,6 +187,11 @@ ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const
     }
     case KK_DW: {
       if constexpr (sizeof(T) == 2) {
+        if (dw_tma_supported(g, src, L.w_dev, dst)) {
+          ee_status_t s = dw_tma_launch(m->tc, L.tc, g, src, L.w_dev, L.scale_dev, L.bias_dev, dst, m->err_flag, st);
+          if (s != EE_OK) return s;
+          break;
+        }
         if (dwconv3x3_supported(g, src, L.w_dev, dst)) {
           EE_CUDA(dwconv3x3_launch((const bf16*)src, (const bf16*)L.w_dev, L.scale_dev, L.bias_dev, (bf16*)dst, g, st));
           break;
@@ -378,6 +384,7 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
   rc = tc_context_init(m->tc);
   if (rc == EE_OK) rc = stem_context_init();
   if (rc == EE_OK) rc = halo_context_init();
+  if (rc == EE_OK) rc = dw_context_init();
   if (rc != EE_OK) return fail(rc);
 
   int h = desc->in_h, w = desc->in_w, c = desc->in_c;
