@@ -3,7 +3,7 @@
 One "step" is one pass of the whole path over one batch of synthetic requests:
   ee_batch_refill (the arrivals are appended to the empty batch buffer) -> for every stage:
   ee_stage_run (convolutions, exit head, threshold, compaction + gather of the survivors) ->
-  the survivor count reaches the host (pinned word + stream sync) and sizes the next stage.
+  the survivor count reaches the host (pinned word, ee_wait_count) and sizes the next stage.
 The batch shrinks stage by stage at the calibrated exit rates, exactly as in serving.
 
 Default workload (N = 1): the ResNet-50-shaped 4-exit model, bf16, batch 64, 224x224 inputs.
@@ -234,6 +234,7 @@ def run_ours(args):
         sizes = []
         for s in range(nst):
             sizes.append(n)
+            bufs[s].arm_count()
             run_stage(s, feat, n, ids)
             nl += stage_launches(s, n)
             if e2e:
@@ -241,11 +242,12 @@ def run_ours(args):
                 res_host[s]["pred"][:n].copy_(bufs[s].pred[:n], non_blocking=True)
                 res_host[s]["mask"][:n].copy_(bufs[s].exit_mask[:n], non_blocking=True)
                 d2h += n * 9 + 4
-            stream.synchronize()                           # B_exit reaches the host: it sizes the next launch
-            n = int(bufs[s].n_surv_host[0])
+            n = bufs[s].wait_count()                       # B_exit reaches the host: it sizes the next launch
             feat, ids = bufs[s].features_out, bufs[s].ids_out
             if n == 0:
                 break
+        if e2e:
+            stream.synchronize()                           # every stage's results have arrived in host memory
         return nl, h2d, d2h, sizes
 
     def barrier():

@@ -139,8 +139,10 @@ typedef struct {
   int32_t* survivor_idx;  /* first n_surv entries: ascending positions (in the input batch) of the survivors */
   int32_t* ids_out;       /* first n_surv entries: ids of the survivors (written iff ids given) */
   int32_t* n_surv_dev;    /* [1] B_rem = B_act - B_exit */
-  int32_t* n_surv_host;   /* optional PINNED HOST [1]: receives the count by an async copy on the stream; valid once the
-                             caller has synchronised the stream (the "B_exit is communicated to the scheduler" step) */
+  int32_t* n_surv_host;   /* optional PINNED HOST [1]: receives the count by an async copy (the "B_exit is communicated
+                             to the scheduler" step).  The copy is issued as soon as the exit decisions are taken,
+                             beside the gather of the survivors' features, so the word is valid once the caller has
+                             synchronised the stream, or earlier: see ee_wait_count */
 } ee_stage_out_t;
 
 /* Runs stage `stage` on a batch: every layer of the subnet (convolutions as implicit GEMM with the
@@ -235,6 +237,13 @@ typedef struct {
   int launches; /* kernels this layer launches at this batch size */
 } ee_layer_plan_t;
 ee_status_t ee_model_plan(const ee_model_t* model, int stage, int batch, int cap, ee_layer_plan_t* out, int* n);
+
+/* Host-side wait for a survivor count without synchronising the stream (Section III, step 4: the scheduler needs
+ * B_exit, not the features, to size its next launch).  Protocol: the caller stores `sentinel` (a negative value) in
+ * its pinned word, passes the word as n_surv_host to ee_stage_run, then calls this: it polls the word until it differs
+ * from the sentinel and returns the value in *value.  Work enqueued on the stream afterwards is still ordered behind
+ * the stage by the stream.  Errors: INVALID_ARG; TIMEOUT when `timeout_s` seconds pass first (*value untouched). */
+ee_status_t ee_wait_count(const int32_t* n_surv_host, int32_t sentinel, double timeout_s, int32_t* value);
 
 /* Synchronises the stream and reports device-side faults the kernels recorded instead of hanging:
  * EE_ERR_TIMEOUT when a bounded wait on a barrier ran out.  The flag is cleared by the call. */

@@ -21,7 +21,7 @@ STATUS_NAMES = ["EE_OK", "EE_ERR_INVALID_ARG", "EE_ERR_SHAPE", "EE_ERR_CAPACITY"
                 "EE_ERR_CUDA", "EE_ERR_TIMEOUT", "EE_ERR_INTERNAL"]
 EXPORTS = ["ee_model_create", "ee_model_destroy", "ee_model_query", "ee_stage_run", "ee_layer_run", "ee_batch_refill", "ee_exit_head",
            "ee_exit_head_scratch_bytes", "ee_exit_head_static", "ee_gather_survivors", "ee_model_set_graphs", "ee_model_set_timing", "ee_model_get_timing",
-           "ee_model_plan", "ee_model_check", "ee_status_string", "ee_last_cuda_error"]
+           "ee_model_plan", "ee_model_check", "ee_wait_count", "ee_status_string", "ee_last_cuda_error"]
 
 
 class EEError(RuntimeError):
@@ -96,6 +96,7 @@ def load_library() -> C.CDLL:
     L.ee_model_set_timing.argtypes = [vp, i]
     L.ee_model_get_timing.argtypes = [vp, i, i, C.POINTER(C.c_float), C.POINTER(C.c_char_p), C.POINTER(i)]
     L.ee_model_plan.argtypes = [vp, i, i, i, C.POINTER(LayerPlan), C.POINTER(i)]
+    L.ee_wait_count.argtypes = [vp, C.c_int32, C.c_double, C.POINTER(C.c_int32)]
     L.ee_model_check.argtypes = [vp, vp]
     L.ee_status_string.argtypes = [i]
     L.ee_status_string.restype = C.c_char_p
@@ -146,6 +147,18 @@ class StageBuffers:
         self.ids_out = torch.empty(B, dtype=torch.int32, device=dev)
         self.n_surv_dev = torch.zeros(1, dtype=torch.int32, device=dev)
         self.n_surv_host = torch.zeros(1, dtype=torch.int32).pin_memory() if pinned_count else None
+        self._count_word = C.c_int32.from_address(self.n_surv_host.data_ptr()) if pinned_count else None
+
+    def arm_count(self):
+        """Stores the sentinel -1 in the pinned count word; call before ee_stage_run, then wait_count()."""
+        self._count_word.value = -1
+
+    def wait_count(self, timeout_s: float = 10.0) -> int:
+        """B_rem of the stage launched after arm_count(), as soon as the exit decisions are taken (ee_wait_count):
+        the stream is not synchronised and the gather of the survivors' features may still be running."""
+        v = C.c_int32(-1)
+        _check(load_library().ee_wait_count(self.n_surv_host.data_ptr(), -1, float(timeout_s), C.byref(v)), "ee_wait_count")
+        return int(v.value)
 
     def as_struct(self) -> StageOut:
         return StageOut(_ptr(self.features_out), _ptr(self.conf), _ptr(self.pred), _ptr(self.logits), _ptr(self.exit_mask),

@@ -1,5 +1,6 @@
 // C ABI of the early-exit CNN stage executor: model creation (weight upload, per-layer kernel
 // plan, workspace layout), ee_stage_run, ee_batch_refill and the stand-alone head / gather calls.
+#include <chrono>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -126,6 +127,9 @@ struct ee_model {
   bool timing = false;
   bool graphs = true;  // replay stages as CUDA graphs on capturable streams
   TcContext tc;
+  // the survivor count travels to the host on a side branch, beside the gather of the survivors' features
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 
 namespace {
@@ -309,12 +313,24 @@ ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, c
                       ? launch_head<bf16>(m, sp, so, B, hw, in->logit_shift, in->shift_class, ws + sp.head_off, in, out, st, true)
                       : launch_head<float>(m, sp, so, B, hw, in->logit_shift, in->shift_class, ws + sp.head_off, in, out, st, true);
   if (s != EE_OK) return s;
+  // B_exit goes to the host as soon as the decisions are taken: the copy runs on a side branch (also when the stage
+  // is captured into a graph) while the survivors' features are gathered, and rejoins the stream behind the gather.
+  const bool fork = out->n_surv_host && !sp.always_exit;
+  if (fork) {
+    EE_CUDA(cudaEventRecord(m->ev_fork, st));
+    EE_CUDA(cudaStreamWaitEvent(m->side, m->ev_fork, 0));
+    EE_CUDA(cudaMemcpyAsync(out->n_surv_host, out->n_surv_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, m->side));
+    EE_CUDA(cudaEventRecord(m->ev_join, m->side));
+  }
   if (!sp.always_exit) {
     s = gather_launch(so, (size_t)hw * sp.out_c * esize(m->dtype), out->survivor_idx, out->n_surv_dev, B, out->features_out, st);
     if (s != EE_OK) return s;
     record(m, sp, st, "gather_survivors");
   }
-  if (out->n_surv_host) EE_CUDA(cudaMemcpyAsync(out->n_surv_host, out->n_surv_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  if (fork)
+    EE_CUDA(cudaStreamWaitEvent(st, m->ev_join, 0));
+  else if (out->n_surv_host)
+    EE_CUDA(cudaMemcpyAsync(out->n_surv_host, out->n_surv_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
   return EE_OK;
 }
 
@@ -350,6 +366,9 @@ ee_status_t ee_model_destroy(ee_model_t* m) {
     for (auto& g : sp.graphs) cudaGraphExecDestroy(g.exec);
   }
   for (void* p : m->owned) cudaFree(p);
+  if (m->ev_fork) cudaEventDestroy(m->ev_fork);
+  if (m->ev_join) cudaEventDestroy(m->ev_join);
+  if (m->side) cudaStreamDestroy(m->side);
   delete m;
   return EE_OK;
 }
@@ -381,6 +400,10 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
     m->err_flag = (int*)p;
     if (cudaMemsetAsync(p, 0, 256, st) != cudaSuccess) return fail(EE_ERR_CUDA);
   }
+  if (cudaStreamCreateWithFlags(&m->side, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&m->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming) != cudaSuccess)
+    return fail(EE_ERR_CUDA);
   rc = tc_context_init(m->tc);
   if (rc == EE_OK) rc = stem_context_init();
   if (rc == EE_OK) rc = halo_context_init();
@@ -546,6 +569,21 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
   if (cudaStreamSynchronize(st) != cudaSuccess) return fail(EE_ERR_CUDA);
   *out = m;
   return EE_OK;
+}
+
+ee_status_t ee_wait_count(const int32_t* n_surv_host, int32_t sentinel, double timeout_s, int32_t* value) {
+  if (!n_surv_host || !value || timeout_s < 0) return EE_ERR_INVALID_ARG;
+  const volatile int32_t* w = n_surv_host;
+  const auto t0 = std::chrono::steady_clock::now();
+  for (unsigned spin = 0;; ++spin) {
+    const int32_t v = *w;
+    if (v != sentinel) {
+      *value = v;
+      return EE_OK;
+    }
+    if ((spin & 1023u) == 1023u && std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count() > timeout_s)
+      return EE_ERR_TIMEOUT;
+  }
 }
 
 ee_status_t ee_model_query(const ee_model_t* m, int stage, ee_stage_info_t* out) {

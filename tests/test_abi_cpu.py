@@ -35,6 +35,23 @@ def test_status_strings_without_a_device():
     assert lib.ee_last_cuda_error() == b""
 
 
+def test_wait_count_returns_the_value_or_times_out():
+    """ee_wait_count is host-only: it polls a word until it leaves the sentinel (here a thread plays the GPU's copy)."""
+    import threading
+    import time
+
+    lib = eb.load_library()
+    word = ctypes.c_int32(-1)
+    out = ctypes.c_int32(-7)
+    assert lib.ee_wait_count(ctypes.addressof(word), -1, 0.05, ctypes.byref(out)) == eb.STATUS_NAMES.index("EE_ERR_TIMEOUT")
+    assert out.value == -7                                   # untouched on timeout
+    t = threading.Thread(target=lambda: (time.sleep(0.02), setattr(word, "value", 5)))
+    t.start()
+    assert lib.ee_wait_count(ctypes.addressof(word), -1, 5.0, ctypes.byref(out)) == 0 and out.value == 5
+    t.join()
+    assert lib.ee_wait_count(None, -1, 1.0, ctypes.byref(out)) == eb.STATUS_NAMES.index("EE_ERR_INVALID_ARG")
+
+
 def test_binding_structs_follow_the_header():
     src = open(os.path.join(ROOT, "include", "ee.h")).read()
 

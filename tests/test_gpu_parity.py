@@ -471,3 +471,28 @@ def test_stage_replay_as_graph_is_bit_identical():
     ref_b = snapshot()
     assert got_b[0] == ref_b[0] and all(torch.equal(g, r) for g, r in zip(got_b[1:], ref_b[1:]))
     m.check()
+
+
+def test_count_reaches_the_host_without_a_stream_sync():
+    """B_exit is copied to the pinned word beside the gather (plain launches and graph replay): ee_wait_count returns it
+    without synchronising the stream, and it equals the count of the synchronised run."""
+    spec = wl.resnet50_ee(seed=1, in_hw=64, n_classes=100, max_batch=6)
+    run = util.GpuRunner(spec)
+    m, out, ws = run.m, run.bufs[0], run.ws
+    B = 6
+    x = eb.to_device("bf16", wl.make_input(spec, B, seed=3))
+    ids = torch.arange(B, dtype=torch.int32, device="cuda")
+    m.set_graphs(False)
+    m.stage_run(0, x, B, out, ws, ids)
+    torch.cuda.synchronize()
+    want = int(out.n_surv_host[0])
+    assert want == B - int(out.exit_mask[:B].sum().item())
+    m.set_graphs(True)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for _ in range(3):                                   # plain capture call, then replays
+            out.arm_count()
+            m.stage_run(0, x, B, out, ws, ids)
+            assert out.wait_count(5.0) == want
+        torch.cuda.synchronize()
+    m.check()
