@@ -211,6 +211,13 @@ ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const
       break;
     }
     case KK_POOL: {
+      if constexpr (sizeof(T) == 2) {
+        if (dw_tma_supported(g, src, nullptr, dst)) {
+          ee_status_t s = dw_tma_launch(m->tc, L.tc, g, src, nullptr, nullptr, nullptr, dst, m->err_flag, st);
+          if (s != EE_OK) return s;
+          break;
+        }
+      }
       const bool vec = L.d.cin % V == 0;
       const long total = (long)B * L.out_h * L.out_w * (vec ? L.d.cin / V : L.d.cin);
       const int grid = (int)std::min<long>(cdiv(total, 256), 148L * 32);

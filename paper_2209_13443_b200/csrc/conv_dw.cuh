@@ -5,7 +5,7 @@
 // flight.  A kernel that loads through registers holds one item's inputs per thread and stalls on every item.  Here
 // one producer warp per persistent CTA asks the TMA unit for whole input tiles, a band of output rows x all columns x
 // one block of up to 64 channels, including the one-pixel frame of the padding (coordinates start at -1; the unit
-// zero-fills outside the image), into a ring of three slots: two or three tiles (up to 48 KB each) are in flight per
+// zero-fills outside the image), into a ring of three slots: two or three tiles (up to 72 KB each) are in flight per
 // SM whatever the consumers do.  Eight consumer warps compute from shared memory: a thread owns one vector of eight
 // channels (its 72 weights stay in registers as stored) and walks strips of four consecutive output pixels of the
 // tile, reading each of the 3 x 6 (stride 2: 3 x 9) input vectors of a strip once.  A quarter warp reads the eight
@@ -35,7 +35,7 @@ struct DwParams {
 constexpr int kDwStages = 3;
 constexpr int kDwConsumers = 256;
 constexpr int kDwThreads = 32 + kDwConsumers;
-constexpr int kDwMaxTileBytes = 48 * 1024;
+constexpr int kDwMaxTileBytes = 72 * 1024;
 
 __device__ __forceinline__ void tma_load_4d_tile(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2, int c3) {
   asm volatile(
@@ -44,7 +44,9 @@ __device__ __forceinline__ void tma_load_4d_tile(uint32_t dst, const CUtensorMap
       : "memory");
 }
 
-template <int STRIDE>
+// POOL: the same staging for a 3x3 pad-1 window maximum (the max-pool behind a ResNet-style stem): taps outside the
+// image are skipped (the frame's zeros must not win against negative inputs), no weights, no epilogue arithmetic.
+template <int STRIDE, bool POOL>
 __global__ void __launch_bounds__(kDwThreads, 1)
 dwconv3x3_tma_kernel(const __grid_constant__ CUtensorMap tmX, DwParams p) {
   constexpr int P = kDwStrip, COLS = (P - 1) * STRIDE + 3;
@@ -96,7 +98,7 @@ dwconv3x3_tma_kernel(const __grid_constant__ CUtensorMap tmX, DwParams p) {
   uint32_t wr[36];   // the vector's 72 weights as stored: element e = channel e / 9, tap e % 9
 #pragma unroll
   for (int i = 0; i < 9; ++i) {
-    const uint4 v = c_in ? __ldg(reinterpret_cast<const uint4*>(p.w + (size_t)c * 9) + i) : make_uint4(0u, 0u, 0u, 0u);
+    const uint4 v = (!POOL && c_in) ? __ldg(reinterpret_cast<const uint4*>(p.w + (size_t)c * 9) + i) : make_uint4(0u, 0u, 0u, 0u);
     wr[4 * i] = v.x, wr[4 * i + 1] = v.y, wr[4 * i + 2] = v.z, wr[4 * i + 3] = v.w;
   }
   auto weight = [&](int tap, int ch) {   // indices are compile-time constants after unrolling
@@ -137,9 +139,11 @@ dwconv3x3_tma_kernel(const __grid_constant__ CUtensorMap tmX, DwParams p) {
 #pragma unroll
         for (int pp = 0; pp < P; ++pp)
 #pragma unroll
-          for (int e = 0; e < 8; ++e) acc[pp][e] = 0.f;
+          for (int e = 0; e < 8; ++e) acc[pp][e] = POOL ? -INFINITY : 0.f;
 #pragma unroll
         for (int r = 0; r < 3; ++r) {
+          const int hi = ho * STRIDE - 1 + r;
+          const bool row_in = hi >= 0 && hi < p.H;
 #pragma unroll
           for (int q = 0; q < COLS; ++q) {
             const uint32_t wd[4] = {v[r][q].x, v[r][q].y, v[r][q].z, v[r][q].w};
@@ -153,8 +157,16 @@ dwconv3x3_tma_kernel(const __grid_constant__ CUtensorMap tmX, DwParams p) {
             for (int pp = 0; pp < P; ++pp) {
               const int sx = q - pp * STRIDE;   // compile-time after unrolling
               if (sx >= 0 && sx < 3) {
+                if constexpr (POOL) {
+                  const int wi = wo0 * STRIDE - 1 + q;
+                  if (row_in && wi >= 0 && wi < p.W) {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[pp][e] = fmaf(f[e], weight(r * 3 + sx, e), acc[pp][e]);
+                    for (int e = 0; e < 8; ++e) acc[pp][e] = fmaxf(acc[pp][e], f[e]);
+                  }
+                } else {
+#pragma unroll
+                  for (int e = 0; e < 8; ++e) acc[pp][e] = fmaf(f[e], weight(r * 3 + sx, e), acc[pp][e]);
+                }
               }
             }
           }
@@ -166,7 +178,7 @@ dwconv3x3_tma_kernel(const __grid_constant__ CUtensorMap tmX, DwParams p) {
             if (wo0 + pp < p.Wo) {
               Vec16<bf16> o;
 #pragma unroll
-              for (int e = 0; e < 8; ++e) o.v[e] = apply_act(fmaf(sc[e], acc[pp][e], bi[e]), p.act);
+              for (int e = 0; e < 8; ++e) o.v[e] = POOL ? acc[pp][e] : apply_act(fmaf(sc[e], acc[pp][e], bi[e]), p.act);
               o.store(yp + (size_t)pp * p.C);
             }
           }
@@ -178,8 +190,8 @@ dwconv3x3_tma_kernel(const __grid_constant__ CUtensorMap tmX, DwParams p) {
   }
 }
 
-// Layers this kernel takes: depthwise 3x3, pad 1, stride 1 or 2, channels a multiple of 8, at most 254 columns, and a
-// tile of one output row that fits a ring slot.
+// Layers this kernel takes: depthwise 3x3 (or a 3x3 max-pool, w == nullptr), pad 1, stride 1 or 2, channels a multiple
+// of 8, at most 254 columns, and a tile of one output row that fits a ring slot.
 inline bool dw_tma_supported(const ConvGeom& g, const void* x, const void* w, const void* y) {
   if (!(g.kh == 3 && g.kw == 3 && g.pad == 1 && (g.stride == 1 || g.stride == 2) && g.Cin % 8 == 0 && g.Cin == g.Cout)) return false;
   if ((((uintptr_t)x | (uintptr_t)w | (uintptr_t)y) & 15) != 0 || g.W + 2 > 256) return false;
@@ -189,8 +201,10 @@ inline bool dw_tma_supported(const ConvGeom& g, const void* x, const void* w, co
 
 inline ee_status_t dw_context_init() {
   const int bytes = kDwStages * kDwMaxTileBytes + 256 + 128;
-  cudaError_t e = cudaFuncSetAttribute(dwconv3x3_tma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(dwconv3x3_tma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  cudaError_t e = cudaFuncSetAttribute(dwconv3x3_tma_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(dwconv3x3_tma_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(dwconv3x3_tma_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(dwconv3x3_tma_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   return e == cudaSuccess ? EE_OK : EE_ERR_CUDA;
 }
 
@@ -259,7 +273,11 @@ inline ee_status_t dw_tma_launch(TcContext& c, const TcLayer& L, const ConvGeom&
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  cudaError_t e = g.stride == 1 ? cudaLaunchKernelEx(&cfg, dwconv3x3_tma_kernel<1>, tmX, p) : cudaLaunchKernelEx(&cfg, dwconv3x3_tma_kernel<2>, tmX, p);
+  cudaError_t e;
+  if (w)
+    e = g.stride == 1 ? cudaLaunchKernelEx(&cfg, dwconv3x3_tma_kernel<1, false>, tmX, p) : cudaLaunchKernelEx(&cfg, dwconv3x3_tma_kernel<2, false>, tmX, p);
+  else
+    e = g.stride == 1 ? cudaLaunchKernelEx(&cfg, dwconv3x3_tma_kernel<1, true>, tmX, p) : cudaLaunchKernelEx(&cfg, dwconv3x3_tma_kernel<2, true>, tmX, p);
   return e == cudaSuccess ? EE_OK : EE_ERR_CUDA;
 }
 
