@@ -209,13 +209,22 @@ def run_sample_serial(model, x1, shifts=None, shift_cls=None):
     raise AssertionError("final exit must always be taken")
 
 
-def serve_trace(n_stages, max_batch, arrivals, exit_of, stage_time):
-    """Algorithm 1 with T_SLO = infinity on a virtual clock (backfill whenever the queue is
-    non-empty and the batch has room; per exit, non-recursive).
+def serve_trace(n_stages, max_batch, arrivals, exit_of, stage_time, slo=float("inf")):
+    """Algorithm 1 on a virtual clock: exit-aware preemptive scheduling with the SLO-aware
+    preemption criterion (Eq. 3-4); backfilling per exit, non-recursive.
 
     ``arrivals``  sorted arrival times; request r has id r.
     ``exit_of``   exit index at which request r leaves (from ``run_sample_serial``).
-    ``stage_time(stage, batch)`` service time of one subnet at a batch size.
+    ``stage_time(stage, batch)`` service time of one subnet at a batch size; it is also the
+                  exit-level latency table the criterion looks up (Section III-B, Exit-Level
+                  Latency Prediction), so on this clock the prediction is exact.
+    ``slo``       T_SLO in the unit of ``arrivals``.  At the preemption point behind exit i, with
+                  B_rem samples left, B_incr = min(N_Q, B_max - B_rem) > 0 candidates queued:
+                    T_slack    = T_SLO - (now - arrival of the oldest sample of the active batch)   (Eq. 3)
+                    T_overhead = T_{0:i}(B_incr) + T_{i+1:L-1}(B_rem + B_incr)                     (Eq. 4)
+                  and the batch is preempted iff T_overhead < T_slack.  An active batch that has
+                  lost all its samples constrains nothing (its slack is infinite).  With
+                  slo = inf every backfill that fits is taken.
     Returns (finish_time per request, list of (stage, ids tuple) launches in order)."""
     n = len(arrivals)
     finish = np.zeros(n)
@@ -241,6 +250,13 @@ def serve_trace(n_stages, max_batch, arrivals, exit_of, stage_time):
                 rem.append(r)
         return rem, now
 
+    def span(first, last, batch):
+        """T_{first:last}^{batch}: subnets first..last (inclusive) at one batch size."""
+        total = 0.0
+        for j in range(first, last + 1):
+            total += stage_time(j, batch)
+        return total
+
     while nxt < n or q:
         admit(t)
         if not q:
@@ -255,6 +271,12 @@ def serve_trace(n_stages, max_batch, arrivals, exit_of, stage_time):
                 incr = min(len(q), max_batch - len(act))
                 if incr == 0:
                     break
+                if act:
+                    oldest = min(arrivals[r] for r in act)
+                    t_slack = slo - (t - oldest)
+                    t_overhead = span(0, i, incr) + span(i + 1, n_stages - 1, len(act) + incr)
+                    if not t_overhead < t_slack:
+                        break
                 new = [q.popleft() for _ in range(incr)]
                 for j in range(i + 1):          # the new batch catches up to exit i
                     new, t = proc(j, new, t)

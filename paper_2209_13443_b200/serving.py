@@ -1,12 +1,15 @@
 """Host-side serving loop over the C-ABI library: the exit-aware preemptive scheduling method
-(Algorithm 1) with T_SLO = infinity.
+(Algorithm 1) with its SLO-aware preemption criterion (Eq. 3-4).
 
 At every exit the scheduler learns B_exit, and while the batch has room and the queue is not
 empty it preempts the active batch (which simply stays parked in its HBM buffer: activations are
 already in device memory, Section III-B "Overhead"), lets B_incr = min(N_Q, B_max - B_rem) new
 requests catch up to the same exit, and merges them (B_merged = B_rem + B_incr - B_exit).
-Backfilling is per exit and non-recursive.  The SLO-aware criterion (Eq. 3-4) is not evaluated:
-every backfill that fits is taken.
+Backfilling is per exit and non-recursive.  A backfill is taken only if it cannot push the oldest
+sample of the active batch past the latency SLO: T_overhead = T_{0:i}(B_incr) + T_{i+1:L-1}(B_merged)
+must be below T_slack = T_SLO - (T_wait + T_exec so far).  The exit-level latencies come from a
+N_exits x B_max table measured on the device (``measure_latency_table``; Section III-B, Exit-Level
+Latency Prediction).  With T_SLO = infinity every backfill that fits is taken.
 
 All device work goes through ``ee_stage_run`` / ``ee_batch_refill`` / ``ee_gather_survivors``;
 this file only keeps the queue, the clocks and the bookkeeping.
@@ -43,6 +46,25 @@ class FluidServer:
         self.cnt_dev = torch.empty(1, dtype=torch.int32, device="cuda")
         self.stage_in_bytes = [self.m.query(s)["in_bytes_per_sample"] for s in range(self.n_stages)]
 
+    def measure_latency_table(self, reps: int = 5) -> np.ndarray:
+        """The N_exits x B_max look-up table of the scheduler: seconds one ee_stage_run of subnet s takes at batch
+        b (CUDA events around ``reps`` replays on random features; column b - 1 holds batch b)."""
+        lut = np.zeros((self.n_stages, self.bmax))
+        td = eb.torch_dtype(self.spec.dtype)
+        a, b_ev = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for s in range(self.n_stages):
+            qi = self.m.query(s)
+            x = (torch.randn(self.bmax, qi["in_h"], qi["in_w"], qi["in_c"], device="cuda") * 0.5).to(td)
+            for b in range(1, self.bmax + 1):
+                self.m.stage_run(s, x, b, self.new[s], self.ws, self.ids_new)        # first call: plain launches / capture
+                a.record()
+                for _ in range(reps):
+                    self.m.stage_run(s, x, b, self.new[s], self.ws, self.ids_new)
+                b_ev.record()
+                b_ev.synchronize()
+                lut[s, b - 1] = a.elapsed_time(b_ev) * 1e-3 / reps
+        return lut
+
     def _form_batch(self, pool, rows: Sequence[int], req_ids: Sequence[int], feat, ids):
         """Copies the requested pool images into the front of ``feat`` (the batch buffer)."""
         n = len(rows)
@@ -72,13 +94,23 @@ class FluidServer:
         return rem, now
 
     def serve(self, arrivals: np.ndarray, image_of: Sequence[int], pool: torch.Tensor,
-              stage_time: Optional[Callable[[int, int], float]] = None):
+              stage_time: Optional[Callable[[int, int], float]] = None, slo: float = float("inf"),
+              latency: Optional[Callable[[int, int], float]] = None):
         """Serves requests r = 0..n-1 arriving at ``arrivals[r]`` (sorted, seconds) and carrying image
         ``pool[image_of[r]]``.  With ``stage_time(stage, batch)`` the clock is virtual (deterministic batch
         compositions); without it the wall clock is used and the loop waits for arrivals.
-        Returns dict(finish, exit_stage, pred, launches)."""
+        ``slo`` is T_SLO in seconds; ``latency(stage, batch)`` is the exit-level latency table the preemption
+        criterion consults (default: ``stage_time``; required on the wall clock when ``slo`` is finite).
+        Returns dict(finish, exit_stage, pred, launches, preemptions, declined)."""
         n = len(arrivals)
-        out = {"finish": np.zeros(n), "exit_stage": np.full(n, -1), "pred": np.full(n, -1), "launches": []}
+        out = {"finish": np.zeros(n), "exit_stage": np.full(n, -1), "pred": np.full(n, -1), "launches": [],
+               "preemptions": 0, "declined": 0}
+        latency = latency or stage_time
+        if np.isfinite(slo) and latency is None:
+            raise ValueError("a finite SLO needs the exit-level latency table (latency=...)")
+
+        def span(first, last, batch):           # T_{first:last}^{batch}
+            return sum(latency(j, batch) for j in range(first, last + 1))
         q: deque = deque()
         nxt = 0
         t0 = time.perf_counter()
@@ -115,6 +147,13 @@ class FluidServer:
                     incr = min(len(q), self.bmax - len(act))                    # B_incr = min(N_Q, B_slack)
                     if incr == 0:
                         break
+                    if act and np.isfinite(slo):                                 # SLO-aware preemption criterion
+                        t_slack = slo - (t - min(arrivals[r] for r in act))      # Eq. 3, oldest sample of the active batch
+                        t_overhead = span(0, i, incr) + span(i + 1, self.n_stages - 1, len(act) + incr)   # Eq. 4
+                        if not t_overhead < t_slack:
+                            out["declined"] += 1
+                            break
+                    out["preemptions"] += 1
                     new = [q.popleft() for _ in range(incr)]
                     self._form_batch(pool, [image_of[r] for r in new], new, self.in_new, self.ids_new)
                     nfeat, nids = self.in_new, self.ids_new

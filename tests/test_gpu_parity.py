@@ -434,6 +434,15 @@ def test_streaming_trace_matches_oracle_schedule():
     assert got["pred"].tolist() == [serial[image_of[r]][1] for r in range(n)]
     np.testing.assert_allclose(got["finish"], fin, rtol=0, atol=1e-9)
     assert len({len(ids) for _, ids in launches}) > 3                          # the trace exercises varying batch sizes
+    # the same trace under the SLO-aware preemption criterion (Eq. 3-4): some backfills are declined, and the server
+    # takes exactly the decisions of the oracle-side replay
+    for slo in (1.2e-3, 2.5e-3):
+        got = srv.serve(arrivals, image_of, eb.to_device("f32", pool_np), stage_time, slo=slo)
+        fin, launches_slo = eo.serve_trace(3, spec.max_batch, arrivals, exit_of, stage_time, slo=slo)
+        assert got["launches"] == launches_slo and got["declined"] > 0
+        assert np.array_equal(got["exit_stage"], exit_of)
+        np.testing.assert_allclose(got["finish"], fin, rtol=0, atol=1e-9)
+    assert launches_slo != launches
 
 
 def test_stage_replay_as_graph_is_bit_identical():

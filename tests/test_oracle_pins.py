@@ -333,3 +333,72 @@ def test_serve_trace_bookkeeping():
             assert seen.get(r, -1) == stage - 1                      # stages visited in order, once
             seen[r] = stage
     assert all(seen[r] == exit_of[r] for r in range(n))              # every request leaves at its exit
+
+
+# ----------------------------------------------------------------------------- SLO-aware preemption criterion (Eq. 3-4)
+
+def test_slo_criterion_worked_example():
+    """Hand-computed from Eq. 3-4.  Three subnets of 1 time unit each at any batch, B_max = 4; request 0 arrives at
+    t = 0, request 1 at t = 0.5, both leave at the last exit.  At the first preemption point (t = 1) one request is
+    queued: T_slack = T_SLO - 1, T_overhead = T_{0:0}(1) + T_{1:2}(2) = 3, so the batch is preempted iff T_SLO > 4.
+    T_SLO = 4.5: request 1 catches up (t = 2), the merged pair finishes at t = 4.
+    T_SLO = 4 (3 < 3 is false: strict inequality): request 0 runs on; at the second point (t = 2) T_slack = 2,
+    T_overhead = T_{0:1}(1) + T_{2:2}(2) = 3: declined again; request 0 finishes at 3, request 1 runs alone, done at 6."""
+    arr = np.array([0.0, 0.5])
+    exit_of = np.array([2, 2])
+    unit = lambda s, b: 1.0   # noqa: E731
+    fin, launches = eo.serve_trace(3, 4, arr, exit_of, unit, slo=4.5)
+    assert launches == [(0, (0,)), (0, (1,)), (1, (0, 1)), (2, (0, 1))] and fin.tolist() == [4.0, 4.0]
+    fin, launches = eo.serve_trace(3, 4, arr, exit_of, unit, slo=4.0)
+    assert launches == [(0, (0,)), (1, (0,)), (2, (0,)), (0, (1,)), (1, (1,)), (2, (1,))] and fin.tolist() == [3.0, 6.0]
+    # a subnet that takes `batch` time units tells the two batch sizes of Eq. 4 apart: at t = 1,
+    # T_overhead = T_{0:0}(B_incr = 1) + T_{1:2}(B_merged = 2) = 1 + 4 = 5 and T_slack = T_SLO - 1: preempt iff T_SLO > 6
+    by_batch = lambda s, b: float(b)   # noqa: E731
+    fin, launches = eo.serve_trace(3, 4, arr, exit_of, by_batch, slo=6.5)
+    assert launches == [(0, (0,)), (0, (1,)), (1, (0, 1)), (2, (0, 1))] and fin.tolist() == [6.0, 6.0]
+    fin, launches = eo.serve_trace(3, 4, arr, exit_of, by_batch, slo=5.0)   # second point: slack 3 against 2 + 2: declined
+    assert launches == [(0, (0,)), (1, (0,)), (2, (0,)), (0, (1,)), (1, (1,)), (2, (1,))] and fin.tolist() == [3.0, 6.0]
+
+
+def _random_trace(seed, n=300, rate=1500.0, n_stages=4):
+    arr = wl.poisson_arrivals(seed, n, rate)
+    exit_of = np.random.default_rng(seed).integers(0, n_stages, n)
+    return arr, exit_of
+
+
+def test_slo_infinite_is_plain_backfilling_and_zero_never_preempts():
+    st = lambda s, b: 2e-4 * (s + 1) + 3e-5 * b   # noqa: E731
+    arr, exit_of = _random_trace(11)
+    ref = eo.serve_trace(4, 8, arr, exit_of, st)
+    big = eo.serve_trace(4, 8, arr, exit_of, st, slo=1e9)
+    assert ref[1] == big[1] and np.array_equal(ref[0], big[0])
+    # T_SLO = 0: the slack of a non-empty active batch is never positive, so a batch with survivors is never preempted:
+    # between two consecutive subnets of a surviving batch nothing else is launched
+    _, launches = eo.serve_trace(4, 8, arr, exit_of, st, slo=0.0)
+    for (s0, ids0), (s1, ids1) in zip(launches, launches[1:]):
+        rem = [r for r in ids0 if exit_of[r] != s0]
+        if rem:
+            assert s1 == s0 + 1 and list(ids1) == rem
+
+
+@pytest.mark.parametrize("slo", [4e-3, 8e-3, 16e-3])
+def test_slo_criterion_never_pushes_a_preempted_sample_past_its_slo(slo):
+    """The overhead estimate is an upper bound when a subnet is not slower at a smaller batch (Section III-B): a sample
+    whose batch was preempted (something ran between two of its consecutive subnets) still meets the SLO."""
+    st = lambda s, b: 2e-4 * (s + 1) + 3e-5 * b   # noqa: E731
+    checked = 0
+    for seed in (1, 2, 3):
+        arr, exit_of = _random_trace(seed)
+        fin, launches = eo.serve_trace(4, 8, arr, exit_of, st, slo=slo)
+        last = {}                                   # request -> index of its latest launch
+        preempted = set()
+        for k, (s, ids) in enumerate(launches):
+            for r in ids:
+                if s > 0 and last[r] != k - 1:
+                    preempted.add(r)
+                last[r] = k
+        assert all(exit_of[r] == launches[last[r]][0] for r in range(len(arr)))
+        for r in preempted:
+            assert fin[r] - arr[r] <= slo + 1e-12, (seed, r, fin[r] - arr[r])
+        checked += len(preempted)
+    assert checked > 20                              # the traces do exercise preemptions at these SLOs
