@@ -538,7 +538,33 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
         L.kind = KK_DW;
       } else if (desc->dtype == EE_BF16 && tc_supported(d, L.in_h, L.in_w)) {
         L.kind = KK_TC;
-        rc = tc_plan_layer(m->tc, d, L.in_h, L.in_w, L.out_h, L.out_w, desc->max_batch, L.w_dev, &L.tc);
+        const int g = pixel_group(d, L.in_h * L.in_w);
+        if (g > 1) {   // narrow 1x1 layer: g pixels per row, block-diagonal weights, scale / bias repeated per pixel
+          void* wp = nullptr;
+          float *sp2 = nullptr, *bp2 = nullptr;
+          if (cudaMalloc(&wp, (size_t)g * d.cout * g * d.cin * 2) != cudaSuccess) return fail(EE_ERR_CUDA);
+          m->owned.push_back(wp);
+          pack_grouped_weights_kernel<<<cdiv((long)g * d.cout * g * d.cin, 256), 256, 0, st>>>((const bf16*)L.w_dev, (bf16*)wp, d.cout, d.cin, g);
+          if (L.scale_dev) {
+            if (cudaMalloc((void**)&sp2, (size_t)g * d.cout * 4) != cudaSuccess) return fail(EE_ERR_CUDA);
+            m->owned.push_back(sp2);
+            replicate_kernel<<<cdiv((long)g * d.cout, 256), 256, 0, st>>>(L.scale_dev, sp2, d.cout, g);
+            L.scale_dev = sp2;
+          }
+          if (L.bias_dev) {
+            if (cudaMalloc((void**)&bp2, (size_t)g * d.cout * 4) != cudaSuccess) return fail(EE_ERR_CUDA);
+            m->owned.push_back(bp2);
+            replicate_kernel<<<cdiv((long)g * d.cout, 256), 256, 0, st>>>(L.bias_dev, bp2, d.cout, g);
+            L.bias_dev = bp2;
+          }
+          if (cudaGetLastError() != cudaSuccess) return fail(EE_ERR_CUDA);
+          ee_layer_desc_t gd = d;
+          gd.cin = g * d.cin, gd.cout = g * d.cout;
+          const int rows = L.in_h * L.in_w / g;
+          rc = tc_plan_layer(m->tc, gd, 1, rows, 1, rows, desc->max_batch, wp, &L.tc);
+        } else {
+          rc = tc_plan_layer(m->tc, d, L.in_h, L.in_w, L.out_h, L.out_w, desc->max_batch, L.w_dev, &L.tc);
+        }
         if (rc != EE_OK) return fail(rc);
         L.tc.halo = halo_supported(d, L.in_w);
       } else if (desc->dtype == EE_BF16 && d.cout % 8 == 0 && d.kh * d.kw * d.cin <= 1024) {

@@ -186,16 +186,11 @@ conv3x3_halo_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
       if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acc_empty(b)) : "memory");
       if (inside && h0 + y < p.H) {
         bf16* dst = p.out + ((size_t)((size_t)n * p.H + h0 + y) * p.W + x) * p.N;
-        scale_bias<32>(va, s_scale, s_bias);
-        scale_bias<32>(vb, s_scale + 32, s_bias + 32);
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
           if (g * 8 < p.N) {
             const float* v = g < 4 ? va + g * 8 : vb + (g - 4) * 8;
-            Vec16<bf16> o;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) o.v[e] = apply_act(v[e], p.act);
-            o.store(dst + g * 8);
+            *reinterpret_cast<uint4*>(dst + g * 8) = epilogue8_act<false>(p.act, v, s_scale + g * 8, s_bias + g * 8, make_uint4(0u, 0u, 0u, 0u));
           }
         }
       }

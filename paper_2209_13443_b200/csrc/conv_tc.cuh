@@ -184,6 +184,67 @@ __device__ __forceinline__ void scale_bias(float* v, const float* scale, const f
   }
 }
 
+// Epilogue arithmetic of eight output channels of one pixel: y = act(scale * acc + bias (+ residual)), one rounding to
+// bf16, packed into 16 bytes.  Two fp32 FMAs per instruction (fma.rn.f32x2: two independent round-to-nearest FMAs, bit
+// for bit the scalar result), and for ReLU the clamp rides on the conversion (cvt.rn.relu.bf16x2.f32: negative -> 0,
+// then round; rounding is monotone and keeps 0, so this equals round(max(y, 0))).  scale / bias: 32-byte aligned
+// shared-memory rows every lane reads at the same address (broadcast).  res: eight bf16 of the residual operand.
+__device__ __forceinline__ void ffma2(float& x0, float& x1, float s0, float s1, float b0, float b1) {
+  asm("{\n .reg .b64 a, s, b, d;\n mov.b64 a, {%0, %1};\n mov.b64 s, {%2, %3};\n mov.b64 b, {%4, %5};\n fma.rn.f32x2 d, a, s, b;\n"
+      " mov.b64 {%0, %1}, d;\n}"
+      : "+f"(x0), "+f"(x1)
+      : "f"(s0), "f"(s1), "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2_relu(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+template <int ACT, bool RES>
+__device__ __forceinline__ uint4 epilogue8(const float* acc, const float* scale, const float* bias, uint4 res) {
+  const float4 s0 = *reinterpret_cast<const float4*>(scale), s1 = *reinterpret_cast<const float4*>(scale + 4);
+  const float4 b0 = *reinterpret_cast<const float4*>(bias), b1 = *reinterpret_cast<const float4*>(bias + 4);
+  float v[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) v[e] = acc[e];
+  ffma2(v[0], v[1], s0.x, s0.y, b0.x, b0.y);
+  ffma2(v[2], v[3], s0.z, s0.w, b0.z, b0.w);
+  ffma2(v[4], v[5], s1.x, s1.y, b1.x, b1.y);
+  ffma2(v[6], v[7], s1.z, s1.w, b1.z, b1.w);
+  if (RES) {
+    const uint32_t w[4] = {res.x, res.y, res.z, res.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {  // bf16 -> f32 is a 16-bit shift
+      v[2 * i] += __uint_as_float(w[i] << 16);
+      v[2 * i + 1] += __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+  uint32_t o[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    if (ACT == EE_ACT_RELU) {
+      o[i] = pack_bf16x2_relu(v[2 * i], v[2 * i + 1]);
+    } else if (ACT == EE_ACT_RELU6) {
+      o[i] = pack_bf16x2(fminf(fmaxf(v[2 * i], 0.f), 6.f), fminf(fmaxf(v[2 * i + 1], 0.f), 6.f));
+    } else {
+      o[i] = pack_bf16x2(v[2 * i], v[2 * i + 1]);
+    }
+  }
+  return make_uint4(o[0], o[1], o[2], o[3]);
+}
+// The same with the activation chosen at run time (one uniform branch per call site, not per element).
+template <bool RES>
+__device__ __forceinline__ uint4 epilogue8_act(int act, const float* acc, const float* scale, const float* bias, uint4 res) {
+  if (act == EE_ACT_RELU) return epilogue8<EE_ACT_RELU, RES>(acc, scale, bias, res);
+  if (act == EE_ACT_RELU6) return epilogue8<EE_ACT_RELU6, RES>(acc, scale, bias, res);
+  return epilogue8<EE_ACT_NONE, RES>(acc, scale, bias, res);
+}
+
 // ----------------------------------------------------------------------------- kernel
 
 // Gather-mode row builders (see the GATHER note on the kernel).  Thread `grow` writes row `grow` of the A tile of
@@ -507,20 +568,11 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
           const int c0 = h * 64 + sub * 32;
           float v[32];
           tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
-          scale_bias<32>(v, s_scale + c0, s_bias + c0);
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
-            bf16* chunk = reinterpret_cast<bf16*>(line + (((sub * 4 + g) ^ (lane & 7)) << 4));
-            if (RES) {
-              Vec16<bf16> r;
-              r.load(chunk);
-#pragma unroll
-              for (int e = 0; e < 8; ++e) v[g * 8 + e] += r.v[e];
-            }
-            Vec16<bf16> o;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) o.v[e] = apply_act(v[g * 8 + e], p.act);
-            o.store(chunk);
+            if (n0 + c0 + g * 8 >= p.N) break;   // columns past Cout: nothing to compute, the store clips them
+            uint4* chunk = reinterpret_cast<uint4*>(line + (((sub * 4 + g) ^ (lane & 7)) << 4));
+            *chunk = epilogue8_act<RES>(p.act, v + g * 8, s_scale + c0 + g * 8, s_bias + c0 + g * 8, RES ? *chunk : make_uint4(0u, 0u, 0u, 0u));
           }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the TMA unit
@@ -791,6 +843,10 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
       if (RES && ok) ok = __all_sync(0xffffffffu, mbar_wait(res_full(b), (uint32_t)(j >> 1) & 1u, p.err_flag));
       if (!ok) break;
       tc_fence_after();
+      if (!RES) {  // two staging tiles: all but this warp's latest store (tile j - 1, the other tile) must have been read
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        __syncwarp();
+      }
       const int ob = RES ? 0 : b;  // output staging tile of this tile
       uint8_t* io = gen + S::kOOff + ob * S::kIoBytes;
       const uint32_t io_s = base + S::kOOff + ob * S::kIoBytes;
@@ -817,27 +873,13 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
 #pragma unroll
         for (int sub = 0; sub < 2; ++sub) {
           const int c0 = h * 64 + sub * 32;
-          float* v = sub ? vb : va;
-          scale_bias<32>(v, sc + c0, sc + BN + c0);
+          const float* v = sub ? vb : va;
 #pragma unroll
           for (int gq = 0; gq < 4; ++gq) {
+            if (n0 + c0 + gq * 8 >= p.N) break;   // columns past Cout: nothing to compute, the store clips them
             const int off = h * 16384 + row * 128 + (((sub * 4 + gq) ^ (lane & 7)) << 4);
-            if (RES) {
-              Vec16<bf16> r;
-              r.load(reinterpret_cast<const bf16*>(rin + off));
-#pragma unroll
-              for (int e = 0; e < 8; ++e) v[gq * 8 + e] += r.v[e];
-            }
-            Vec16<bf16> o;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) o.v[e] = apply_act(v[gq * 8 + e], p.act);
-            o.store(reinterpret_cast<bf16*>(io + off));
-          }
-          if (!RES && h == h0 && sub == 0 && lane == 0 && pending) {
-            // One chunk into tile j, this warp's store of tile j - 1 has long finished reading its staging tile:
-            // confirm it (no stall in the steady state); it licenses the next iteration to overwrite that tile.
-            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-            pending = false;
+            const uint4 r = RES ? *reinterpret_cast<const uint4*>(rin + off) : make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(io + off) = epilogue8_act<RES>(p.act, v + gq * 8, sc + c0 + gq * 8, sc + BN + c0 + gq * 8, r);
           }
         }
       }
@@ -864,6 +906,34 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * BN) : "memory");
   }
+}
+
+// Pixel grouping for narrow 1x1 layers.  A pixel row of Cin <= 32 channels is 16-64 bytes, and a TMA box over such
+// rows moves one short row per request (a 16-channel layer loads at a quarter of the rate of a 64-channel one).  g
+// consecutive pixels are one contiguous row of g * Cin channels, so the layer is run as a 1x1 layer over M / g rows
+// with Cin' = g * Cin and Cout' = g * Cout and the block-diagonal weight matrix below: row (j, n) holds w[n][:] in
+// columns [j * Cin, (j + 1) * Cin) and zeros elsewhere.  Output row i, column j * Cout + n is channel n of pixel
+// g * i + j, which is exactly where the dense [M][Cout] output keeps it.  The zero blocks add g - 1 idle MMA passes
+// on layers that do not come near the tensor pipe's rate; each output is still the same sum of Cin products.
+__global__ void pack_grouped_weights_kernel(const bf16* __restrict__ w, bf16* __restrict__ out, int cout, int cin, int g) {
+  const long total = (long)g * cout * g * cin;
+  for (long idx = (long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long)gridDim.x * blockDim.x) {
+    const int col = (int)(idx % ((long)g * cin));
+    const int row = (int)(idx / ((long)g * cin));
+    const int j = row / cout, n = row - j * cout, jc = col / cin, c = col - jc * cin;
+    out[idx] = j == jc ? w[(long)n * cin + c] : __float2bfloat16_rn(0.f);
+  }
+}
+__global__ void replicate_kernel(const float* __restrict__ src, float* __restrict__ dst, int n, int g) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n * g; i += gridDim.x * blockDim.x) dst[i] = src[i % n];
+}
+// Pixels per row for a 1x1 / stride 1 / pad 0 layer on hw pixels per sample: the largest g with g * Cin <= 64 that
+// divides hw (so no row straddles two samples); 1 = leave the layer as it is.
+inline int pixel_group(const ee_layer_desc_t& d, int hw) {
+  if (!(d.kh == 1 && d.kw == 1 && d.stride == 1 && d.pad == 0) || d.cin > 32) return 1;
+  int g = kTcBK / d.cin;
+  while (g > 1 && hw % g != 0) --g;
+  return g;
 }
 
 // Gather mode: weight rows [Cout][kh][kw*Cin] copied into rows [Cout][kh][runp] padded to Kp columns, zeros elsewhere.
