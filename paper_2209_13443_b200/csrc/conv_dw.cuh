@@ -165,7 +165,11 @@ dwconv3x3_tma_kernel(const __grid_constant__ CUtensorMap tmX, DwParams p) {
                   }
                 } else {
 #pragma unroll
-                  for (int e = 0; e < 8; ++e) acc[pp][e] = fmaf(f[e], weight(r * 3 + sx, e), acc[pp][e]);
+                  for (int e = 0; e < 8; e += 2) {   // two independent round-to-nearest FMAs per instruction
+                    float a0 = f[e], a1 = f[e + 1];
+                    ffma2(a0, a1, weight(r * 3 + sx, e), weight(r * 3 + sx, e + 1), acc[pp][e], acc[pp][e + 1]);
+                    acc[pp][e] = a0, acc[pp][e + 1] = a1;
+                  }
                 }
               }
             }

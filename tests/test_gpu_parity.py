@@ -127,6 +127,31 @@ HALO_GEOMS = [
 ]
 
 
+# narrow 1x1 layers, which run with g pixels per row (g * Cin <= 64, g divides H * W): g = 4 and 2 with full 64-column
+# rows, g = 3 (48 columns: ragged K block), g = 1 because nothing divides, 8 channels (g = 7 of 49 pixels), with and
+# without a residual operand
+GROUP_GEOMS = [
+    (8, 8, 16, 96, wl.ACT_RELU6, False),
+    (6, 10, 32, 16, wl.ACT_NONE, True),
+    (5, 3, 16, 24, wl.ACT_RELU, True),
+    (7, 7, 24, 144, wl.ACT_RELU6, False),
+    (7, 7, 8, 40, wl.ACT_RELU, False),
+]
+
+
+@pytest.mark.parametrize("geom", GROUP_GEOMS)
+def test_narrow_pointwise_layer(geom):
+    H, W, cin, cout, act, residual = geom
+    spec = util.single_layer_model("bf16", H, W, cin, cout, 1, 1, 0, act, residual, seed=hash(geom) % 1000, max_batch=5)
+    run = util.GpuRunner(spec)
+    for B in (1, 5):
+        x = wl.random_features((B, H, W, cin), seed=B, bf16=True, relu=False)
+        o = util.oracle_stage(spec, 0, x)
+        g = run.stage(0, x)
+        util.check_stage(spec, g, o, f"narrow 1x1 {geom} B={B}", elementwise=True)
+        assert g["n_surv"] == B
+
+
 @pytest.mark.parametrize("geom", HALO_GEOMS)
 def test_conv3x3_halo_layer(geom):
     H, W, cin, cout, act = geom
