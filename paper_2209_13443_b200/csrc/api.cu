@@ -253,11 +253,16 @@ ee_status_t launch_head(ee_model* m, StagePlan& sp, const void* x, int B, int hw
   if (timed) record(m, sp, st, "head_gap");
   DecideArgs da{shift, shift_cls, sp.threshold, sp.always_exit, out->conf, out->pred, out->exit_mask,
                 in_ids ? in_ids->ids : nullptr, out->survivor_idx, out->ids_out, out->n_surv_dev, cnt, cnt + m->max_batch};
-  dim3 fgrid(cdiv(K, kFcClasses), cdiv(B, kFcSamples));
-  if (C % V == 0 && ((uintptr_t)sp.fc_w & 15) == 0)
-    EE_CUDA(launch_pdl(fc_kernel<T, true>, fgrid, dim3(kFcThreads), st, (const float*)gap, (const T*)sp.fc_w, (const float*)sp.fc_b, B, C, K, z, da));
+  const int fs = fc_tile_samples(B);
+  dim3 fgrid(cdiv(K, kFcClasses), cdiv(B, fs));
+  const bool fal = C % V == 0 && ((uintptr_t)sp.fc_w & 15) == 0;
+  auto fc_launch = [&](auto kernel) {
+    return launch_pdl(kernel, fgrid, dim3(kFcThreads), st, (const float*)gap, (const T*)sp.fc_w, (const float*)sp.fc_b, B, C, K, z, da);
+  };
+  if (fs == 4)
+    EE_CUDA(fal ? fc_launch(fc_kernel<T, true, 4>) : fc_launch(fc_kernel<T, false, 4>));
   else
-    EE_CUDA(launch_pdl(fc_kernel<T, false>, fgrid, dim3(kFcThreads), st, (const float*)gap, (const T*)sp.fc_w, (const float*)sp.fc_b, B, C, K, z, da));
+    EE_CUDA(fal ? fc_launch(fc_kernel<T, true, 8>) : fc_launch(fc_kernel<T, false, 8>));
   if (timed) record(m, sp, st, "head_fc_softmax_scan");
   return EE_OK;
 }

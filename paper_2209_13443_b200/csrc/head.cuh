@@ -217,13 +217,14 @@ __device__ __forceinline__ void exit_scan(int B, const DecideArgs& d) {
   if (tid == 0) d.n_surv[0] = base;
 }
 
-constexpr int kFcWarps = 8, kFcClassesPerWarp = 2, kFcSamples = 16, kFcChunk = 128;
+constexpr int kFcWarps = 8, kFcClassesPerWarp = 2, kFcChunk = 128;
 constexpr int kFcClasses = kFcWarps * kFcClassesPerWarp;
 constexpr int kFcThreads = kFcWarps * 32;
 
-// z[b][k] = bfc[k] + sum_c wfc[k][c] * gap[b][c].  CTA (x, y) owns 16 classes (two per warp) of the 16 samples of
-// tile y and walks the channels 128 at a time: the tile's pooled values and the classes' weights of a chunk arrive
-// in shared memory through cp.async, two chunks ahead of the arithmetic (ALIGNED; rows that are not whole 16-byte
+// z[b][k] = bfc[k] + sum_c wfc[k][c] * gap[b][c].  CTA (x, y) owns 16 classes (two per warp) of the S samples of
+// tile y (S = 8, or 4 for batches of at most 16: one warp per sample in the exit decision, shorter chains; the tile
+// height changes no sum) and walks the channels 128 at a time: the tile's pooled values and the classes' weights of a
+// chunk arrive in shared memory through cp.async, two chunks ahead of the arithmetic (ALIGNED; rows that are not whole 16-byte
 // vectors take plain loads, one chunk at a time).  Per (b, k): every lane adds its four channels of each chunk in
 // ascending order, then a shuffle tree; the order does not depend on the batch size or the sample's position.
 //
@@ -231,17 +232,17 @@ constexpr int kFcThreads = kFcWarps * 32;
 // exit decisions: softmax top-1 and threshold.  The CTA that completes the last tile's decisions (a second
 // counter) runs the stable scan of the survivors over the whole batch and leaves all counters at zero.
 // Launched with programmatic stream serialization.
-template <typename T, bool ALIGNED>
+template <typename T, bool ALIGNED, int S>
 __global__ void __launch_bounds__(kFcThreads)
 fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float* __restrict__ bfc, int B, int C, int K, float* z,
           DecideArgs d) {
   constexpr int STAGES = ALIGNED ? (sizeof(T) == 2 ? 3 : 2) : 1;
   constexpr int PER = kFcChunk / 32;  // channels per lane per chunk (4)
-  __shared__ __align__(16) float gs[STAGES][kFcSamples][kFcChunk];
+  __shared__ __align__(16) float gs[STAGES][S][kFcChunk];
   __shared__ __align__(16) T wsm[STAGES][kFcClasses][kFcChunk];
   __shared__ bool last_flag;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int k0 = blockIdx.x * kFcClasses, b0 = blockIdx.y * kFcSamples;
+  const int k0 = blockIdx.x * kFcClasses, b0 = blockIdx.y * S;
   const int nchunk = (C + kFcChunk - 1) / kFcChunk;
 
   auto stage_load = [&](int chunk, int buf) {
@@ -249,7 +250,7 @@ fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float*
     if constexpr (ALIGNED) {
       constexpr int WV = 16 / (int)sizeof(T);       // weight elements per 16-byte vector
       constexpr int WPC = kFcChunk / WV;            // vectors per class
-      for (int i = tid; i < kFcSamples * (kFcChunk / 4); i += kFcThreads) {
+      for (int i = tid; i < S * (kFcChunk / 4); i += kFcThreads) {
         const int sidx = i / (kFcChunk / 4), c = (i % (kFcChunk / 4)) * 4;
         const bool in = b0 + sidx < B && c0 + c < C;
         cp_async16(&gs[buf][sidx][c], in ? gap + (size_t)(b0 + sidx) * C + c0 + c : gap, in ? 16 : 0);
@@ -260,7 +261,7 @@ fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float*
         cp_async16(&wsm[buf][cls][c], in ? wfc + (size_t)(k0 + cls) * C + c0 + c : wfc, in ? 16 : 0);
       }
     } else {
-      for (int i = tid; i < kFcSamples * kFcChunk; i += kFcThreads) {
+      for (int i = tid; i < S * kFcChunk; i += kFcThreads) {
         const int sidx = i / kFcChunk, c = i % kFcChunk;
         gs[buf][sidx][c] = (b0 + sidx < B && c0 + c < C) ? gap[(size_t)(b0 + sidx) * C + c0 + c] : 0.f;
       }
@@ -273,11 +274,11 @@ fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float*
 
   pdl_wait();
   pdl_launch_dependents();
-  float acc[kFcClassesPerWarp][kFcSamples];
+  float acc[kFcClassesPerWarp][S];
 #pragma unroll
   for (int q = 0; q < kFcClassesPerWarp; ++q)
 #pragma unroll
-    for (int s2 = 0; s2 < kFcSamples; ++s2) acc[q][s2] = 0.f;
+    for (int s2 = 0; s2 < S; ++s2) acc[q][s2] = 0.f;
   if constexpr (ALIGNED) {
 #pragma unroll
     for (int s0 = 0; s0 < STAGES - 1; ++s0) {
@@ -304,7 +305,7 @@ fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float*
 #pragma unroll
       for (int e = 0; e < PER; ++e) wv[q][e] = Elem<T>::ld(&wsm[buf][warp * kFcClassesPerWarp + q][lane * PER + e]);
 #pragma unroll
-    for (int s2 = 0; s2 < kFcSamples; ++s2) {
+    for (int s2 = 0; s2 < S; ++s2) {
       const float4 g = *reinterpret_cast<const float4*>(&gs[buf][s2][lane * PER]);
       const float gv[PER] = {g.x, g.y, g.z, g.w};
 #pragma unroll
@@ -318,7 +319,7 @@ fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float*
     const int k = k0 + warp * kFcClassesPerWarp + q;
     const float bk = (bfc && k < K) ? bfc[k] : 0.f;
 #pragma unroll
-    for (int s2 = 0; s2 < kFcSamples; ++s2) {
+    for (int s2 = 0; s2 < S; ++s2) {
       float v = acc[q][s2];
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -331,7 +332,7 @@ fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float*
   __syncthreads();
   if (!last_flag) return;
   __threadfence();
-  exit_decide_samples(z, b0, min(B, b0 + kFcSamples), K, warp, kFcWarps, d);
+  exit_decide_samples(z, b0, min(B, b0 + S), K, warp, kFcWarps, d);
   __threadfence();
   __syncthreads();
   if (tid == 0) {
@@ -344,6 +345,9 @@ fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float*
   if (tid == 0) *d.done = 0;
   exit_scan<kFcThreads>(B, d);
 }
+
+// Samples per FC tile for a batch.
+inline int fc_tile_samples(int B) { return B <= 16 ? 4 : 8; }
 
 constexpr int kCopyThreads = 256, kCopyUnroll = 8;
 
