@@ -1,7 +1,7 @@
 """Throughput of the early-exit CNN stage executor on B200: samples/s of the whole hot path.
 
 One "step" is one pass of the whole path over one batch of synthetic requests:
-  ee_batch_refill (the arrivals are appended to the empty batch buffer) -> for every stage:
+  ee_batch_refill (the arrivals are appended to the empty batch buffer) -> for every stage (ee_run_until_exit):
   ee_stage_run (convolutions, exit head, threshold, compaction + gather of the survivors) ->
   the survivor count reaches the host (pinned word, ee_wait_count) and sizes the next stage.
 The batch shrinks stage by stage at the calibrated exit rates, exactly as in serving.
@@ -253,6 +253,19 @@ def run_ours(args):
         nl = 1
         feat, ids = batch0, ids0
         sizes = []
+        if args.exit_rate is None:
+            # ee_run_until_exit: the stage chain inside the library (ee_stage_run, wait for B_exit, next stage)
+            sizes = [v for v in model.run_until_exit(0, feat, n, bufs, ws, ids) if v > 0]
+            for s, v in enumerate(sizes):
+                nl += stage_launches(s, v)
+                if e2e:
+                    res_host[s]["conf"][:v].copy_(bufs[s].conf[:v], non_blocking=True)
+                    res_host[s]["pred"][:v].copy_(bufs[s].pred[:v], non_blocking=True)
+                    res_host[s]["mask"][:v].copy_(bufs[s].exit_mask[:v], non_blocking=True)
+                    d2h += v * 9 + 4
+            if e2e:
+                stream.synchronize()                       # every stage's results have arrived in host memory
+            return nl, h2d, d2h, sizes
         for s in range(nst):
             sizes.append(n)
             bufs[s].arm_count()

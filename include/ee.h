@@ -238,6 +238,21 @@ typedef struct {
 } ee_layer_plan_t;
 ee_status_t ee_model_plan(const ee_model_t* model, int stage, int batch, int cap, ee_layer_plan_t* out, int* n);
 
+/* Runs a batch from stage `first_stage` on until it is empty or the last stage has been launched: ee_stage_run for a
+ * stage, the host's wait for its survivor count (the protocol of ee_wait_count on outs[s].n_surv_host, which must be
+ * a pinned host word for every stage but the last), then the next stage on the survivors (features_out / ids_out of
+ * the stage before).  This is Algorithm 1's "ProcUntilExit" chain without preemption, kept inside the library so that
+ * a stage boundary costs one poll and one launch and no trip through the caller's language runtime.
+ * `in` describes the batch at `first_stage`; its logit_shift applies to that stage only.  `outs` holds one
+ * ee_stage_out_t per stage of the model, indexed by stage (entries below first_stage are ignored).
+ * batch_per_stage (HOST, optional, n_stages ints) receives the batch every stage ran on, 0 for stages not reached.
+ * The last stage is launched but not waited for: its results are ordered on the stream like any other call's.
+ * Errors: those of ee_stage_run; INVALID_ARG when a needed n_surv_host is NULL; TIMEOUT when a count does not arrive
+ * within `timeout_s` seconds. */
+ee_status_t ee_run_until_exit(ee_model_t* model, int first_stage, const ee_stage_in_t* in, void* workspace,
+                              size_t workspace_bytes, const ee_stage_out_t* outs, int32_t* batch_per_stage,
+                              double timeout_s, void* cuda_stream);
+
 /* Host-side wait for a survivor count without synchronising the stream (Section III, step 4: the scheduler needs
  * B_exit, not the features, to size its next launch).  Protocol: the caller stores `sentinel` (a negative value) in
  * its pinned word, passes the word as n_surv_host to ee_stage_run, then calls this: it polls the word until it differs

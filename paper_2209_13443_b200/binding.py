@@ -8,7 +8,7 @@ from __future__ import annotations
 
 import ctypes as C
 import os
-from typing import Optional
+from typing import Optional, Sequence
 
 import numpy as np
 import torch
@@ -21,7 +21,7 @@ STATUS_NAMES = ["EE_OK", "EE_ERR_INVALID_ARG", "EE_ERR_SHAPE", "EE_ERR_CAPACITY"
                 "EE_ERR_CUDA", "EE_ERR_TIMEOUT", "EE_ERR_INTERNAL"]
 EXPORTS = ["ee_model_create", "ee_model_destroy", "ee_model_query", "ee_stage_run", "ee_layer_run", "ee_batch_refill", "ee_exit_head",
            "ee_exit_head_scratch_bytes", "ee_exit_head_static", "ee_gather_survivors", "ee_model_set_graphs", "ee_model_set_timing", "ee_model_get_timing",
-           "ee_model_plan", "ee_model_check", "ee_wait_count", "ee_status_string", "ee_last_cuda_error"]
+           "ee_model_plan", "ee_model_check", "ee_wait_count", "ee_run_until_exit", "ee_status_string", "ee_last_cuda_error"]
 
 
 class EEError(RuntimeError):
@@ -96,6 +96,7 @@ def load_library() -> C.CDLL:
     L.ee_model_set_timing.argtypes = [vp, i]
     L.ee_model_get_timing.argtypes = [vp, i, i, C.POINTER(C.c_float), C.POINTER(C.c_char_p), C.POINTER(i)]
     L.ee_model_plan.argtypes = [vp, i, i, i, C.POINTER(LayerPlan), C.POINTER(i)]
+    L.ee_run_until_exit.argtypes = [vp, i, C.POINTER(StageIn), vp, C.c_size_t, C.POINTER(StageOut), C.POINTER(C.c_int32), C.c_double, vp]
     L.ee_wait_count.argtypes = [vp, C.c_int32, C.c_double, C.POINTER(C.c_int32)]
     L.ee_model_check.argtypes = [vp, vp]
     L.ee_status_string.argtypes = [i]
@@ -148,6 +149,7 @@ class StageBuffers:
         self.n_surv_dev = torch.zeros(1, dtype=torch.int32, device=dev)
         self.n_surv_host = torch.zeros(1, dtype=torch.int32).pin_memory() if pinned_count else None
         self._count_word = C.c_int32.from_address(self.n_surv_host.data_ptr()) if pinned_count else None
+        self._struct = None
 
     def arm_count(self):
         """Stores the sentinel -1 in the pinned count word; call before ee_stage_run, then wait_count()."""
@@ -161,8 +163,11 @@ class StageBuffers:
         return int(v.value)
 
     def as_struct(self) -> StageOut:
-        return StageOut(_ptr(self.features_out), _ptr(self.conf), _ptr(self.pred), _ptr(self.logits), _ptr(self.exit_mask),
-                        _ptr(self.survivor_idx), _ptr(self.ids_out), _ptr(self.n_surv_dev), _ptr(self.n_surv_host))
+        """The ee_stage_out_t of these buffers (built once: the buffers never move)."""
+        if self._struct is None:
+            self._struct = StageOut(_ptr(self.features_out), _ptr(self.conf), _ptr(self.pred), _ptr(self.logits), _ptr(self.exit_mask),
+                                    _ptr(self.survivor_idx), _ptr(self.ids_out), _ptr(self.n_surv_dev), _ptr(self.n_surv_host))
+        return self._struct
 
 
 class EEModel:
@@ -204,6 +209,7 @@ class EEModel:
             _check(self._L.ee_model_create(C.byref(desc), _stream(stream), C.byref(h)), "ee_model_create")
         self._h = h
         self._keep = []
+        self._outs_key, self._outs_arr = None, None
 
     def close(self):
         if getattr(self, "_h", None):
@@ -235,6 +241,25 @@ class EEModel:
         so = out.as_struct() if isinstance(out, StageBuffers) else out
         _check(self._L.ee_stage_run(self._h, stage, C.byref(sin), aligned, workspace.numel() - (aligned - base), C.byref(so),
                                     _stream(stream)), "ee_stage_run")
+
+    def run_until_exit(self, first_stage: int, features, batch: int, outs: Sequence[StageBuffers], workspace: torch.Tensor, ids=None,
+                       logit_shift=None, shift_class=None, timeout_s: float = 10.0, stream=None):
+        """ee_run_until_exit: every stage from ``first_stage`` on, each on the survivors of the one before, until the
+        batch is empty or the last stage has been launched.  ``outs`` holds one StageBuffers per stage of the model.
+        Returns the batch each stage ran on (0 for stages not reached)."""
+        key = tuple(id(o) for o in outs)
+        if self._outs_key != key:       # the array of ee_stage_out_t is built once per set of buffers
+            arr = (StageOut * self.n_stages)()
+            for s, o in enumerate(outs):
+                arr[s] = o.as_struct()
+            self._outs_key, self._outs_arr = key, arr
+        base = workspace.data_ptr()
+        aligned = (base + 255) // 256 * 256
+        sin = StageIn(_ptr(features), _ptr(ids), int(batch), _ptr(logit_shift), _ptr(shift_class))
+        sizes = (C.c_int32 * self.n_stages)()
+        _check(self._L.ee_run_until_exit(self._h, first_stage, C.byref(sin), aligned, workspace.numel() - (aligned - base),
+                                         self._outs_arr, sizes, float(timeout_s), _stream(stream)), "ee_run_until_exit")
+        return list(sizes)
 
     def layer_run(self, stage: int, layer: int, x, residual, batch: int, out, workspace: torch.Tensor, stream=None):
         base = workspace.data_ptr()

@@ -624,6 +624,35 @@ ee_status_t ee_wait_count(const int32_t* n_surv_host, int32_t sentinel, double t
   }
 }
 
+ee_status_t ee_run_until_exit(ee_model_t* m, int first_stage, const ee_stage_in_t* in, void* workspace, size_t workspace_bytes,
+                              const ee_stage_out_t* outs, int32_t* batch_per_stage, double timeout_s, void* cuda_stream) {
+  if (!m || !in || !outs || timeout_s < 0) return EE_ERR_INVALID_ARG;
+  const int n_stages = (int)m->stages.size();
+  if (first_stage < 0 || first_stage >= n_stages) return EE_ERR_STAGE;
+  for (int s = first_stage; s + 1 < n_stages; ++s)
+    if (!outs[s].n_surv_host) return EE_ERR_INVALID_ARG;
+  if (batch_per_stage)
+    for (int s = 0; s < n_stages; ++s) batch_per_stage[s] = 0;
+  ee_stage_in_t cur = *in;
+  for (int s = first_stage; s < n_stages; ++s) {
+    const bool last = s + 1 == n_stages;
+    if (!last) *(volatile int32_t*)outs[s].n_surv_host = -1;
+    ee_status_t rc = ee_stage_run(m, s, &cur, workspace, workspace_bytes, &outs[s], cuda_stream);
+    if (rc != EE_OK) return rc;
+    if (batch_per_stage) batch_per_stage[s] = cur.batch;
+    if (last) break;
+    int32_t n = 0;
+    if ((rc = ee_wait_count(outs[s].n_surv_host, -1, timeout_s, &n)) != EE_OK) return rc;
+    if (n <= 0) break;
+    cur.features = outs[s].features_out;
+    cur.ids = (in->ids && outs[s].ids_out) ? outs[s].ids_out : nullptr;
+    cur.batch = n;
+    cur.logit_shift = nullptr;
+    cur.shift_class = nullptr;
+  }
+  return EE_OK;
+}
+
 ee_status_t ee_model_query(const ee_model_t* m, int stage, ee_stage_info_t* out) {
   if (!m || !out) return EE_ERR_INVALID_ARG;
   if (stage < 0 || stage >= (int)m->stages.size()) return EE_ERR_STAGE;

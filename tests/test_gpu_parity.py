@@ -530,3 +530,40 @@ def test_count_reaches_the_host_without_a_stream_sync():
             assert out.wait_count(5.0) == want
         torch.cuda.synchronize()
     m.check()
+
+
+@pytest.mark.parametrize("which", ["tiny", "resnet"])
+def test_run_until_exit_matches_the_stage_by_stage_loop(which):
+    """ee_run_until_exit chains the stages inside the library; it must leave exactly what a caller's own loop of
+    ee_stage_run + count read-back leaves: same batch per stage, same masks, predictions, ids and survivors.
+    tiny: exits at every stage; resnet: flat heads, the whole batch reaches the last stage."""
+    spec = wl.tiny_ee_cnn(seed=0) if which == "tiny" else wl.resnet50_ee(seed=1, in_hw=64, n_classes=100, max_batch=8, alphas=[0.01] * 4)
+    run = util.GpuRunner(spec)
+    m, ws = run.m, run.ws
+    B = 8
+    x = eb.to_device(spec.dtype, wl.make_input(spec, B, seed=5))
+    ids = torch.arange(100, 100 + B, dtype=torch.int32, device="cuda")
+    ref = []
+    feat, idv, n = x, ids, B
+    for s in range(m.n_stages):
+        m.stage_run(s, feat, n, run.bufs[s], ws, idv)
+        torch.cuda.synchronize()
+        b = run.bufs[s]
+        ns = int(b.n_surv_host[0])
+        ref.append((n, b.exit_mask[:n].clone(), b.pred[:n].clone(), b.conf[:n].clone(), b.ids_out[:ns].clone(), b.features_out[:ns].clone()))
+        feat, idv, n = b.features_out.clone(), b.ids_out.clone(), ns
+        if n == 0:
+            break
+    assert len(ref) >= 2                                   # the batch does reach a later stage
+    bufs2 = [eb.StageBuffers(m, s) for s in range(m.n_stages)]
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for _ in range(2):                                 # plain launches / capture, then graph replay
+            sizes = m.run_until_exit(0, x, B, bufs2, ws, ids)
+            torch.cuda.synchronize()
+            assert sizes[:len(ref)] == [r[0] for r in ref] and all(v == 0 for v in sizes[len(ref):])
+            for s, (n, mask, pred, conf, ids_out, feats) in enumerate(ref):
+                b = bufs2[s]
+                assert torch.equal(b.exit_mask[:n], mask) and torch.equal(b.pred[:n], pred) and torch.equal(b.conf[:n], conf)
+                assert torch.equal(b.ids_out[:len(ids_out)], ids_out) and torch.equal(b.features_out[:len(feats)], feats)
+    m.check()
