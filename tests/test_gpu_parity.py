@@ -337,6 +337,21 @@ def test_error_codes_and_empty_batch():
     m.stage_run(0, None, 0, run.bufs[0], run.ws)                       # empty batch: only the count is written
     torch.cuda.synchronize()
     assert int(run.bufs[0].n_surv_dev.cpu()[0]) == 0 and int(run.bufs[0].n_surv_host[0]) == 0
+    # ee_run_until_exit: an empty batch runs nothing past the first stage; a stage that is not the last needs its pinned
+    # count word; stage and capacity errors are those of ee_stage_run
+    bufs = [eb.StageBuffers(m, s) for s in range(m.n_stages)]
+    assert m.run_until_exit(0, x, 0, bufs, run.ws) == [0] * m.n_stages
+    assert m.run_until_exit(m.n_stages - 1, bufs[m.n_stages - 2].features_out, 0, bufs, run.ws) == [0] * m.n_stages
+    no_word = [eb.StageBuffers(m, s, pinned_count=False) for s in range(m.n_stages)]
+    with pytest.raises(eb.EEError) as e:
+        m.run_until_exit(0, x, 1, no_word, run.ws)
+    assert e.value.status == 1
+    with pytest.raises(eb.EEError) as e:
+        m.run_until_exit(m.n_stages, x, 1, bufs, run.ws)
+    assert e.value.status == 4
+    with pytest.raises(eb.EEError) as e:
+        m.run_until_exit(0, x, spec.max_batch + 1, bufs, run.ws)
+    assert e.value.status == 3
     bad = wl.tiny_ee_cnn(seed=0)
     bad.stages[1].layers[0].cin = 5                                    # does not chain
     with pytest.raises(eb.EEError) as e:
