@@ -1252,8 +1252,11 @@ inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, co
   p.gH = L.g_h, p.gW = L.g_w, p.gCin = L.g_cin, p.gkh = L.g_kh, p.grun = L.g_kw * L.g_cin, p.grunp = L.g_runp;
   if (L.gather) p.stride = L.g_stride, p.pad = L.g_pad;
   dim3 grid(cdiv(p.M, kTcBM), cdiv(L.cout, L.bn), split ? L.splits : 1);
-  // at most one CTA per SM anyway: take the deep operand ring
-  const bool deep = (long)grid.x * grid.y * grid.z <= 148;
+  // At most one CTA per SM anyway: take the deep operand ring.  A cluster grid close to the SM count does not: its
+  // clusters need all their CTAs inside one GPC, a 192 KB CTA owns its SM, and the last clusters then wait for a second
+  // wave (measured: the split-3 3x3 layers of 132 CTAs lose 6 us each with the deep ring).
+  const long n_ctas = (long)grid.x * grid.y * grid.z;
+  const bool deep = split ? n_ctas * 4 <= 3L * c.sm_count : n_ctas <= c.sm_count;
   const bool tma_res = res && !split;
   if (L.gather) {
     if (res || split) return EE_ERR_INTERNAL;
