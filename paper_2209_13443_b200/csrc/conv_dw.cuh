@@ -250,11 +250,22 @@ inline ee_status_t dw_tma_launch(TcContext& c, const TcLayer& L, const ConvGeom&
   const int row_bytes = (g.W + 2) * p.cb * 2;
   int in_rows = kDwMaxTileBytes / row_bytes;                      // input rows a slot holds
   if (in_rows > 256) in_rows = 256;
-  p.RB = (in_rows - 3) / g.stride + 1;
-  if (p.RB > g.Ho) p.RB = g.Ho;
-  // enough tiles for every SM: shrink the band while the grid would leave SMs idle
+  int rb_max = (in_rows - 3) / g.stride + 1;
+  if (rb_max > g.Ho) rb_max = g.Ho;
+  // Band height: a CTA's eight consumer warps take 256 / (cb / 8) strips per pass over a tile, a tile costs about one
+  // more pass (waiting for the slot, hand-over), and the busiest CTA walks ceil(tiles / CTAs) tiles.  Take the height
+  // that minimises that CTA's passes (bytes moved rise with shorter bands: each band re-reads two frame rows).
   const int chunks = cdiv(g.Cin, 64);
-  while (p.RB > 1 && (long)g.B * cdiv(g.Ho, p.RB) * chunks < 2L * c.sm_count) p.RB = (p.RB + 1) / 2;
+  const int ctas_x = std::max(1, c.sm_count / chunks);
+  const int strips = (g.Wo + kDwStrip - 1) / kDwStrip;
+  const int per_pass = kDwConsumers / std::max(1, p.cb / 8);
+  long best = -1;
+  p.RB = 1;
+  for (int rb = 1; rb <= rb_max; ++rb) {
+    const long tiles = (long)g.B * cdiv(g.Ho, rb);
+    const long cost = cdiv(tiles, std::min<long>(tiles, ctas_x)) * (cdiv((long)rb * strips, per_pass) + 1);
+    if (best < 0 || cost <= best) best = cost, p.RB = rb;   // ties: the taller band (fewer frame rows re-read)
+  }
   const int rows = (p.RB - 1) * g.stride + 3;
   p.bands = cdiv(g.Ho, p.RB);
   p.tiles = g.B * p.bands;
