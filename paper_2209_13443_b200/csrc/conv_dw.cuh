@@ -21,7 +21,7 @@ struct DwParams {
   int RB;          // output rows per tile
   int bands;       // ceil(Ho / RB)
   int tiles;       // B * bands, per channel block
-  int cb;          // channels per block: min(64, C)
+  int cb;          // channels per block (dw_block_channels)
   int tile_bytes;  // ((RB - 1) * stride + 3) * (W + 2) * cb * 2
   int slot_bytes;  // tile_bytes rounded up to 128
   int act;
@@ -61,7 +61,7 @@ dwconv3x3_tma_kernel(const __grid_constant__ CUtensorMap tmX, DwParams p) {
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int my_tiles = (int)blockIdx.x < p.tiles ? (p.tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-  const int c0 = (int)blockIdx.y * 64;
+  const int c0 = (int)blockIdx.y * p.cb;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kDwStages; ++s) {
@@ -196,10 +196,17 @@ dwconv3x3_tma_kernel(const __grid_constant__ CUtensorMap tmX, DwParams p) {
 
 // Layers this kernel takes: depthwise 3x3 (or a 3x3 max-pool, w == nullptr), pad 1, stride 1 or 2, channels a multiple
 // of 8, at most 254 columns, and a tile of one output row that fits a ring slot.
+// Channels per block: the channels are cut into ceil(C / 64) blocks of equal size (a multiple of 8), so that no block
+// is mostly empty (144 channels: 3 x 48, not 64 + 64 + 16).
+inline int dw_block_channels(int C) {
+  const int blocks = (C + 63) / 64;
+  return ((C + blocks - 1) / blocks + 7) / 8 * 8;
+}
+
 inline bool dw_tma_supported(const ConvGeom& g, const void* x, const void* w, const void* y) {
   if (!(g.kh == 3 && g.kw == 3 && g.pad == 1 && (g.stride == 1 || g.stride == 2) && g.Cin % 8 == 0 && g.Cin == g.Cout)) return false;
   if ((((uintptr_t)x | (uintptr_t)w | (uintptr_t)y) & 15) != 0 || g.W + 2 > 256) return false;
-  const int cb = g.Cin < 64 ? g.Cin : 64;
+  const int cb = dw_block_channels(g.Cin);
   return 3 * (g.W + 2) * cb * 2 <= kDwMaxTileBytes;
 }
 
@@ -246,7 +253,7 @@ inline ee_status_t dw_tma_launch(TcContext& c, const TcLayer& L, const ConvGeom&
                                  const float* bias, void* y, int* err_flag, cudaStream_t st) {
   DwParams p;
   p.H = g.H, p.W = g.W, p.C = g.Cin, p.Ho = g.Ho, p.Wo = g.Wo;
-  p.cb = g.Cin < 64 ? g.Cin : 64;
+  p.cb = dw_block_channels(g.Cin);
   const int row_bytes = (g.W + 2) * p.cb * 2;
   int in_rows = kDwMaxTileBytes / row_bytes;                      // input rows a slot holds
   if (in_rows > 256) in_rows = 256;
@@ -255,7 +262,7 @@ inline ee_status_t dw_tma_launch(TcContext& c, const TcLayer& L, const ConvGeom&
   // Band height: a CTA's eight consumer warps take 256 / (cb / 8) strips per pass over a tile, a tile costs about one
   // more pass (waiting for the slot, hand-over), and the busiest CTA walks ceil(tiles / CTAs) tiles.  Take the height
   // that minimises that CTA's passes (bytes moved rise with shorter bands: each band re-reads two frame rows).
-  const int chunks = cdiv(g.Cin, 64);
+  const int chunks = cdiv(g.Cin, p.cb);
   const int ctas_x = std::max(1, c.sm_count / chunks);
   const int strips = (g.Wo + kDwStrip - 1) / kDwStrip;
   const int per_pass = kDwConsumers / std::max(1, p.cb / 8);
