@@ -400,10 +400,15 @@ def run_ours(args):
     n_cpu = min(B, args.cpu_samples)
     x_np = x_host[:n_cpu].float().numpy()
     t0 = time.perf_counter()
-    oracle_pass(spec, x_np, np.arange(n_cpu, dtype=np.int32))
-    cpu_dt = time.perf_counter() - t0
-    cpu = {"value": n_cpu / cpu_dt, "unit": UNIT, "cores": eo.n_threads(), "kind": "oracle",
-           "sample": f"first {n_cpu} of {B} samples, whole path once, {cpu_dt:.1f} s"}
+    cpu_reps = 0
+    while True:                                            # about 10 s of CPU work, four passes at most
+        oracle_pass(spec, x_np, np.arange(n_cpu, dtype=np.int32))
+        cpu_reps += 1
+        cpu_dt = time.perf_counter() - t0
+        if cpu_dt >= 10.0 or cpu_reps >= 4 or args.cpu_samples < B:
+            break
+    cpu = {"value": n_cpu * cpu_reps / cpu_dt, "unit": UNIT, "cores": eo.n_threads(), "kind": "oracle",
+           "sample": f"first {n_cpu} of {B} samples, whole path {cpu_reps} time(s), {cpu_dt:.1f} s"}
 
     value = replicas.job_throughput(world, B, K, total_ms)
     out = {
