@@ -99,6 +99,8 @@ GEOMS = [
     (12, 12, 128, 128, 3, 2, 1, wl.ACT_RELU, False),
     (6, 6, 320, 96, 1, 1, 0, wl.ACT_NONE, False),
     (5, 5, 136, 72, 3, 1, 1, wl.ACT_RELU, False),       # K and N not multiples of 64
+    (11, 9, 3, 32, 3, 2, 1, wl.ACT_RELU6, False),       # 3x3 stem on 3 channels, stride 2, odd image
+    (8, 8, 3, 16, 3, 1, 1, wl.ACT_NONE, False),         # the same, stride 1
 ]
 
 
