@@ -34,7 +34,7 @@ if ROOT not in sys.path:
 # DRAM bytes (read + written) per launch of the tensor-core conv kernels, from one ncu capture of the default workload
 # (ResNet-50-shaped, B=64, calibrated exits: 52 launches per pass, 1730.7 MB).  Reported only for that workload; it
 # has to be taken again (or set to None) whenever one of those kernels changes.
-NCU_CONV_TRAFFIC_PER_LAUNCH = {("resnet50", 64): 33.28e6}
+NCU_CONV_TRAFFIC_PER_LAUNCH = {("resnet50", 64): 33.29e6}
 
 METRIC = "EE-CNN samples/sec on 1 B200 vs exit rate & batch 1-64; tensor-pipe % of peak"
 UNIT = "samples/s"
