@@ -74,6 +74,7 @@ struct StagePlan {
   float* fc_b = nullptr;
   float threshold = 0.f;
   int always_exit = 0;
+  bool gap_rev = false, gather_rev = false;   // walk directions of the pooling and gather kernels
   double flops_per_sample = 0;
   // timing of the last run
   std::vector<cudaEvent_t> ev;
@@ -247,9 +248,9 @@ ee_status_t launch_head(ee_model* m, StagePlan& sp, const void* x, int B, int hw
   const int n_zero = m->max_batch + 1;   // the pooling kernel leaves the FC kernel's counters at zero
   dim3 ggrid(cdiv(vec ? C / V : C, lanes), B);
   if (vec)
-    EE_CUDA(launch_pdl(gap_kernel<T, V>, ggrid, dim3(kGapThreads), st, (const T*)x, hw, C, lanes, gap, cnt, n_zero));
+    EE_CUDA(launch_pdl(gap_kernel<T, V>, ggrid, dim3(kGapThreads), st, (const T*)x, hw, C, lanes, gap, cnt, n_zero, sp.gap_rev ? 1 : 0));
   else
-    EE_CUDA(launch_pdl(gap_kernel<T, 1>, ggrid, dim3(kGapThreads), st, (const T*)x, hw, C, lanes, gap, cnt, n_zero));
+    EE_CUDA(launch_pdl(gap_kernel<T, 1>, ggrid, dim3(kGapThreads), st, (const T*)x, hw, C, lanes, gap, cnt, n_zero, sp.gap_rev ? 1 : 0));
   if (timed) record(m, sp, st, "head_gap");
   DecideArgs da{shift, shift_cls, sp.threshold, sp.always_exit, out->conf, out->pred, out->exit_mask,
                 in_ids ? in_ids->ids : nullptr, out->survivor_idx, out->ids_out, out->n_surv_dev, cnt, cnt + m->max_batch};
@@ -269,10 +270,10 @@ ee_status_t launch_head(ee_model* m, StagePlan& sp, const void* x, int B, int hw
 
 template <typename V>
 ee_status_t gather_launch_t(const void* feat, size_t bytes_per_sample, const int32_t* idx, const int32_t* n_dev, int max_rows,
-                            void* out, cudaStream_t st) {
+                            void* out, bool rev, cudaStream_t st) {
   const size_t vecs = bytes_per_sample / sizeof(V);
   dim3 grid(cdiv((long)vecs, kCopyThreads * kCopyUnroll), max_rows);
-  gather_rows_kernel<V><<<grid, kCopyThreads, 0, st>>>((const V*)feat, vecs, idx, n_dev, (V*)out);
+  gather_rows_kernel<V><<<grid, kCopyThreads, 0, st>>>((const V*)feat, vecs, idx, n_dev, (V*)out, rev ? 1 : 0);
   EE_CUDA(cudaGetLastError());
   return EE_OK;
 }
@@ -284,13 +285,13 @@ int copy_width(size_t bytes_per_sample, const void* a, const void* b) {
 }
 
 ee_status_t gather_launch(const void* feat, size_t bytes_per_sample, const int32_t* idx, const int32_t* n_dev, int max_rows,
-                          void* out, cudaStream_t st) {
+                          void* out, bool rev, cudaStream_t st) {
   if (max_rows <= 0 || bytes_per_sample == 0) return EE_OK;
   switch (copy_width(bytes_per_sample, feat, out)) {
-    case 16: return gather_launch_t<uint4>(feat, bytes_per_sample, idx, n_dev, max_rows, out, st);
-    case 4: return gather_launch_t<uint32_t>(feat, bytes_per_sample, idx, n_dev, max_rows, out, st);
-    case 2: return gather_launch_t<uint16_t>(feat, bytes_per_sample, idx, n_dev, max_rows, out, st);
-    default: return gather_launch_t<uint8_t>(feat, bytes_per_sample, idx, n_dev, max_rows, out, st);
+    case 16: return gather_launch_t<uint4>(feat, bytes_per_sample, idx, n_dev, max_rows, out, rev, st);
+    case 4: return gather_launch_t<uint32_t>(feat, bytes_per_sample, idx, n_dev, max_rows, out, rev, st);
+    case 2: return gather_launch_t<uint16_t>(feat, bytes_per_sample, idx, n_dev, max_rows, out, rev, st);
+    default: return gather_launch_t<uint8_t>(feat, bytes_per_sample, idx, n_dev, max_rows, out, rev, st);
   }
 }
 
@@ -335,7 +336,7 @@ ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, c
     EE_CUDA(cudaEventRecord(m->ev_join, m->side));
   }
   if (!sp.always_exit) {
-    s = gather_launch(so, (size_t)hw * sp.out_c * esize(m->dtype), out->survivor_idx, out->n_surv_dev, B, out->features_out, st);
+    s = gather_launch(so, (size_t)hw * sp.out_c * esize(m->dtype), out->survivor_idx, out->n_surv_dev, B, out->features_out, sp.gather_rev, st);
     if (s != EE_OK) return s;
     record(m, sp, st, "gather_survivors");
   }
@@ -423,6 +424,7 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
   if (rc != EE_OK) return fail(rc);
 
   int h = desc->in_h, w = desc->in_w, c = desc->in_c;
+  bool in_rev = false;   // direction in which the stage input was last walked (by the gather of the stage before)
   m->stages.resize(desc->n_stages);
   for (int s = 0; s < desc->n_stages; ++s) {
     const ee_stage_desc_t& sd = desc->stages[s];
@@ -599,6 +601,27 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
       } else {
         L.kind = KK_SIMT;
       }
+    }
+    // Walk directions.  Feature maps of a large batch exceed the L2, so a kernel that walks its input from the first
+    // row finds the rows its producer wrote first already evicted, and evicts the newest ones before it reaches them.
+    // Every kernel therefore walks opposite to the kernel that last touched its largest operand: it starts on the rows
+    // that are still cached.  The order of the sums inside a tile does not depend on the direction.
+    {
+      std::vector<char> slot_rev(sp.slot_off.size(), 0);
+      auto dir_of = [&](int slot) { return slot < 0 ? in_rev : slot_rev[slot] != 0; };
+      for (int i = 0; i < sd.n_layers; ++i) {
+        LayerPlan& L = sp.layers[i];
+        const size_t in_sz = (size_t)L.in_h * L.in_w * L.d.cin, res_sz = L.res_slot == -2 ? 0 : (size_t)L.out_h * L.out_w * L.d.cout;
+        const bool rev = L.kind != KK_SIMT && !(res_sz > in_sz ? dir_of(L.res_slot) : dir_of(L.src_slot));   // the CUDA-core kernel walks forward
+        L.tc.rev = rev;
+        if (L.src_slot < 0 || L.res_slot == -1) in_rev = rev;
+        if (L.src_slot >= 0) slot_rev[L.src_slot] = rev;
+        if (L.res_slot >= 0) slot_rev[L.res_slot] = rev;
+        slot_rev[L.out_slot] = rev;
+      }
+      sp.gap_rev = !slot_rev[sp.out_slot];
+      sp.gather_rev = !sp.gap_rev;
+      in_rev = sp.gather_rev;
     }
     if ((rc = upload_bytes(m, sd.fc_weight, (size_t)sd.n_classes * sp.out_c * es, ondev, st, &sp.fc_w)) != EE_OK) return fail(rc);
     if ((rc = upload<float>(m, sd.fc_bias, sd.n_classes, ondev, st, &sp.fc_b)) != EE_OK) return fail(rc);
@@ -846,7 +869,7 @@ ee_status_t ee_exit_head_static(ee_model_t* m, int stage, const void* x, int bat
 ee_status_t ee_gather_survivors(const void* feat, size_t bytes_per_sample, const int32_t* survivor_idx, const int32_t* n_surv_dev,
                                 int max_rows, void* feat_out, void* cuda_stream) {
   if (!feat || !survivor_idx || !n_surv_dev || !feat_out || max_rows < 0) return EE_ERR_INVALID_ARG;
-  return gather_launch(feat, bytes_per_sample, survivor_idx, n_surv_dev, max_rows, feat_out, (cudaStream_t)cuda_stream);
+  return gather_launch(feat, bytes_per_sample, survivor_idx, n_surv_dev, max_rows, feat_out, false, (cudaStream_t)cuda_stream);
 }
 
 ee_status_t ee_model_set_graphs(ee_model_t* m, int enabled) {

@@ -25,6 +25,7 @@ struct DwParams {
   int tile_bytes;  // ((RB - 1) * stride + 3) * (W + 2) * cb * 2
   int slot_bytes;  // tile_bytes rounded up to 128
   int act;
+  int rev;         // 1: walk the tiles from the last one down
   const bf16* w;   // [C][3][3]
   const float* scale;
   const float* bias;
@@ -78,7 +79,7 @@ dwconv3x3_tma_kernel(const __grid_constant__ CUtensorMap tmX, DwParams p) {
   if (warp == 0) {
     if (lane == 0) {
       for (int j = 0; j < my_tiles; ++j) {
-        const int t = (int)blockIdx.x + j * (int)gridDim.x;
+        const int tf = (int)blockIdx.x + j * (int)gridDim.x, t = p.rev ? p.tiles - 1 - tf : tf;
         const int b = t / p.bands, band = t - b * p.bands;
         const int s = j % kDwStages;
         if (!mbar_wait(empty(s), ((uint32_t)(j / kDwStages) & 1u) ^ 1u, p.err_flag)) break;
@@ -115,7 +116,7 @@ dwconv3x3_tma_kernel(const __grid_constant__ CUtensorMap tmX, DwParams p) {
   const int Wc = p.W + 2;
   const int items = p.RB * strips;
   for (int j = 0; j < my_tiles; ++j) {
-    const int t = (int)blockIdx.x + j * (int)gridDim.x;
+    const int tf = (int)blockIdx.x + j * (int)gridDim.x, t = p.rev ? p.tiles - 1 - tf : tf;
     const int b = t / p.bands, band = t - b * p.bands;
     const int s = j % kDwStages;
     if (!__all_sync(0xffffffffu, mbar_wait(full(s), (uint32_t)(j / kDwStages) & 1u, p.err_flag))) break;
@@ -279,6 +280,7 @@ inline ee_status_t dw_tma_launch(TcContext& c, const TcLayer& L, const ConvGeom&
   p.tile_bytes = rows * row_bytes;
   p.slot_bytes = (int)align_up((size_t)p.tile_bytes, 128);
   p.act = g.act;
+  p.rev = L.rev ? 1 : 0;
   p.w = (const bf16*)w, p.scale = scale, p.bias = bias, p.y = (bf16*)y;
   p.err_flag = err_flag;
   const CUtensorMap* t = nullptr;

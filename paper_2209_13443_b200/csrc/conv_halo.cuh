@@ -28,6 +28,7 @@ struct HaloParams {
   int H, W, Wp, R;    // image size, padded row length W + 2, output rows per tile
   int N;              // Cout (<= 64, a multiple of 8)
   int act;
+  int rev;            // 1: walk the tiles from the last one down
   const float* scale;
   const float* bias;
   bf16* out;          // [B][H][W][N]
@@ -120,7 +121,7 @@ conv3x3_halo_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
     if (lane == 0) {
       const uint32_t block_bytes = (uint32_t)(p.Wp * (p.R + 2) * 128);
       for (int j = 0; j < my_tiles; ++j) {
-        const int t = (int)blockIdx.x + j * (int)gridDim.x;
+        const int tf = (int)blockIdx.x + j * (int)gridDim.x, t = p.rev ? p.tiles - 1 - tf : tf;
         const int n = t / p.tiles_per_img, h0 = (t - n * p.tiles_per_img) * p.R;
         const int s = j % kHaloStages;
         const uint32_t ph = (uint32_t)(j / kHaloStages) & 1u;
@@ -171,7 +172,7 @@ conv3x3_halo_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
     const int y = row / p.Wp, x = row - y * p.Wp;
     const bool inside = y < p.R && x < p.W;
     for (int j = 0; j < my_tiles; ++j) {
-      const int t = (int)blockIdx.x + j * (int)gridDim.x;
+      const int tf = (int)blockIdx.x + j * (int)gridDim.x, t = p.rev ? p.tiles - 1 - tf : tf;
       const int n = t / p.tiles_per_img, h0 = (t - n * p.tiles_per_img) * p.R;
       const int b = j & 1;
       if (!__all_sync(0xffffffffu, mbar_wait(acc_full(b), (uint32_t)(j >> 1) & 1u, p.err_flag))) break;
@@ -232,6 +233,7 @@ inline ee_status_t halo_launch(TcContext& c, const TcLayer& L, const void* src, 
   p.tiles = B * p.tiles_per_img;
   p.N = L.cout;
   p.act = L.act;
+  p.rev = L.rev ? 1 : 0;
   p.scale = scale, p.bias = bias;
   p.out = (bf16*)dst;
   p.err_flag = err_flag;

@@ -23,6 +23,7 @@ struct StemParams {
   int tiles;            // B * Ho output rows
   int Ho, Wo, N;        // output height, width (<= kStemMaxWo) and Cout (<= 64)
   int act;
+  int rev;              // 1: walk the output rows from the last one down
   const float* scale;
   const float* bias;
   int* err_flag;
@@ -128,7 +129,7 @@ conv_stem7x7_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
   if (warp == 0) {
     if (lane == 0) {
       for (int j = 0; j < my_tiles; ++j) {
-        const int t = (int)blockIdx.x + j * (int)gridDim.x;
+        const int tf = (int)blockIdx.x + j * (int)gridDim.x, t = p.rev ? p.tiles - 1 - tf : tf;
         const int n = t / p.Ho, oy = t - n * p.Ho;
         const int b = j & 1;
         if (j >= 2 && !mbar_wait(patch_empty(b), (uint32_t)((j >> 1) - 1) & 1u, p.err_flag)) break;
@@ -222,7 +223,7 @@ conv_stem7x7_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
     uint8_t* oline = gen + S::kOOff + row * 128;
     bool pending = false;  // lane 0: a bulk store of this warp may still be reading the staging rows
     for (int j = 0; j < my_tiles; ++j) {
-      const int t = (int)blockIdx.x + j * (int)gridDim.x;
+      const int tf = (int)blockIdx.x + j * (int)gridDim.x, t = p.rev ? p.tiles - 1 - tf : tf;
       const int b = j & 1;
       if (!__all_sync(0xffffffffu, mbar_wait(acc_full(b), (uint32_t)(j >> 1) & 1u, p.err_flag))) break;
       tc_fence_after();
@@ -312,6 +313,7 @@ inline ee_status_t stem_launch(TcContext& c, const TcLayer& L, const void* src, 
   p.tiles = B * L.out_h;
   p.Ho = L.out_h, p.Wo = L.out_w, p.N = L.cout;
   p.act = L.act;
+  p.rev = L.rev ? 1 : 0;
   p.scale = scale, p.bias = bias;
   p.err_flag = err_flag;
   cudaLaunchConfig_t cfg = {};

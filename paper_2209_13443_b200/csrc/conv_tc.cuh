@@ -46,6 +46,8 @@ struct TcParams {
   bf16* out;
   int* err_flag;
   int kb_per;           // split-K: K blocks per range (a property of the layer)
+  int rev;              // 1: walk the M tiles from the last one down (start where the producer of the input finished: its
+                        // newest rows are the ones still in L2)
   // gather mode (layers whose pixel rows are not 16-byte units, e.g. a 3-channel stem): the epilogue warps build the A tile
   const bf16* gx;       // input feature map [B][gH][gW][gCin]
   int gH, gW, gCin, gkh, grun, grunp;  // run = kw*Cin contiguous taps of one filter row, zero-padded to runp columns
@@ -384,7 +386,7 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * kTcBM, n0 = blockIdx.y * BN;
+  const int m0 = (p.rev ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x) * kTcBM, n0 = blockIdx.y * BN;
   const int num_kb_all = p.taps * p.cblocks;
   const int kb_begin = SPLIT ? (int)blockIdx.z * p.kb_per : 0;
   const int kb_end = SPLIT ? min(num_kb_all, kb_begin + p.kb_per) : num_kb_all;
@@ -731,7 +733,7 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
   // kernel writes them
   const int w_ahead = my_tiles > 0 ? min(num_kb, kStages) : 0;
   if (warp == 0 && lane == 0) {
-    const int n0 = ((int)blockIdx.x % n_tiles) * BN;
+    const int n0 = ((p.rev ? total - 1 - (int)blockIdx.x : (int)blockIdx.x) % n_tiles) * BN;
     for (int i = 0; i < w_ahead; ++i) {
       const int tap = i / p.cblocks, cb = i - tap * p.cblocks;
       mbar_expect_tx(full_bar(i), S::kStage);
@@ -746,7 +748,7 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
       int g = 0;  // K blocks issued so far, across tiles: the ring never drains at a tile boundary
       bool ok = true;
       for (int j = 0; j < my_tiles && ok; ++j) {
-        const int t = (int)blockIdx.x + j * (int)gridDim.x;
+        const int tf = (int)blockIdx.x + j * (int)gridDim.x, t = p.rev ? total - 1 - tf : tf;
         const int m0 = (t / n_tiles) * kTcBM, n0 = (t % n_tiles) * BN;
         const int b = j & 1;
         if (RES) {
@@ -826,7 +828,7 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
     int sc_n0 = -1;
     bool pending = false;  // lane 0: a bulk store group of this warp may still be reading shared memory
     for (int j = 0; j < my_tiles; ++j) {
-      const int t = (int)blockIdx.x + j * (int)gridDim.x;
+      const int tf = (int)blockIdx.x + j * (int)gridDim.x, t = p.rev ? total - 1 - tf : tf;
       const int m0 = (t / n_tiles) * kTcBM, n0 = (t % n_tiles) * BN;
       const int b = j & 1;
       if (n0 != sc_n0) {  // consecutive tiles of a CTA usually share the N tile: reload only on change
@@ -968,6 +970,7 @@ struct TcLayer {
   int bn = 128;
   bool im2col = false;
   int splits = 1, kb_per = 0;    // split-K ranges of this layer (fixed per layer, independent of the batch)
+  bool rev = false;              // walk the output tiles from the last one down (see TcParams::rev)
   // gather mode: geometry of the real convolution (cin/kh/... above then describe the packed 1x1 GEMM view)
   bool gather = false;
   bool stem7 = false;   // the 7x7/2 stem kernel of conv_stem.cuh takes this layer
@@ -1248,6 +1251,7 @@ inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, co
   p.err_flag = err_flag;
   const bool split = L.splits > 1;
   p.kb_per = L.kb_per;
+  p.rev = L.rev ? 1 : 0;
   p.gx = (const bf16*)src;
   p.gH = L.g_h, p.gW = L.g_w, p.gCin = L.g_cin, p.gkh = L.g_kh, p.grun = L.g_kw * L.g_cin, p.grunp = L.g_runp;
   if (L.gather) p.stride = L.g_stride, p.pad = L.g_pad;

@@ -28,9 +28,10 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 // FC kernel behind it in the stream relies on.  Launched with programmatic stream serialization.
 template <typename T, int VEC>
 __global__ void __launch_bounds__(kGapThreads)
-gap_kernel(const T* __restrict__ x, int HW, int C, int lanes, float* __restrict__ gap, unsigned* __restrict__ zero_me, int n_zero) {
+gap_kernel(const T* __restrict__ x, int HW, int C, int lanes, float* __restrict__ gap, unsigned* __restrict__ zero_me, int n_zero,
+           int rev) {
   __shared__ float red[kGapThreads * VEC];
-  const int tid = threadIdx.x, b = blockIdx.y;
+  const int tid = threadIdx.x, b = rev ? (int)(gridDim.y - 1 - blockIdx.y) : (int)blockIdx.y;   // rev: last sample first
   const int cv = C / VEC;
   const int groups = kGapThreads / lanes;
   const int grp = tid / lanes, lv = tid - grp * lanes;
@@ -356,12 +357,13 @@ constexpr int kCopyThreads = 256, kCopyUnroll = 8;
 template <typename V>
 __global__ void __launch_bounds__(kCopyThreads)
 gather_rows_kernel(const V* __restrict__ src, size_t vecs_per_row, const int32_t* __restrict__ surv_idx,
-                   const int32_t* __restrict__ n_surv, V* __restrict__ dst) {
-  const int j = blockIdx.y;
+                   const int32_t* __restrict__ n_surv, V* __restrict__ dst, int rev) {
+  const int j = rev ? (int)(gridDim.y - 1 - blockIdx.y) : (int)blockIdx.y;   // rev: last row first, each row from its end
+  const unsigned bx = rev ? gridDim.x - 1 - blockIdx.x : blockIdx.x;
   if (j >= *n_surv) return;
   const V* s = src + (size_t)surv_idx[j] * vecs_per_row;
   V* d = dst + (size_t)j * vecs_per_row;
-  const size_t v0 = (size_t)blockIdx.x * (kCopyThreads * kCopyUnroll) + threadIdx.x;
+  const size_t v0 = (size_t)bx * (kCopyThreads * kCopyUnroll) + threadIdx.x;
   V r[kCopyUnroll];
 #pragma unroll
   for (int u = 0; u < kCopyUnroll; ++u) {
