@@ -319,6 +319,131 @@ def test_activation_scale_stays_order_one():
         x = r["stage_out"]
 
 
+def _torch_conv(x, l, residual=None):
+    """One layer from torch CPU fp64 primitives: conv2d (groups for depthwise), folded-BN scale and bias,
+    the residual operand before the activation.  x and the result are NCHW float64 tensors."""
+    w = torch.from_numpy(l.weight.astype(np.float64)).permute(0, 3, 1, 2)
+    y = F.conv2d(x, w, stride=l.stride, padding=l.pad, groups=l.groups)
+    y = y * torch.from_numpy(l.scale.astype(np.float64)).view(1, -1, 1, 1) + torch.from_numpy(l.bias.astype(np.float64)).view(1, -1, 1, 1)
+    if residual is not None:
+        y = y + residual
+    if l.act == wl.ACT_RELU:
+        y = torch.relu(y)
+    elif l.act == wl.ACT_RELU6:
+        y = torch.clamp(y, 0.0, 6.0)
+    return y
+
+
+def _nhwc(t):
+    return t.permute(0, 2, 3, 1).numpy()
+
+
+def test_run_layers_wires_bottlenecks_and_inverted_residuals_like_the_block_definitions():
+    """The driver that chains layers (input_from / residual_from / depthwise groups) against the block
+    definitions written out by hand with torch fp64 calls: a ResNet bottleneck with a projection shortcut
+    (1x1 -> 3x3 stride s -> 1x1, shortcut = strided 1x1 of the BLOCK input), one with an identity shortcut
+    (the block input itself), and inverted-residual blocks with (stride 1, Cin == Cout) and without a
+    residual connection.  A wrong source for an input or a residual operand changes the result by O(1)."""
+    # ---- two chained bottlenecks: projection (stride 2), then identity
+    rng = wl._rng(7, 950)
+    layers = []
+    last = wl._bottleneck(rng, layers, 16, 8, 2, True, False, wl.FROM_STAGE_INPUT)
+    last = wl._bottleneck(rng, layers, 32, 8, 1, False, False, last)
+    assert len(layers) == 7 and last == 6
+    fw, fb = wl._head(rng, 32, 5, 1.0, False)
+    m = wl.Model("blocks", "f32", 9, 9, 16, [wl.Stage(layers, 5, fw, fb, 2.0, False)], 2)
+    x_np = wl.random_features((2, 9, 9, 16), seed=5, bf16=False, relu=False)
+    outs = eo.run_layers(m, 0, x_np, keep_all=True)
+    x = torch.from_numpy(x_np.astype(np.float64)).permute(0, 3, 1, 2)
+    a1 = _torch_conv(x, layers[0])                      # 1x1 reduce of the block input
+    a2 = _torch_conv(a1, layers[1])                     # 3x3, stride 2
+    sc = _torch_conv(x, layers[2])                      # projection shortcut: strided 1x1 of the block input
+    a3 = _torch_conv(a2, layers[3], residual=sc)        # 1x1 expand + shortcut, then ReLU
+    b1 = _torch_conv(a3, layers[4])
+    b2 = _torch_conv(b1, layers[5])
+    b3 = _torch_conv(b2, layers[6], residual=a3)        # identity shortcut: the block input itself
+    for got, want in zip(outs, (a1, a2, sc, a3, b1, b2, b3)):
+        want = _nhwc(want)
+        assert got.shape == want.shape
+        assert np.max(np.abs(got - want)) <= 2e-6 * max(1.0, float(np.max(np.abs(want))))
+    # the check has teeth: the same block with its shortcut taken from the wrong tensor is far away
+    assert float(np.max(np.abs(_nhwc(b3) - _nhwc(_torch_conv(b2, layers[6], residual=sc))))) > 0.1
+    # ---- inverted-residual blocks as the MobileNetV2-shaped builder lays them out: stem, t=1 block (no expand,
+    # no residual: 32 -> 16), t=6 stride-2 block (no residual), t=6 stride-1 block with Cin == Cout (residual)
+    mv = wl.mobilenetv2_ee(seed=2, in_hw=32, n_classes=10, max_batch=2, dtype="f32")
+    st = mv.stages[0]
+    L = st.layers
+    assert [l.op for l in L[:9]] == [wl.OP_CONV, wl.OP_DWCONV, wl.OP_CONV, wl.OP_CONV, wl.OP_DWCONV, wl.OP_CONV,
+                                     wl.OP_CONV, wl.OP_DWCONV, wl.OP_CONV]
+    x_np = wl.make_input(mv, 2, seed=6)
+    outs = eo.run_layers(mv, 0, x_np, keep_all=True)
+    x = torch.from_numpy(x_np.astype(np.float64)).permute(0, 3, 1, 2)
+    s0 = _torch_conv(x, L[0])                           # stem 3x3 s2
+    d1 = _torch_conv(s0, L[1])                          # block 1 (t = 1): depthwise straight on the block input
+    p1 = _torch_conv(d1, L[2])                          # linear projection 32 -> 16, no residual (Cin != Cout)
+    e2 = _torch_conv(p1, L[3])                          # block 2: expand
+    d2 = _torch_conv(e2, L[4])                          # depthwise stride 2
+    p2 = _torch_conv(d2, L[5])                          # projection, no residual (stride 2)
+    e3 = _torch_conv(p2, L[6])                          # block 3: expand
+    d3 = _torch_conv(e3, L[7])                          # depthwise stride 1
+    p3 = _torch_conv(d3, L[8], residual=p2)             # projection + the block input (stride 1, 24 -> 24)
+    assert L[8].residual_from != wl.NO_RESIDUAL and L[5].residual_from == wl.NO_RESIDUAL and L[2].residual_from == wl.NO_RESIDUAL
+    for got, want in zip(outs[:9], (s0, d1, p1, e2, d2, p2, e3, d3, p3)):
+        want = _nhwc(want)
+        assert got.shape == want.shape
+        assert np.max(np.abs(got - want)) <= 2e-6 * max(1.0, float(np.max(np.abs(want))))
+    # the stage output is the last layer's; run_layers without keep_all returns exactly it
+    assert np.array_equal(eo.run_layers(mv, 0, x_np), outs[st.out_layer])
+
+
+def _run_layers_fp32_accumulator(model, stage, x):
+    """The stage's layers with the SAME arithmetic as the oracle except that every accumulator is rounded to fp32
+    once before an fp32 epilogue (what any fp32-accumulating implementation does at best): a second correct
+    implementation, built from the oracle's raw convolution sums and numpy."""
+    st = model.stages[stage]
+    outs = []
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    for i, l in enumerate(st.layers):
+        src = x if (l.input_from == wl.FROM_STAGE_INPUT or (l.input_from == wl.FROM_PREV and i == 0)) else \
+            (outs[i - 1] if l.input_from == wl.FROM_PREV else outs[l.input_from])
+        if l.op == wl.OP_MAXPOOL:
+            outs.append(eo.maxpool(src, l.kh, l.stride, l.pad))
+            continue
+        res = x if l.residual_from == wl.FROM_STAGE_INPUT else (outs[l.residual_from] if l.residual_from >= 0 else None)
+        y = eo.conv2d(src, l.weight, l.stride, l.pad, l.groups) * l.scale.astype(np.float32) + l.bias.astype(np.float32)
+        if res is not None:
+            y = y + res
+        y = np.maximum(y, 0) if l.act == wl.ACT_RELU else (np.clip(y, 0, 6) if l.act == wl.ACT_RELU6 else y)
+        outs.append(wl.to_bf16_grid(y.astype(np.float32)))
+    return outs[st.out_layer]
+
+
+@pytest.mark.parametrize("name", ["resnet50", "mobilenetv2"])
+def test_bf16_chain_drift_between_two_correct_cpu_implementations(name):
+    """Why whole bf16 stages are not held element-wise to 1e-2: two CPU implementations of the benchmark's stages
+    that differ only by one fp32 rounding of each accumulator agree on most elements bit for bit, yet a measurable
+    share of the elements ends up more than 1e-2 apart (each flipped bf16 rounding perturbs everything downstream),
+    while the max-norm stays within two bf16 ulps and the L2 error between 1e-3 and 6e-3.  The stage bars of the GPU parity tests
+    (tests/util.py: STAGE_TOL, STAGE_L2, STAGE_EXCEED) must admit this pair, and the drift must be real (otherwise the
+    element-wise bar could be asked of whole stages)."""
+    from tests import util
+
+    spec = wl.resnet50_ee(seed=1, max_batch=2) if name == "resnet50" else wl.mobilenetv2_ee(seed=2, max_batch=2)
+    x = wl.make_input(spec, 2, seed=1)
+    worst_share = 0.0
+    for s in range(4):
+        a = eo.run_layers(spec, s, x)
+        b = _run_layers_fp32_accumulator(spec, s, x)
+        share = util.exceed_share(b, a, util.TOL["bf16"], util.STAGE_FLOOR)
+        worst_share = max(worst_share, share)
+        assert util.norm_err(b, a) <= util.STAGE_TOL["bf16"]
+        assert util.l2_err(b, a) <= util.STAGE_L2["bf16"]
+        assert share <= util.STAGE_EXCEED
+        assert float(np.mean(a != b)) > 1e-3                 # the two do part ways
+        x = a
+    assert worst_share > 1e-2                                # ... by more than the element-wise bar, for whole percents of a stage
+
+
 def test_serve_trace_bookkeeping():
     n, bmax = 200, 8
     arr = wl.poisson_arrivals(3, n, 1000.0)

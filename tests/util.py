@@ -11,32 +11,67 @@ from paper_2209_13443_b200 import workloads as wl
 
 # Parity bars (max relative error of features and logits against the fp64 oracle):
 #   fp32 path 1e-5, bf16 activations with fp32 accumulation 1e-2.
-# "Relative" is taken element-wise against max(|oracle|, FLOOR * max|oracle|).  Post-ReLU maps contain
-# exact zeros and values far below the tensor's scale, where a pure element-wise ratio is undefined, and
-# the rounding error of a length-K fp32 dot product scales with sum|x_i w_i| (the tensor's scale), not with
-# the element's own value: an element at 1e-3 of the scale legitimately carries ~K*2^-24/1e-3 relative
-# error in ANY fp32 summation order.  FLOOR = 0.05 keeps the bar meaningful for every element that
-# matters and still bounds the small ones in absolute terms (tol * 0.05 * scale).
+# "Relative" is taken element-wise against max(|oracle|, FLOOR * max|oracle|): post-ReLU maps contain exact
+# zeros, where a pure element-wise ratio is undefined.
+#   bf16: FLOOR = 1e-3.  Both sides round the same pre-activation once to bf16, so an element differs by at most
+#         one bf16 ulp of its own magnitude (2^-8 relative) plus the fp32 accumulation error, which is far below
+#         that ulp for every element above 1e-3 of the tensor's scale.
+#   fp32: FLOOR = 0.05.  The rounding error of a length-K fp32 dot product scales with sum|x_i w_i| (the
+#         tensor's scale), not with the element's own value: an element at 1e-3 of the scale legitimately
+#         carries ~sqrt(K) * 2^-24 / 1e-3 relative error in ANY fp32 summation order (measured 3.7e-5 on the
+#         tiny model), so the 1e-5 bar can only be asked of elements that are not small against the scale.
+#         The value of the 1e-3-floor metric is still computed and returned (rel_err_floor3) so it is on record.
 TOL = {"f32": 1e-5, "bf16": 1e-2}
 # Whole stages of a bf16 model (10-19 layers, each output rounded to bf16 on both sides) are held to two bf16 ulps in
 # the max-norm, 2^-6: a legitimate last-bit difference early in the chain moves later pre-rounding values across
 # rounding boundaries, so the largest elements of a 10^7-element map end up one to two ulps (2^-7 each at the bottom
 # of a binade) apart in ANY correct implementation.  The 1e-2 bar itself is enforced layer by layer
-# (test_every_layer_of_the_full_size_models), where both sides round the same pre-activation once.
+# (test_every_layer_of_the_full_size_models), where both sides round the same pre-activation once.  For whole
+# stages the relaxation is measured, not open-ended: besides the max-norm, the same two-ulp bar is applied to the error
+# in the L2 norm relative to the tensor's L2 norm (STAGE_L2: a dropped term or a wrong operand is O(0.1-1) there, the
+# rounding drift 1e-3 to 5e-3), and the elements whose floored error exceeds 1e-2 are counted like the near-threshold samples
+# with their share bounded by STAGE_EXCEED.  Two correct CPU implementations that differ by a single fp32 rounding of
+# the accumulator drift by the same kind of amount over these chains (test_oracle_pins.py:
+# test_bf16_chain_drift_between_two_correct_cpu_implementations: up to 13 % of a stage's elements), which is where
+# the bound comes from.
 STAGE_TOL = {"f32": 1e-5, "bf16": 2.0 ** -6}
-FLOOR = 0.05
+STAGE_L2 = {"f32": 1e-5, "bf16": 2.0 ** -6}
+FLOOR = {"f32": 0.05, "bf16": 1e-3}
+STAGE_FLOOR = 0.05          # floor of the element count over whole bf16 stages
+STAGE_EXCEED = 0.25         # largest tolerated share of a stage's elements off by more than 1e-2 (floored at STAGE_FLOOR)
 BAND = 1e-3   # samples whose oracle confidence is within BAND of the threshold may flip; they are listed and counted
+CANARY = 0xA5
+GUARD_BYTES = 4096
 
 
-def rel_err(a: np.ndarray, o: np.ndarray) -> float:
+def _floored(a, o, floor):
     a = np.asarray(a, dtype=np.float64)
     o = np.asarray(o, dtype=np.float64)
+    scale = float(np.max(np.abs(o))) if o.size else 0.0
+    if o.size == 0:
+        return np.zeros(0)
+    if scale == 0.0:
+        return np.abs(a)
+    return np.abs(a - o) / np.maximum(np.abs(o), floor * scale)
+
+
+def rel_err(a: np.ndarray, o: np.ndarray, dtype: str = "bf16", floor=None) -> float:
+    r = _floored(a, o, FLOOR[dtype] if floor is None else floor)
+    return float(np.max(r)) if r.size else 0.0
+
+
+def exceed_share(a, o, tol, floor) -> float:
+    """Share of the elements whose floored relative error is above ``tol``."""
+    r = _floored(a, o, floor)
+    return float(np.mean(r > tol)) if r.size else 0.0
+
+
+def l2_err(a, o) -> float:
+    a = np.asarray(a, dtype=np.float64).ravel()
+    o = np.asarray(o, dtype=np.float64).ravel()
     if o.size == 0:
         return 0.0
-    scale = float(np.max(np.abs(o)))
-    if scale == 0.0:
-        return float(np.max(np.abs(a)))
-    return float(np.max(np.abs(a - o) / np.maximum(np.abs(o), FLOOR * scale)))
+    return float(np.linalg.norm(a - o) / max(float(np.linalg.norm(o)), 1e-30))
 
 
 def norm_err(a, o) -> float:
@@ -47,6 +82,30 @@ def norm_err(a, o) -> float:
     return float(np.max(np.abs(a - o)) / max(float(np.max(np.abs(o))), 1e-30))
 
 
+def guarded(shape, dtype, device="cuda"):
+    """A tensor of ``shape`` followed by GUARD_BYTES canary bytes in the same allocation.  Returns (view, guard)."""
+    n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+    pad = (-n) % 16
+    raw = torch.empty(n + pad + GUARD_BYTES, dtype=torch.uint8, device=device)
+    raw[n:].fill_(CANARY)
+    return raw[:n].view(dtype).view(shape), raw[n:]
+
+
+def guard_stage_buffers(bufs: "eb.StageBuffers"):
+    """Moves every device buffer of a StageBuffers into a guarded allocation; returns the list of guards."""
+    guards = []
+    for name in ("features_out", "conf", "pred", "logits", "exit_mask", "survivor_idx", "ids_out", "n_surv_dev"):
+        t = getattr(bufs, name)
+        if t is None:
+            continue
+        view, g = guarded(tuple(t.shape), t.dtype, t.device)
+        view.copy_(t)
+        setattr(bufs, name, view)
+        guards.append((name, g))
+    bufs._struct = None
+    return guards
+
+
 class GpuRunner:
     """One model on the GPU with the buffers a caller allocates once (sized for max_batch)."""
 
@@ -54,7 +113,19 @@ class GpuRunner:
         self.spec = spec
         self.m = eb.EEModel(spec)
         self.bufs = [eb.StageBuffers(self.m, s) for s in range(self.m.n_stages)]
-        self.ws = self.m.workspace()
+        # canary bytes behind every output buffer and behind the workspace (the workspace is handed to the library
+        # at exactly the size ee_model_query reports), checked after every call
+        self.guards = []
+        for s, b in enumerate(self.bufs):
+            self.guards += [(f"stage {s} {n}", g) for n, g in guard_stage_buffers(b)]
+        need = max(self.m.query(s)["workspace_bytes"] for s in range(self.m.n_stages))
+        self.ws, g = guarded((need,), torch.uint8)
+        assert self.ws.data_ptr() % 256 == 0
+        self.guards.append(("workspace", g))
+
+    def check_guards(self):
+        for name, g in self.guards:
+            assert bool(torch.all(g == CANARY)), f"bytes past the end of {name} were overwritten"
 
     def stage(self, s, x_np, ids=None, shift=None, shift_cls=None):
         """Runs stage ``s`` on host features ``x_np``; returns host copies of every output."""
@@ -68,6 +139,7 @@ class GpuRunner:
         self.m.stage_run(s, x, B, out, self.ws, ids_d, sh, sc)
         torch.cuda.synchronize()
         self.m.check()
+        self.check_guards()
         n = int(out.n_surv_host[0])
         assert n == int(out.n_surv_dev.cpu()[0])
         return {
@@ -91,14 +163,17 @@ def check_stage(spec, g: dict, o: dict, where="", tol=None, elementwise=False):
     element-wise ratio is not a property of an implementation: one legitimate last-bit difference
     perturbs every downstream pre-rounding value, and each perturbed value that straddles a bf16
     rounding boundary moves by a full ulp (2^-8 relative), so individual elements drift by a few
-    percent in any summation order while the max-norm error stays near one ulp."""
+    percent in any summation order while the max-norm error stays near one ulp.  For such chains the
+    elements off by more than the 1e-2 bar are counted (floor STAGE_FLOOR) and their share is bounded by
+    STAGE_EXCEED; the unfloored max-norm error and the 1e-3-floor metric are returned for the record."""
+    dt = spec.dtype
     if tol is None:
-        tol = TOL[spec.dtype] if elementwise else STAGE_TOL[spec.dtype]
-    ferr = rel_err if elementwise else norm_err
+        tol = TOL[dt] if elementwise else STAGE_TOL[dt]
+    ferr = (lambda a, b: rel_err(a, b, dt)) if elementwise else norm_err
     B = len(o["conf"])
     st_thr = o.get("threshold")
     e_z = ferr(g["z"], o["z"])
-    assert e_z <= TOL[spec.dtype], f"{where}: logits rel err {e_z:.3e} > {TOL[spec.dtype]}"
+    assert e_z <= TOL[dt], f"{where}: logits rel err {e_z:.3e} > {TOL[dt]}"
     # softmax top-1 is 1/2-Lipschitz in the max-norm of the logits (d conf = conf (1 - conf) d(z_top - z_k)):
     # the confidence may move by at most half the largest logit difference, plus fp32 rounding of the exp-sum
     dz = np.max(np.abs(g["z"] - o["z"]), axis=1) if B else np.zeros(0)
@@ -119,13 +194,22 @@ def check_stage(spec, g: dict, o: dict, where="", tol=None, elementwise=False):
         assert g["n_surv"] == o["n_surv"] and np.array_equal(g["surv_idx"], o["surv_idx"]), f"{where}: compaction"
         if o.get("ids_out") is not None:
             assert np.array_equal(g["ids_out"], o["ids_out"]), f"{where}: ids"
-        e_f = ferr(g["features_out"], o["features_out"])
-        assert e_f <= tol, f"{where}: features rel err {e_f:.3e} > {tol}"
+        want_f = o["features_out"]
     else:
-        so = o["stage_out"][g["surv_idx"]]
-        e_f = ferr(g["features_out"], so)
-        assert e_f <= tol, f"{where}: features rel err {e_f:.3e} > {tol}"
-    return {"z_err": e_z, "feat_err": e_f, "band": int(band.sum()), "flips": flips}
+        want_f = o["stage_out"][g["surv_idx"]]
+    e_f = ferr(g["features_out"], want_f)
+    assert e_f <= tol, f"{where}: features rel err {e_f:.3e} > {tol}"
+    stats = {"z_err": e_z, "feat_err": e_f, "band": int(band.sum()), "flips": flips,
+             "feat_norm_err": norm_err(g["features_out"], want_f),
+             "feat_err_floor3": rel_err(g["features_out"], want_f, dt, floor=1e-3)}
+    if not elementwise:
+        stats["feat_l2_err"] = l2_err(g["features_out"], want_f)
+        assert stats["feat_l2_err"] <= STAGE_L2[dt], f"{where}: features L2 rel err {stats['feat_l2_err']:.3e} > {STAGE_L2[dt]}"
+        share = exceed_share(g["features_out"], want_f, TOL[dt], STAGE_FLOOR)
+        stats["exceed_share"] = share
+        stats["exceed_share_floor3"] = exceed_share(g["features_out"], want_f, TOL[dt], 1e-3)
+        assert share <= STAGE_EXCEED, f"{where}: {share:.2e} of the elements are off by more than {TOL[dt]} (bound {STAGE_EXCEED})"
+    return stats
 
 
 def oracle_stage(spec, s, x_np, ids=None, shift=None, shift_cls=None):
