@@ -238,6 +238,28 @@ typedef struct {
 } ee_layer_plan_t;
 ee_status_t ee_model_plan(const ee_model_t* model, int stage, int batch, int cap, ee_layer_plan_t* out, int* n);
 
+/* Per-(layer, batch) kernel table.  The paper's NPU looks up, for every (layer, active batch size), how to map the batch
+ * onto its array (Section III-A Eq. 1; Section III-C: an L x B_max table addressed by (l, B_act)) and fills the table
+ * offline by an exhaustive search over the design space (Section III-D Eq. 2).  Here the table holds, for every
+ * tensor-core layer and every batch size 1..max_batch, which kernel variant runs the layer:
+ *   0  one-CTA tiles (128 x 128 or 128 x 64; one-tile, persistent or cluster split-K kernels chosen from the grid),
+ *   1  CTA pairs, 256 x 256 tiles (tcgen05 cta_group::2, persistent (tile, K-range) units),
+ *   2  CTA pairs, 256 x 128 tiles.
+ * The number of K ranges of a layer (`splits`) is one value per layer for all batch sizes and all variants, and the
+ * partial sums of the ranges are always added in ascending order, so a sample's result is bit-identical whichever
+ * variant the table picks for the batch it rides in.  Both setters drop the stage's captured graphs.
+ * ee_model_set_layer_splits may change ee_stage_info_t.workspace_bytes: query again before the next run.
+ * ee_model_get_layer_config: tensor_core = -1 (not a tensor-core layer with a table), else the highest variant the
+ * layer supports.  Errors: INVALID_ARG, STAGE, CAPACITY (batch range beyond max_batch; partial tiles of more than 256 MB),
+ * UNSUPPORTED (the layer cannot run as that variant). */
+ee_status_t ee_model_set_layer_variant(ee_model_t* model, int stage, int layer, int batch_lo, int batch_hi, int variant);
+ee_status_t ee_model_set_layer_splits(ee_model_t* model, int stage, int layer, int splits);
+ee_status_t ee_model_get_layer_config(const ee_model_t* model, int stage, int layer, int batch, int* variant, int* splits,
+                                      int* tensor_core);
+
+/* Limit, in SM clock cycles, of the bounded device-side waits (default about 2 s).  Errors: INVALID_ARG. */
+ee_status_t ee_model_set_wait_limit(ee_model_t* model, long long cycles);
+
 /* Runs a batch from stage `first_stage` on until it is empty or the last stage has been launched: ee_stage_run for a
  * stage, the host's wait for its survivor count (the protocol of ee_wait_count on outs[s].n_surv_host, which must be
  * a pinned host word for every stage but the last), then the next stage on the survivors (features_out / ids_out of

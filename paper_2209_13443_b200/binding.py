@@ -21,7 +21,8 @@ STATUS_NAMES = ["EE_OK", "EE_ERR_INVALID_ARG", "EE_ERR_SHAPE", "EE_ERR_CAPACITY"
                 "EE_ERR_CUDA", "EE_ERR_TIMEOUT", "EE_ERR_INTERNAL"]
 EXPORTS = ["ee_model_create", "ee_model_destroy", "ee_model_query", "ee_stage_run", "ee_layer_run", "ee_batch_refill", "ee_exit_head",
            "ee_exit_head_scratch_bytes", "ee_exit_head_static", "ee_gather_survivors", "ee_model_set_graphs", "ee_model_set_timing", "ee_model_get_timing",
-           "ee_model_plan", "ee_model_check", "ee_wait_count", "ee_run_until_exit", "ee_status_string", "ee_last_cuda_error"]
+           "ee_model_plan", "ee_model_check", "ee_model_set_layer_variant", "ee_model_set_layer_splits", "ee_model_get_layer_config",
+           "ee_model_set_wait_limit", "ee_wait_count", "ee_run_until_exit", "ee_status_string", "ee_last_cuda_error"]
 
 
 class EEError(RuntimeError):
@@ -99,6 +100,10 @@ def load_library() -> C.CDLL:
     L.ee_run_until_exit.argtypes = [vp, i, C.POINTER(StageIn), vp, C.c_size_t, C.POINTER(StageOut), C.POINTER(C.c_int32), C.c_double, vp]
     L.ee_wait_count.argtypes = [vp, C.c_int32, C.c_double, C.POINTER(C.c_int32)]
     L.ee_model_check.argtypes = [vp, vp]
+    L.ee_model_set_layer_variant.argtypes = [vp, i, i, i, i, i]
+    L.ee_model_set_layer_splits.argtypes = [vp, i, i, i]
+    L.ee_model_get_layer_config.argtypes = [vp, i, i, i, C.POINTER(i), C.POINTER(i), C.POINTER(i)]
+    L.ee_model_set_wait_limit.argtypes = [vp, C.c_longlong]
     L.ee_status_string.argtypes = [i]
     L.ee_status_string.restype = C.c_char_p
     L.ee_last_cuda_error.restype = C.c_char_p
@@ -313,6 +318,20 @@ class EEModel:
         return [dict(kernel=arr[i].kernel.decode(), m=arr[i].m, n=arr[i].n, k=arr[i].k, flops=arr[i].flops, bytes=arr[i].bytes,
                      launches=arr[i].launches)
                 for i in range(n.value)]
+
+    def set_layer_variant(self, stage: int, layer: int, batch_lo: int, batch_hi: int, variant: int):
+        _check(self._L.ee_model_set_layer_variant(self._h, stage, layer, batch_lo, batch_hi, variant), "ee_model_set_layer_variant")
+
+    def set_layer_splits(self, stage: int, layer: int, splits: int):
+        _check(self._L.ee_model_set_layer_splits(self._h, stage, layer, splits), "ee_model_set_layer_splits")
+
+    def layer_config(self, stage: int, layer: int, batch: int) -> dict:
+        v, s, t = C.c_int(0), C.c_int(0), C.c_int(0)
+        _check(self._L.ee_model_get_layer_config(self._h, stage, layer, batch, C.byref(v), C.byref(s), C.byref(t)), "ee_model_get_layer_config")
+        return {"variant": v.value, "splits": s.value, "tensor_core": t.value}
+
+    def set_wait_limit(self, cycles: int):
+        _check(self._L.ee_model_set_wait_limit(self._h, int(cycles)), "ee_model_set_wait_limit")
 
     def check(self, stream=None):
         _check(self._L.ee_model_check(self._h, _stream(stream)), "ee_model_check")

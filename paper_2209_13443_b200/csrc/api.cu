@@ -12,6 +12,7 @@
 #include "conv_tc.cuh"
 #include "conv_stem.cuh"
 #include "conv_halo.cuh"
+#include "conv_pair.cuh"
 #include "conv_dw.cuh"
 #include "head.cuh"
 
@@ -44,6 +45,10 @@ struct LayerPlan {
   float* scale_dev = nullptr;
   float* bias_dev = nullptr;
   TcLayer tc;  // tensor-core plan (valid iff kind == KK_TC or KK_TC_GATHER)
+  // Kernel variant per batch size, index 0..max_batch (TcVariant; empty = TCV_AUTO everywhere).  The analogue of the
+  // paper's per-(layer, batch) look-up table that configures the array for the active batch (Section III-C): the
+  // variant may change with the batch, the layer's K ranges (tc.splits) may not.
+  std::vector<uint8_t> variant;
 };
 
 struct StageCallKey {  // everything that distinguishes one ee_stage_run call from another
@@ -69,6 +74,7 @@ struct StagePlan {
   int in_h, in_w, in_c, out_h, out_w, out_c, out_slot;
   std::vector<size_t> slot_off;  // byte offsets at max_batch
   size_t head_off = 0, ws_bytes = 0, head_bytes = 0;
+  size_t split_off = 0, split_bytes = 0;   // split-K partial tiles of the pair kernel, behind the head scratch
   int n_classes = 0;
   void* fc_w = nullptr;
   float* fc_b = nullptr;
@@ -125,6 +131,10 @@ struct ee_model {
   std::vector<StagePlan> stages;
   std::vector<void*> owned;  // device allocations
   int* err_flag = nullptr;   // device word set by kernels whose bounded waits ran out
+  unsigned* pair_counters = nullptr;   // arrival counters of the pair kernel's split-K reduction; zero between launches
+  size_t pair_counter_words = 0;
+  long long wait_cycles = kTcWaitCycles;   // limit of the bounded device-side waits of the pair kernel and the self-test
+  int device = -1;           // the GPU the model lives on
   bool timing = false;
   bool graphs = true;  // replay stages as CUDA graphs on capturable streams
   TcContext tc;
@@ -163,8 +173,21 @@ void record(ee_model* m, StagePlan& sp, cudaStream_t st, const char* name) {
   cudaEventRecord(sp.ev[sp.ev_used++], st);
 }
 
+// Recomputes the workspace layout of a stage behind its layer slots: head scratch, then the split-K partial tiles of
+// the layers that may run on the pair kernel.
+void layout_stage_tail(ee_model* m, StagePlan& sp) {
+  size_t need = 0;
+  for (const LayerPlan& L : sp.layers)
+    if (L.kind == KK_TC && !L.tc.gather && !L.tc.halo && L.tc.splits > 1)
+      need = std::max(need, std::max(pair_partial_bytes(L.tc, m->max_batch, 256), pair_partial_bytes(L.tc, m->max_batch, 128)));
+  sp.split_off = align_up(sp.head_off + sp.head_bytes, 1024);
+  sp.split_bytes = need;
+  sp.ws_bytes = sp.split_off + need;
+}
+
 template <typename T>
-ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const void* res, void* dst, int B, cudaStream_t st) {
+ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const void* res, void* dst, int B, float* partial,
+                         size_t partial_bytes, cudaStream_t st) {
   ConvGeom g{B, L.in_h, L.in_w, L.d.cin, L.out_h, L.out_w, L.d.cout, L.d.kh, L.d.kw, L.d.stride, L.d.pad, L.d.act};
   constexpr int V = Elem<T>::kVec;
   switch (L.kind) {
@@ -175,8 +198,16 @@ ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const
       break;
     }
     case KK_TC: {
-      ee_status_t s = L.tc.halo ? halo_launch(m->tc, L.tc, src, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st)
-                                : tc_launch(m->tc, L.tc, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st);
+      const int v = L.variant.empty() ? (int)TCV_AUTO : (int)L.variant[B];
+      ee_status_t s = EE_ERR_INTERNAL;
+      if constexpr (sizeof(T) == 2) {
+        if (v != TCV_AUTO && pair_supported(L.tc, v))
+          s = pair_launch(m->tc, L.tc, v, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, partial, partial_bytes, m->pair_counters,
+                          m->wait_cycles, st);
+        else
+          s = L.tc.halo ? halo_launch(m->tc, L.tc, src, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st)
+                        : tc_launch(m->tc, L.tc, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st);
+      }
       if (s != EE_OK) return s;
       break;
     }
@@ -315,8 +346,9 @@ ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, c
     const void* src = L.src_slot < 0 ? in->features : ws + sp.slot_off[L.src_slot];
     const void* res = L.res_slot == -2 ? nullptr : (L.res_slot == -1 ? in->features : ws + sp.slot_off[L.res_slot]);
     void* dst = ws + sp.slot_off[L.out_slot];
-    ee_status_t s = m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, src, res, dst, B, st)
-                                        : launch_layer<float>(m, L, src, res, dst, B, st);
+    float* partial = (float*)(ws + sp.split_off);
+    ee_status_t s = m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, src, res, dst, B, partial, sp.split_bytes, st)
+                                        : launch_layer<float>(m, L, src, res, dst, B, partial, sp.split_bytes, st);
     if (s != EE_OK) return s;
     record(m, sp, st, kKernelNames[L.kind]);
   }
@@ -398,6 +430,10 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
   m->in_w = desc->in_w;
   m->in_c = desc->in_c;
   m->max_batch = desc->max_batch;
+  if (cudaGetDevice(&m->device) != cudaSuccess) {
+    delete m;
+    return EE_ERR_CUDA;
+  }
   const size_t es = esize(desc->dtype);
   const int ondev = desc->weights_on_device;
   ee_status_t rc = EE_OK;
@@ -420,6 +456,7 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
   rc = tc_context_init(m->tc);
   if (rc == EE_OK) rc = stem_context_init();
   if (rc == EE_OK) rc = halo_context_init();
+  if (rc == EE_OK) rc = pair_context_init();
   if (rc == EE_OK) rc = dw_context_init();
   if (rc != EE_OK) return fail(rc);
 
@@ -524,7 +561,7 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
     HeadLayout hl = head_layout(desc->max_batch, sp.out_c, sd.n_classes);
     sp.head_off = align_up(off, 1024);
     sp.head_bytes = hl.bytes;
-    sp.ws_bytes = sp.head_off + hl.bytes;
+    sp.ws_bytes = sp.head_off + hl.bytes;   // the split-K region is added once the layers are planned
     sp.n_classes = sd.n_classes;
     sp.threshold = sd.threshold;
     sp.always_exit = sd.always_exit;
@@ -623,9 +660,19 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
       sp.gather_rev = !sp.gap_rev;
       in_rev = sp.gather_rev;
     }
+    layout_stage_tail(m, sp);
+    for (const LayerPlan& L : sp.layers)
+      if (L.kind == KK_TC && !L.tc.gather && !L.tc.halo) m->pair_counter_words = std::max(m->pair_counter_words, pair_counter_words(L.tc, desc->max_batch));
     if ((rc = upload_bytes(m, sd.fc_weight, (size_t)sd.n_classes * sp.out_c * es, ondev, st, &sp.fc_w)) != EE_OK) return fail(rc);
     if ((rc = upload<float>(m, sd.fc_bias, sd.n_classes, ondev, st, &sp.fc_b)) != EE_OK) return fail(rc);
     h = sp.out_h, w = sp.out_w, c = sp.out_c;
+  }
+  if (m->pair_counter_words) {
+    void* p = nullptr;
+    if (cudaMalloc(&p, m->pair_counter_words * sizeof(unsigned)) != cudaSuccess) return fail(EE_ERR_CUDA);
+    m->owned.push_back(p);
+    m->pair_counters = (unsigned*)p;
+    if (cudaMemsetAsync(p, 0, m->pair_counter_words * sizeof(unsigned), st) != cudaSuccess) return fail(EE_ERR_CUDA);
   }
   if (cudaStreamSynchronize(st) != cudaSuccess) return fail(EE_ERR_CUDA);
   *out = m;
@@ -760,11 +807,16 @@ ee_status_t ee_layer_run(ee_model_t* m, int stage, int layer, const void* input,
   const bool has_res = L.res_slot != -2;
   if (!input || !output || (has_res && !residual) || ((uintptr_t)input & 15) || ((uintptr_t)output & 15) || ((uintptr_t)residual & 15))
     return EE_ERR_INVALID_ARG;
-  (void)workspace;
-  (void)workspace_bytes;
+  // the only scratch a layer may need: the split-K partial tiles of the pair kernel, at their place in the stage workspace
+  float* partial = nullptr;
+  size_t partial_bytes = 0;
+  if (workspace && !((uintptr_t)workspace & 255) && workspace_bytes >= sp.split_off + sp.split_bytes) {
+    partial = (float*)((char*)workspace + sp.split_off);
+    partial_bytes = sp.split_bytes;
+  }
   cudaStream_t st = (cudaStream_t)cuda_stream;
-  return m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, input, has_res ? residual : nullptr, output, batch, st)
-                             : launch_layer<float>(m, L, input, has_res ? residual : nullptr, output, batch, st);
+  return m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, input, has_res ? residual : nullptr, output, batch, partial, partial_bytes, st)
+                             : launch_layer<float>(m, L, input, has_res ? residual : nullptr, output, batch, partial, partial_bytes, st);
 }
 
 ee_status_t ee_batch_refill(ee_model_t* m, int boundary, void* batch_feat, int32_t* batch_ids, int n_surv, const void* arr_feat,
@@ -924,6 +976,59 @@ ee_status_t ee_model_plan(const ee_model_t* m, int stage, int batch, int cap, ee
   return EE_OK;
 }
 
+ee_status_t ee_model_set_layer_variant(ee_model_t* m, int stage, int layer, int batch_lo, int batch_hi, int variant) {
+  if (!m || variant < 0 || variant >= TCV_COUNT || batch_lo < 1 || batch_hi < batch_lo) return EE_ERR_INVALID_ARG;
+  if (stage < 0 || stage >= (int)m->stages.size()) return EE_ERR_STAGE;
+  StagePlan& sp = m->stages[stage];
+  if (layer < 0 || layer >= (int)sp.layers.size()) return EE_ERR_STAGE;
+  if (batch_hi > m->max_batch) return EE_ERR_CAPACITY;
+  LayerPlan& L = sp.layers[layer];
+  if (variant != TCV_AUTO && (L.kind != KK_TC || !pair_supported(L.tc, variant))) return EE_ERR_UNSUPPORTED;
+  if (L.variant.empty()) L.variant.assign((size_t)m->max_batch + 1, (uint8_t)TCV_AUTO);
+  for (int b = batch_lo; b <= batch_hi; ++b) L.variant[b] = (uint8_t)variant;
+  for (auto& g : sp.graphs) cudaGraphExecDestroy(g.exec);   // captured stages hold the old choice
+  sp.graphs.clear();
+  return EE_OK;
+}
+
+ee_status_t ee_model_set_layer_splits(ee_model_t* m, int stage, int layer, int splits) {
+  if (!m) return EE_ERR_INVALID_ARG;
+  if (stage < 0 || stage >= (int)m->stages.size()) return EE_ERR_STAGE;
+  StagePlan& sp = m->stages[stage];
+  if (layer < 0 || layer >= (int)sp.layers.size()) return EE_ERR_STAGE;
+  LayerPlan& L = sp.layers[layer];
+  if (L.kind != KK_TC || L.tc.gather || L.tc.halo) return EE_ERR_UNSUPPORTED;
+  TcLayer trial = L.tc;
+  if (!tc_set_splits(trial, splits)) return EE_ERR_INVALID_ARG;
+  if (std::max(pair_partial_bytes(trial, m->max_batch, 256), pair_partial_bytes(trial, m->max_batch, 128)) > ((size_t)256 << 20))
+    return EE_ERR_CAPACITY;
+  L.tc.splits = trial.splits, L.tc.kb_per = trial.kb_per;
+  layout_stage_tail(m, sp);
+  for (auto& g : sp.graphs) cudaGraphExecDestroy(g.exec);
+  sp.graphs.clear();
+  return EE_OK;
+}
+
+ee_status_t ee_model_get_layer_config(const ee_model_t* m, int stage, int layer, int batch, int* variant, int* splits, int* tensor_core) {
+  if (!m || batch < 0) return EE_ERR_INVALID_ARG;
+  if (stage < 0 || stage >= (int)m->stages.size()) return EE_ERR_STAGE;
+  const StagePlan& sp = m->stages[stage];
+  if (layer < 0 || layer >= (int)sp.layers.size()) return EE_ERR_STAGE;
+  if (batch > m->max_batch) return EE_ERR_CAPACITY;
+  const LayerPlan& L = sp.layers[layer];
+  const bool tc = L.kind == KK_TC && !L.tc.gather && !L.tc.halo;
+  if (variant) *variant = L.variant.empty() ? (int)TCV_AUTO : (int)L.variant[batch];
+  if (splits) *splits = L.kind == KK_TC ? L.tc.splits : 1;
+  if (tensor_core) *tensor_core = tc ? (pair_supported(L.tc, TCV_PAIR256) ? 2 : pair_supported(L.tc, TCV_PAIR128) ? 1 : 0) : -1;
+  return EE_OK;
+}
+
+ee_status_t ee_model_set_wait_limit(ee_model_t* m, long long cycles) {
+  if (!m || cycles < 1) return EE_ERR_INVALID_ARG;
+  m->wait_cycles = cycles;
+  return EE_OK;
+}
+
 ee_status_t ee_model_check(ee_model_t* m, void* cuda_stream) {
   if (!m) return EE_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -931,6 +1036,8 @@ ee_status_t ee_model_check(ee_model_t* m, void* cuda_stream) {
   EE_CUDA(cudaMemcpyAsync(&flag, m->err_flag, sizeof(int), cudaMemcpyDeviceToHost, st));
   EE_CUDA(cudaStreamSynchronize(st));
   if (flag) {
+    // a kernel that gave up may have left arrival counters of a split-K reduction behind
+    if (m->pair_counters) EE_CUDA(cudaMemsetAsync(m->pair_counters, 0, m->pair_counter_words * sizeof(unsigned), st));
     EE_CUDA(cudaMemsetAsync(m->err_flag, 0, sizeof(int), st));
     EE_CUDA(cudaStreamSynchronize(st));
     return EE_ERR_TIMEOUT;

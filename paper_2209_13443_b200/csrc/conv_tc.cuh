@@ -977,6 +977,7 @@ struct TcLayer {
   bool halo = false;    // the 3x3 halo-block kernel of conv_halo.cuh takes this layer
   int g_h = 0, g_w = 0, g_cin = 0, g_kh = 0, g_kw = 0, g_stride = 1, g_pad = 0, g_runp = 0;
   CUtensorMap tm_w;
+  CUtensorMap tm_w_half[2];   // the same weights with boxes of 128 and 64 filters: one CTA's half of a 256- or 128-wide pair tile
   struct Cached {
     const void* ptr;
     int batch;
@@ -1086,6 +1087,12 @@ inline ee_status_t tc_plan_layer(TcContext& c, const ee_layer_desc_t& d, int in_
   CUresult r = c.encode_tiled(&L->tm_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(w_dev), dims, strides, box, es,
                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  for (int i = 0; i < 2 && r == CUDA_SUCCESS; ++i) {
+    const cuuint32_t hbox[3] = {kTcBK, 1, (cuuint32_t)(i == 0 ? 128 : 64)};
+    r = c.encode_tiled(&L->tm_w_half[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(w_dev), dims, strides, hbox, es,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
   return r == CUDA_SUCCESS ? EE_OK : EE_ERR_CUDA;
 }
 
@@ -1216,6 +1223,18 @@ inline cudaError_t tc_launch_persistent(int ctas, cudaStream_t st, const CUtenso
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_persistent_kernel<BN, RES>, a, w, r, o, p);
+}
+
+// Sets the number of K ranges of a layer (1 = no split).  Ranges are equal runs of ceil(num_kb / splits) K blocks, the last
+// one shorter; returns false when a range would be empty or shorter than two K blocks.
+inline bool tc_set_splits(TcLayer& L, int splits) {
+  const int num_kb = L.kh * L.kw * cdiv(L.cin, kTcBK);
+  if (splits < 1 || splits > 8) return false;
+  const int per = cdiv(num_kb, splits);
+  if (splits > 1 && (per < 2 || (splits - 1) * per >= num_kb)) return false;
+  L.splits = splits;
+  L.kb_per = per;
+  return true;
 }
 
 inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, const void* res, void* dst, int B, const float* scale,

@@ -154,6 +154,55 @@ def test_narrow_pointwise_layer(geom):
         assert g["n_surv"] == B
 
 
+# layers forced onto the CTA-pair kernel (variant 1: 256 x 256 tiles, 2: 256 x 128 tiles) with a forced number of K ranges:
+# 1x1 and 3x3, stride 1 and 2, with and without residual, M tails (a pair whose second CTA has no valid row: 7x7 maps at
+# B = 1), N tails (200 and 136 columns), a K tail (136 channels), split-K through global memory with 2, 3 and 5 ranges
+PAIR_GEOMS = [
+    # H, W, cin, cout, k, stride, pad, act, residual, variant, splits
+    (14, 14, 256, 256, 1, 1, 0, wl.ACT_RELU, False, 1, 1),
+    (14, 14, 1024, 256, 1, 1, 0, wl.ACT_RELU, False, 1, 3),
+    (14, 14, 256, 1024, 1, 1, 0, wl.ACT_RELU, True, 1, 1),
+    (14, 14, 256, 256, 3, 1, 1, wl.ACT_RELU, False, 1, 3),
+    (28, 28, 128, 128, 3, 2, 1, wl.ACT_RELU, False, 2, 2),
+    (7, 7, 512, 2048, 1, 1, 0, wl.ACT_RELU, True, 1, 2),
+    (7, 7, 2048, 512, 1, 1, 0, wl.ACT_RELU, False, 1, 5),
+    (14, 14, 512, 512, 3, 2, 1, wl.ACT_NONE, False, 1, 3),
+    (9, 7, 136, 200, 3, 1, 1, wl.ACT_RELU6, False, 1, 2),
+    (9, 7, 136, 200, 1, 1, 0, wl.ACT_RELU6, True, 2, 1),
+    (13, 11, 64, 136, 3, 1, 1, wl.ACT_RELU, False, 2, 3),
+    (15, 9, 64, 256, 1, 2, 0, wl.ACT_NONE, False, 1, 1),
+]
+
+
+@pytest.mark.parametrize("geom", PAIR_GEOMS)
+def test_pair_kernel_layer(geom):
+    H, W, cin, cout, k, stride, pad, act, residual, variant, splits = geom
+    max_batch = 11
+    spec = util.single_layer_model("bf16", H, W, cin, cout, k, stride, pad, act, residual, seed=hash(geom) % 1000, max_batch=max_batch)
+    layer = 1 if residual else 0
+
+    def configure(m):
+        m.set_layer_splits(0, layer, splits)
+        m.set_layer_variant(0, layer, 1, max_batch, variant)
+        assert m.layer_config(0, layer, 3) == {"variant": variant, "splits": splits, "tensor_core": 2 if cout > 128 else 1}
+
+    m = eb.EEModel(spec)
+    configure(m)
+    ws, ws_guard = util.guarded((m.query(0)["workspace_bytes"],), torch.uint8)
+    for B in (1, 5, 11):
+        x = wl.random_features((B, H, W, cin), seed=B, bf16=True, relu=False)
+        outs = eo.run_layers(spec, 0, x, keep_all=True)        # the layer runs alone on the oracle's input and residual operand
+        res = eb.to_device("bf16", outs[0]) if residual else None
+        for rep in range(2):                                   # twice: the split-K counters must be back at zero
+            out, guard = util.guarded(outs[layer].shape, torch.bfloat16)
+            m.layer_run(0, layer, eb.to_device("bf16", x), res, B, out, ws)
+            torch.cuda.synchronize()
+            m.check()
+            assert bool(torch.all(guard == util.CANARY)) and bool(torch.all(ws_guard == util.CANARY))
+            e = util.rel_err(out.float().cpu().numpy(), outs[layer], "bf16")
+            assert e <= util.TOL["bf16"], f"pair {geom} B={B} run {rep}: {e:.3e}"
+
+
 @pytest.mark.parametrize("geom", HALO_GEOMS)
 def test_conv3x3_halo_layer(geom):
     H, W, cin, cout, act = geom

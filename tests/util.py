@@ -109,9 +109,11 @@ def guard_stage_buffers(bufs: "eb.StageBuffers"):
 class GpuRunner:
     """One model on the GPU with the buffers a caller allocates once (sized for max_batch)."""
 
-    def __init__(self, spec):
+    def __init__(self, spec, configure=None):
         self.spec = spec
         self.m = eb.EEModel(spec)
+        if configure is not None:           # e.g. force kernel variants or split counts before the buffers are sized
+            configure(self.m)
         self.bufs = [eb.StageBuffers(self.m, s) for s in range(self.m.n_stages)]
         # canary bytes behind every output buffer and behind the workspace (the workspace is handed to the library
         # at exactly the size ee_model_query reports), checked after every call
