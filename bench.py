@@ -52,15 +52,10 @@ def load_peaks():
 def make_spec(workload: str, batch: int, flat_heads: bool = False):
     from paper_2209_13443_b200 import workloads as wl
 
-    if workload == "resnet50":
-        # flat_heads: FC weights scaled down so that unshifted confidences sit near 1/1000 and only the forced
-        # Bernoulli logit shifts of the exit-rate sweep decide who leaves
-        return wl.resnet50_ee(seed=1, max_batch=batch, alphas=[0.01] * 4 if flat_heads else None), 1
-    if workload == "mobilenetv2":
-        return wl.mobilenetv2_ee(seed=2, max_batch=batch), 2
-    if workload == "tiny":
-        return wl.tiny_ee_cnn(seed=0, max_batch=batch), 0
-    raise SystemExit(f"unknown workload {workload}")
+    try:
+        return wl.benchmark_model(workload, batch, flat_heads)
+    except ValueError as e:
+        raise SystemExit(str(e))
 
 
 def workload_name(spec, batch, exit_rate=None):

@@ -195,8 +195,9 @@ size_t ee_exit_head_scratch_bytes(const ee_model_t* model, int stage);
  * the library image (each GPU that loads the library holds it until the process exits).
  *   - A model/shape whose head needs more than EE_STATIC_HEAD_SCRATCH_BYTES (what ee_exit_head_scratch_bytes reports
  *     for the stage) is refused with EE_ERR_CAPACITY and an explanatory ee_last_cuda_error() text.
- *   - The first call on a device resolves the array's device address (the calling thread's current device must be the
- *     one the model lives on); make that first call outside any stream capture.
+ *   - The first call on a device resolves the array's device address; make that first call outside any stream
+ *     capture.  As for every call, the calling thread's current device must be the one the model lives on
+ *     (EE_ERR_INVALID_ARG otherwise: another GPU's copy of the array must not be paired with this model's weights).
  *   - No cudaMalloc / cudaFree or allocating library routine is called.
  *   - All calls, from every model and stream, share the one array and it keeps the previous call's contents; the call
  *     clears what has to start at zero.  Two calls whose kernels overlap on the GPU race on it: serialise them
@@ -249,8 +250,8 @@ ee_status_t ee_model_plan(const ee_model_t* model, int stage, int batch, int cap
  * partial sums of the ranges are always added in ascending order, so a sample's result is bit-identical whichever
  * variant the table picks for the batch it rides in.  Both setters drop the stage's captured graphs.
  * ee_model_set_layer_splits may change ee_stage_info_t.workspace_bytes: query again before the next run.
- * ee_model_get_layer_config: tensor_core = -1 (not a tensor-core layer with a table), else the highest variant the
- * layer supports.  Errors: INVALID_ARG, STAGE, CAPACITY (batch range beyond max_batch; partial tiles of more than 256 MB),
+ * ee_model_get_layer_config: tensor_core = -1 (not a tensor-core layer with a table), else a bit mask of the pair
+ * variants the layer supports (bit 0: variant 1, bit 1: variant 2).  Errors: INVALID_ARG, STAGE, CAPACITY (batch range beyond max_batch; partial tiles of more than 256 MB),
  * UNSUPPORTED (the layer cannot run as that variant). */
 ee_status_t ee_model_set_layer_variant(ee_model_t* model, int stage, int layer, int batch_lo, int batch_hi, int variant);
 ee_status_t ee_model_set_layer_splits(ee_model_t* model, int stage, int layer, int splits);
@@ -259,6 +260,13 @@ ee_status_t ee_model_get_layer_config(const ee_model_t* model, int stage, int la
 
 /* Limit, in SM clock cycles, of the bounded device-side waits (default about 2 s).  Errors: INVALID_ARG. */
 ee_status_t ee_model_set_wait_limit(ee_model_t* model, long long cycles);
+
+/* Self-test of the device-side time-out path (no counterpart in the paper; the kernels' waits on barriers are
+ * bounded so that a fault of the pipeline shows up as an error code, never as a hung GPU).  Launches one thread that
+ * waits, with the given limit in SM clock cycles (at most 2e9), on a barrier that nothing signals, and synchronises
+ * the stream.  Returns EE_OK when the wait ran out and the kernel returned normally; afterwards ee_model_check
+ * reports EE_ERR_TIMEOUT once (and clears it).  Errors: INVALID_ARG, CUDA, INTERNAL (the wait did not give up). */
+ee_status_t ee_model_selftest_wait(ee_model_t* model, long long limit_cycles, void* cuda_stream);
 
 /* Runs a batch from stage `first_stage` on until it is empty or the last stage has been launched: ee_stage_run for a
  * stage, the host's wait for its survivor count (the protocol of ee_wait_count on outs[s].n_surv_host, which must be

@@ -22,7 +22,7 @@ STATUS_NAMES = ["EE_OK", "EE_ERR_INVALID_ARG", "EE_ERR_SHAPE", "EE_ERR_CAPACITY"
 EXPORTS = ["ee_model_create", "ee_model_destroy", "ee_model_query", "ee_stage_run", "ee_layer_run", "ee_batch_refill", "ee_exit_head",
            "ee_exit_head_scratch_bytes", "ee_exit_head_static", "ee_gather_survivors", "ee_model_set_graphs", "ee_model_set_timing", "ee_model_get_timing",
            "ee_model_plan", "ee_model_check", "ee_model_set_layer_variant", "ee_model_set_layer_splits", "ee_model_get_layer_config",
-           "ee_model_set_wait_limit", "ee_wait_count", "ee_run_until_exit", "ee_status_string", "ee_last_cuda_error"]
+           "ee_model_set_wait_limit", "ee_model_selftest_wait", "ee_wait_count", "ee_run_until_exit", "ee_status_string", "ee_last_cuda_error"]
 
 
 class EEError(RuntimeError):
@@ -104,6 +104,7 @@ def load_library() -> C.CDLL:
     L.ee_model_set_layer_splits.argtypes = [vp, i, i, i]
     L.ee_model_get_layer_config.argtypes = [vp, i, i, i, C.POINTER(i), C.POINTER(i), C.POINTER(i)]
     L.ee_model_set_wait_limit.argtypes = [vp, C.c_longlong]
+    L.ee_model_selftest_wait.argtypes = [vp, C.c_longlong, vp]
     L.ee_status_string.argtypes = [i]
     L.ee_status_string.restype = C.c_char_p
     L.ee_last_cuda_error.restype = C.c_char_p
@@ -178,7 +179,7 @@ class StageBuffers:
 class EEModel:
     """Handle of one early-exit model on the current CUDA device (wraps ee_model_t)."""
 
-    def __init__(self, spec, device: str = "cuda", stream=None):
+    def __init__(self, spec, device: str = "cuda", stream=None, apply_tables: bool = True):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required: this library has no CPU path")
         self._L = load_library()
@@ -215,6 +216,9 @@ class EEModel:
         self._h = h
         self._keep = []
         self._outs_key, self._outs_arr = None, None
+        self.table = None
+        if apply_tables:
+            self.table = apply_table(self, spec)
 
     def close(self):
         if getattr(self, "_h", None):
@@ -333,8 +337,44 @@ class EEModel:
     def set_wait_limit(self, cycles: int):
         _check(self._L.ee_model_set_wait_limit(self._h, int(cycles)), "ee_model_set_wait_limit")
 
+    def selftest_wait(self, limit_cycles: int, stream=None):
+        _check(self._L.ee_model_selftest_wait(self._h, int(limit_cycles), _stream(stream)), "ee_model_selftest_wait")
+
     def check(self, stream=None):
         _check(self._L.ee_model_check(self._h, _stream(stream)), "ee_model_check")
+
+
+def apply_table(model: EEModel, spec, path: Optional[str] = None):
+    """Loads the measured per-(layer, batch) kernel table written by ``autotune.py`` for this (model name, max_batch),
+    checks that it describes this model's layers, and installs it (ee_model_set_layer_splits / _variant).
+    Returns the table's path, or None when there is none (the library's built-in choices stay in force)."""
+    import json
+
+    if path is None:
+        path = os.path.join(_HERE, "tables", f"{spec.name}_b{spec.max_batch}.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        t = json.load(f)
+    if t.get("max_batch") != spec.max_batch or t.get("input") != [spec.in_h, spec.in_w, spec.in_c]:
+        return None
+    for e in t["layers"]:
+        s, i = e["stage"], e["layer"]
+        if s >= len(spec.stages) or i >= len(spec.stages[s].layers):
+            return None
+        l = spec.stages[s].layers[i]
+        if [l.kh, l.cin, l.cout, l.stride] != e["geom"][:4] or len(e["variants"]) != spec.max_batch:
+            return None
+    for e in t["layers"]:
+        s, i = e["stage"], e["layer"]
+        model.set_layer_splits(s, i, e["splits"])
+        v = e["variants"]
+        lo = 1
+        for b in range(2, spec.max_batch + 2):     # runs of equal entries
+            if b == spec.max_batch + 1 or v[b - 1] != v[lo - 1]:
+                model.set_layer_variant(s, i, lo, b - 1, v[lo - 1])
+                lo = b
+    return path
 
 
 def gather_survivors(feat, bytes_per_sample: int, survivor_idx, n_surv_dev, max_rows: int, feat_out, stream=None):

@@ -1,5 +1,6 @@
 // C ABI of the early-exit CNN stage executor: model creation (weight upload, per-layer kernel
 // plan, workspace layout), ee_stage_run, ee_batch_refill and the stand-alone head / gather calls.
+#include <atomic>
 #include <chrono>
 #include <cstdio>
 #include <cstring>
@@ -71,6 +72,7 @@ inline bool same_call(const StageCallKey& a, const StageCallKey& b) {  // field 
 struct StagePlan {
   std::vector<LayerPlan> layers;
   std::vector<StageGraph> graphs;  // captured stage executions by call signature
+  std::vector<cudaGraphExec_t> retired;   // evicted executables: they may still be in flight, destroyed later
   int in_h, in_w, in_c, out_h, out_w, out_c, out_slot;
   std::vector<size_t> slot_off;  // byte offsets at max_batch
   size_t head_off = 0, ws_bytes = 0, head_bytes = 0;
@@ -379,6 +381,13 @@ ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, c
   return EE_OK;
 }
 
+// The GPU that is current must be the one the model lives on: kernels launched elsewhere would dereference this
+// model's weights from another device.
+bool on_model_device(const ee_model* m) {
+  int dev = -1;
+  return cudaGetDevice(&dev) == cudaSuccess && dev == m->device;
+}
+
 bool valid_out(const ee_stage_out_t* o, bool need_feat) {
   return o && o->exit_mask && o->survivor_idx && o->n_surv_dev && (!need_feat || o->features_out);
 }
@@ -409,6 +418,7 @@ ee_status_t ee_model_destroy(ee_model_t* m) {
   for (auto& sp : m->stages) {
     for (auto e : sp.ev) cudaEventDestroy(e);
     for (auto& g : sp.graphs) cudaGraphExecDestroy(g.exec);
+    for (auto e : sp.retired) cudaGraphExecDestroy(e);
   }
   for (void* p : m->owned) cudaFree(p);
   if (m->ev_fork) cudaEventDestroy(m->ev_fork);
@@ -689,6 +699,11 @@ ee_status_t ee_wait_count(const int32_t* n_surv_host, int32_t sentinel, double t
       *value = v;
       return EE_OK;
     }
+#if defined(__x86_64__) || defined(__i386__)
+    __builtin_ia32_pause();   // be kind to the sibling hardware thread while spinning
+#elif defined(__aarch64__)
+    asm volatile("yield" ::: "memory");
+#endif
     if ((spin & 1023u) == 1023u && std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count() > timeout_s)
       return EE_ERR_TIMEOUT;
   }
@@ -740,7 +755,7 @@ ee_status_t ee_model_query(const ee_model_t* m, int stage, ee_stage_info_t* out)
 
 ee_status_t ee_stage_run(ee_model_t* m, int stage, const ee_stage_in_t* in, void* workspace, size_t workspace_bytes,
                          const ee_stage_out_t* out, void* cuda_stream) {
-  if (!m || !in || !valid_out(out, true) || in->batch < 0) return EE_ERR_INVALID_ARG;
+  if (!m || !in || !valid_out(out, true) || in->batch < 0 || !on_model_device(m)) return EE_ERR_INVALID_ARG;
   if (stage < 0 || stage >= (int)m->stages.size()) return EE_ERR_STAGE;
   if (in->logit_shift && !in->shift_class) return EE_ERR_INVALID_ARG;
   StagePlan& sp = m->stages[stage];
@@ -777,16 +792,26 @@ ee_status_t ee_stage_run(ee_model_t* m, int stage, const ee_stage_in_t* in, void
         cudaGraphExec_t exec = nullptr;
         if (es == EE_OK && ce == cudaSuccess && graph && cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess) {
           cudaGraphDestroy(graph);
-          if (sp.graphs.size() >= 96) {  // bounded cache: drop the oldest
-            cudaGraphExecDestroy(sp.graphs.front().exec);
+          // Bounded cache, sized for a server that keeps two buffer sets and sees every batch size (2 * B_max
+          // signatures per stage).  An evicted executable may still be running: it is parked and destroyed once the
+          // stream has passed it.
+          if (sp.graphs.size() >= (size_t)std::max(96, 2 * m->max_batch + 8)) {
+            sp.retired.push_back(sp.graphs.front().exec);
             sp.graphs.erase(sp.graphs.begin());
+            if (sp.retired.size() >= 32) {
+              cudaStreamSynchronize(st);
+              for (auto e : sp.retired) cudaGraphExecDestroy(e);
+              sp.retired.clear();
+            }
           }
           sp.graphs.push_back({key, exec});
           EE_CUDA(cudaGraphLaunch(exec, st));
           return EE_OK;
         }
         if (graph) cudaGraphDestroy(graph);
-        cudaGetLastError();   // capture is not available here: fall back to plain launches from now on
+        // capture is not available here: plain launches from now on; ee_last_cuda_error() says why
+        g_cuda_err = std::string("stage replay switched off, capture failed: ") + cudaGetErrorString(ce != cudaSuccess ? ce : cudaGetLastError());
+        cudaGetLastError();
         m->graphs = false;
         if (es != EE_OK) return es;
       }
@@ -797,7 +822,7 @@ ee_status_t ee_stage_run(ee_model_t* m, int stage, const ee_stage_in_t* in, void
 
 ee_status_t ee_layer_run(ee_model_t* m, int stage, int layer, const void* input, const void* residual, int batch, void* output,
                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  if (!m || batch < 0) return EE_ERR_INVALID_ARG;
+  if (!m || batch < 0 || !on_model_device(m)) return EE_ERR_INVALID_ARG;
   if (stage < 0 || stage >= (int)m->stages.size()) return EE_ERR_STAGE;
   StagePlan& sp = m->stages[stage];
   if (layer < 0 || layer >= (int)sp.layers.size()) return EE_ERR_STAGE;
@@ -821,7 +846,7 @@ ee_status_t ee_layer_run(ee_model_t* m, int stage, int layer, const void* input,
 
 ee_status_t ee_batch_refill(ee_model_t* m, int boundary, void* batch_feat, int32_t* batch_ids, int n_surv, const void* arr_feat,
                             const int32_t* arr_ids, int n_arr, int* n_accepted, int* n_merged, void* cuda_stream) {
-  if (!m || !n_accepted || !n_merged || n_surv < 0 || n_arr < 0) return EE_ERR_INVALID_ARG;
+  if (!m || !n_accepted || !n_merged || n_surv < 0 || n_arr < 0 || !on_model_device(m)) return EE_ERR_INVALID_ARG;
   if (boundary < 0 || boundary > (int)m->stages.size() - 1) return EE_ERR_STAGE;
   if (n_surv > m->max_batch) return EE_ERR_CAPACITY;
   if (n_arr > 0 && (!batch_feat || !arr_feat)) return EE_ERR_INVALID_ARG;
@@ -856,7 +881,7 @@ size_t ee_exit_head_scratch_bytes(const ee_model_t* m, int stage) {
 ee_status_t ee_exit_head(ee_model_t* m, int stage, const void* x, int batch, int hw, const float* logit_shift,
                          const int32_t* shift_class, void* scratch, size_t scratch_bytes, const ee_stage_out_t* out,
                          void* cuda_stream) {
-  if (!m || !valid_out(out, false) || batch < 0 || hw < 1) return EE_ERR_INVALID_ARG;
+  if (!m || !valid_out(out, false) || batch < 0 || hw < 1 || !on_model_device(m)) return EE_ERR_INVALID_ARG;
   if (stage < 0 || stage >= (int)m->stages.size()) return EE_ERR_STAGE;
   if (logit_shift && !shift_class) return EE_ERR_INVALID_ARG;
   StagePlan& sp = m->stages[stage];
@@ -880,7 +905,7 @@ static __device__ __align__(256) unsigned char g_static_head_scratch[EE_STATIC_H
 
 namespace {
 constexpr int kMaxDevices = 64;
-void* g_static_head_ptr[kMaxDevices];   // device address of the array, resolved once per device
+std::atomic<void*> g_static_head_ptr[kMaxDevices];   // device address of the array, resolved once per device
 }  // namespace
 
 ee_status_t ee_exit_head_static(ee_model_t* m, int stage, const void* x, int batch, int hw, const float* logit_shift,
@@ -896,14 +921,14 @@ ee_status_t ee_exit_head_static(ee_model_t* m, int stage, const void* x, int bat
                  std::to_string((size_t)EE_STATIC_HEAD_SCRATCH_BYTES);
     return EE_ERR_CAPACITY;
   }
-  int dev = -1;
-  EE_CUDA(cudaGetDevice(&dev));
+  if (!on_model_device(m)) return EE_ERR_INVALID_ARG;   // the array of the model's own GPU is the one to use
+  const int dev = m->device;
   if (dev < 0 || dev >= kMaxDevices) return EE_ERR_UNSUPPORTED;
-  if (!g_static_head_ptr[dev]) {  // first call on this device (the device is current): ask the runtime where the array lives
-    void* ptr = nullptr;
-    EE_CUDA(cudaGetSymbolAddress(&ptr, g_static_head_scratch));
-    if (!ptr) return EE_ERR_INTERNAL;
-    g_static_head_ptr[dev] = ptr;
+  void* resolved = g_static_head_ptr[dev].load(std::memory_order_acquire);
+  if (!resolved) {  // first call on this device (the device is current): ask the runtime where the array lives
+    EE_CUDA(cudaGetSymbolAddress(&resolved, g_static_head_scratch));
+    if (!resolved) return EE_ERR_INTERNAL;
+    g_static_head_ptr[dev].store(resolved, std::memory_order_release);   // every thread resolves the same address
   }
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (batch == 0) {
@@ -911,7 +936,7 @@ ee_status_t ee_exit_head_static(ee_model_t* m, int stage, const void* x, int bat
     return EE_OK;
   }
   if (!x) return EE_ERR_INVALID_ARG;
-  char* scratch = (char*)g_static_head_ptr[dev];
+  char* scratch = (char*)resolved;
   // the pooling kernel zeroes the counters the FC kernel needs; everything else in the array is overwritten before it is read
   return m->dtype == EE_BF16
              ? launch_head<bf16>(m, sp, x, batch, hw, logit_shift, shift_class, scratch, nullptr, out, st, false)
@@ -1019,7 +1044,7 @@ ee_status_t ee_model_get_layer_config(const ee_model_t* m, int stage, int layer,
   const bool tc = L.kind == KK_TC && !L.tc.gather && !L.tc.halo;
   if (variant) *variant = L.variant.empty() ? (int)TCV_AUTO : (int)L.variant[batch];
   if (splits) *splits = L.kind == KK_TC ? L.tc.splits : 1;
-  if (tensor_core) *tensor_core = tc ? (pair_supported(L.tc, TCV_PAIR256) ? 2 : pair_supported(L.tc, TCV_PAIR128) ? 1 : 0) : -1;
+  if (tensor_core) *tensor_core = tc ? ((pair_supported(L.tc, TCV_PAIR256) ? 1 : 0) | (pair_supported(L.tc, TCV_PAIR128) ? 2 : 0)) : -1;
   return EE_OK;
 }
 
@@ -1027,6 +1052,19 @@ ee_status_t ee_model_set_wait_limit(ee_model_t* m, long long cycles) {
   if (!m || cycles < 1) return EE_ERR_INVALID_ARG;
   m->wait_cycles = cycles;
   return EE_OK;
+}
+
+ee_status_t ee_model_selftest_wait(ee_model_t* m, long long limit_cycles, void* cuda_stream) {
+  if (!m || limit_cycles < 1 || limit_cycles > 2000000000LL) return EE_ERR_INVALID_ARG;   // at most about a second
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int* end_word = m->err_flag + 1;   // second word of the model's 256-byte status block
+  EE_CUDA(cudaMemsetAsync(end_word, 0, sizeof(int), st));
+  wait_selftest_kernel<<<1, 32, 0, st>>>(m->err_flag, limit_cycles, end_word);
+  EE_CUDA(cudaGetLastError());
+  int reached = 0;
+  EE_CUDA(cudaMemcpyAsync(&reached, end_word, sizeof(int), cudaMemcpyDeviceToHost, st));
+  EE_CUDA(cudaStreamSynchronize(st));
+  return reached == 1 ? EE_OK : EE_ERR_INTERNAL;   // the kernel must have returned through the give-up path
 }
 
 ee_status_t ee_model_check(ee_model_t* m, void* cuda_stream) {

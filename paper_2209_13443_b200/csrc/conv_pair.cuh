@@ -435,6 +435,18 @@ conv_igemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __
   }
 }
 
+// Self-test of the bounded wait: one thread waits on a barrier nobody will ever signal.  The wait must run out after
+// `limit` cycles, record EE_ERR_TIMEOUT in the error word and let the kernel return normally.
+__global__ void wait_selftest_kernel(int* err_flag, long long limit, int* reached_end) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const bool ok = mbar_wait_for(smem_u32(&bar), 0, err_flag, limit);
+    *reached_end = ok ? 2 : 1;   // 1: the wait gave up and the thread went on
+  }
+}
+
 // ----------------------------------------------------------------------------- host side
 
 // Kernel variants a tensor-core layer can run as (the per-(layer, batch) table of LayerPlan holds one of these).

@@ -298,6 +298,18 @@ def mobilenetv2_ee(seed: int = 2, max_batch: int = 32, alphas=None, threshold: f
                  {"seed": seed, "alphas": list(alphas), "threshold": threshold})
 
 
+def benchmark_model(workload: str, max_batch: int, flat_heads: bool = False):
+    """The benchmark configurations by name: (model, input seed).  ``flat_heads`` scales the FC weights down so that
+    unshifted confidences sit near 1/n_classes and only forced logit shifts (exit-rate sweep) decide who leaves."""
+    if workload == "resnet50":
+        return resnet50_ee(seed=1, max_batch=max_batch, alphas=[0.01] * 4 if flat_heads else None), 1
+    if workload == "mobilenetv2":
+        return mobilenetv2_ee(seed=2, max_batch=max_batch, alphas=[0.01] * 4 if flat_heads else None), 2
+    if workload == "tiny":
+        return tiny_ee_cnn(seed=0, max_batch=max_batch), 0
+    raise ValueError(f"unknown workload {workload}")
+
+
 # ----------------------------------------------------------------------------- inputs
 
 def make_input(model: Model, batch: int, seed: int, first_id: int = 0, rho: float = 0.5, grid: int = 4) -> np.ndarray:

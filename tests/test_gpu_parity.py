@@ -184,7 +184,7 @@ def test_pair_kernel_layer(geom):
     def configure(m):
         m.set_layer_splits(0, layer, splits)
         m.set_layer_variant(0, layer, 1, max_batch, variant)
-        assert m.layer_config(0, layer, 3) == {"variant": variant, "splits": splits, "tensor_core": 2 if cout > 128 else 1}
+        assert m.layer_config(0, layer, 3) == {"variant": variant, "splits": splits, "tensor_core": 3 if cout > 128 else 2}
 
     m = eb.EEModel(spec)
     configure(m)
@@ -408,6 +408,25 @@ def test_error_codes_and_empty_batch():
     with pytest.raises(eb.EEError) as e:
         eb.EEModel(bad)
     assert e.value.status == 2
+
+
+def test_device_side_timeout_is_reported_and_the_model_keeps_working():
+    """The bounded waits of the kernels: a wait that nothing will ever satisfy runs out after its limit, the kernel returns,
+    ee_model_check reports EE_ERR_TIMEOUT exactly once, and a normal stage then runs and matches the oracle."""
+    spec = wl.tiny_ee_cnn(seed=0)
+    run = util.GpuRunner(spec)
+    m = run.m
+    m.check()
+    m.selftest_wait(2_000_000)                                         # about 1 ms of SM clocks
+    with pytest.raises(eb.EEError) as e:
+        m.check()
+    assert e.value.status == 7                                         # EE_ERR_TIMEOUT
+    m.check()                                                          # the flag was cleared by the failing check
+    with pytest.raises(eb.EEError) as e:
+        m.selftest_wait(0)
+    assert e.value.status == 1
+    x = wl.make_input(spec, 8, seed=0)
+    util.check_stage(spec, run.stage(0, x), util.oracle_stage(spec, 0, x), "after the time-out self-test")
 
 
 # ----------------------------------------------------------------------------- full benchmark sizes
