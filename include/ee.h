@@ -222,6 +222,13 @@ ee_status_t ee_gather_survivors(const void* feat, size_t bytes_per_sample, const
  * Errors: INVALID_ARG. */
 ee_status_t ee_model_set_graphs(ee_model_t* model, int enabled);
 
+/* Branch execution.  On by default for batches of up to 32 samples: a layer whose output is only a residual operand of a later layer (the projection
+ * shortcut of a residual block) runs on a stream of the model's own, beside the layers between its input and its
+ * consumer, forked from and joined to the caller's stream by events (also inside captured stages).  Results are
+ * identical either way: the layers and their kernels are the same, only their order in time changes.
+ * Errors: INVALID_ARG. */
+ee_status_t ee_model_set_branches(ee_model_t* model, int enabled);
+
 /* Per-layer device timing.  When enabled, ee_stage_run brackets every kernel with CUDA events on the
  * stream it launches on.  ee_model_get_timing synchronises those events and writes, for the last run
  * of `stage`, up to `cap` entries: the layers in order, then the head and the gather kernels.

@@ -677,6 +677,35 @@ def test_stage_replay_as_graph_is_bit_identical():
     m.check()
 
 
+def test_branch_execution_of_shortcut_layers_is_bit_identical():
+    """The projection shortcut of a block runs on the model's branch stream beside the block's main chain (plain
+    launches and captured stages); switching that off must not change a bit of the stage's results."""
+    spec = wl.resnet50_ee(seed=1, in_hw=96, n_classes=100, max_batch=7)
+    run = util.GpuRunner(spec)
+    m, ws = run.m, run.ws
+    B = 7
+    x = wl.make_input(spec, B, seed=4)
+    side = torch.cuda.Stream()
+    for s in range(m.n_stages):
+        o = util.oracle_stage(spec, s, x)
+        xd = eb.to_device("bf16", x)
+        snaps = []
+        for branches, stream in ((False, None), (True, None), (True, side), (True, side)):
+            m.set_branches(branches)
+            run.bufs[s].logits.fill_(0)
+            run.bufs[s].features_out.fill_(0)
+            with torch.cuda.stream(stream or torch.cuda.current_stream()):
+                m.stage_run(s, xd, B, run.bufs[s], ws)
+            torch.cuda.synchronize()
+            n = int(run.bufs[s].n_surv_host[0])
+            snaps.append((n, run.bufs[s].logits[:B].clone(), run.bufs[s].features_out[:n].clone()))
+        for n, z, f in snaps[1:]:
+            assert n == snaps[0][0] and torch.equal(z, snaps[0][1]) and torch.equal(f, snaps[0][2]), f"stage {s}"
+        x = o["stage_out"]
+    run.check_guards()
+    m.check()
+
+
 def test_count_reaches_the_host_without_a_stream_sync():
     """B_exit is copied to the pinned word beside the gather (plain launches and graph replay): ee_wait_count returns it
     without synchronising the stream, and it equals the count of the synchronised run."""
