@@ -321,6 +321,33 @@ def run_ours(args):
         step(True, k)
     e2e_ms, _, h2d, d2h, _ = timed(True, K)
 
+    # per-stage pass, un-instrumented: CUDA events on the launching stream around every ee_stage_run (graph replay and
+    # programmatic launch overlap stay on inside a stage); the host learns each count from its pinned word as in a step
+    stage_ms = [0.0] * nst
+    stage_batch = [0] * nst
+    stage_flops = [0.0] * nst
+    stage_conv_launches = [0] * nst
+    for _ in range(K):
+        flush.zero_()
+        model.batch_refill(0, batch0, ids0, 0, x_dev, ids_dev, B)
+        feat, ids, n = batch0, ids0, B
+        for s in range(nst):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            bufs[s].arm_count()
+            a.record()
+            run_stage(s, feat, n, ids)
+            b.record()
+            ns = bufs[s].wait_count()
+            b.synchronize()
+            stage_ms[s] += a.elapsed_time(b) / K
+            stage_batch[s] = n
+            convs = [pl for pl in model.plan(s, n) if pl["kernel"].startswith("conv_igemm_tcgen05")]
+            stage_flops[s] = sum(pl["flops"] for pl in convs)
+            stage_conv_launches[s] = len(convs)
+            feat, ids, n = bufs[s].features_out, bufs[s].ids_out, ns
+            if n == 0:
+                break
+
     # instrumented pass: per-kernel device time by CUDA events on the launching stream
     model.set_timing(True)
     fam = {}
@@ -384,10 +411,25 @@ def run_ours(args):
         roof = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "peak_source": f"copy bandwidth, {peaks['source']}"}
     roof["frac"] = roof["achieved"] / roof["peak"]
+    if roof["bound"] == "tensor":
+        # The instrumented pass brackets every kernel with events, which switches off stage replay and the overlap of
+        # consecutive kernels, so its per-kernel times are upper bounds.  The headline fraction comes from the
+        # un-instrumented per-stage pass: FLOPs of the stage's tensor-core conv launches over the device time of the
+        # whole ee_stage_run (head, compaction and gather included: a lower bound on the conv kernels' own rate).
+        roof["achieved_instrumented"], roof["frac_instrumented"] = roof["achieved"], roof["frac"]
+        tot_ms = sum(stage_ms)
+        roof["achieved"] = sum(stage_flops) / (tot_ms * 1e-3) / 1e12 if tot_ms > 0 else 0.0
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof["timing"] = "un-instrumented: conv FLOPs / device time of the stages (CUDA events around ee_stage_run, graph replay on)"
+        roof["per_stage"] = [{"stage": s, "batch": stage_batch[s], "ms": stage_ms[s], "conv_launches": stage_conv_launches[s],
+                              "conv_tflops": stage_flops[s] / (stage_ms[s] * 1e-3) / 1e12 if stage_ms[s] > 0 else 0.0,
+                              "frac": stage_flops[s] / (stage_ms[s] * 1e-3) / 1e12 / roof["peak"] if stage_ms[s] > 0 else 0.0}
+                             for s in range(nst) if stage_batch[s] > 0]
     roof["traffic"] = (NCU_CONV_TRAFFIC_PER_LAUNCH.get((args.workload, B)) if roof["bound"] == "tensor" and args.exit_rate is None else None)
     roof["traffic_warm_l2"] = (NCU_CONV_TRAFFIC_WARM_L2.get((args.workload, B)) if roof["traffic"] is not None else None)
-    roof["avg_launch_ms"] = fam[dom]["ms"] / max(fam[dom]["launches"], 1)
+    roof["avg_launch_ms_instrumented"] = fam[dom]["ms"] / max(fam[dom]["launches"], 1)
     roof["per_launch"] = (fam[dom]["flops"] if roof["bound"] == "tensor" else fam[dom]["bytes"]) / max(fam[dom]["launches"], 1)
+    roof["avg_launch_ms"] = (sum(stage_ms) / max(sum(stage_conv_launches), 1)) if roof["bound"] == "tensor" else roof["avg_launch_ms_instrumented"]
     roof["hbm_kernels"] = {k: {"gbs": kernels[k]["gbs"], "frac": kernels[k]["gbs"] / peaks["hbm_gbs"]}
                            for k in ("head_gap", "gather_survivors", "maxpool", "dwconv") if k in kernels}
 
@@ -438,8 +480,9 @@ def run_ours(args):
 
 
 def run_trace(args):
-    """Streaming fluid-batch trace: seeded Poisson arrivals served by the exit-aware preemptive loop (Algorithm 1,
-    T_SLO = infinity) on the wall clock; request r carries image r mod 256 of a fixed pool."""
+    """Streaming fluid-batch trace: seeded Poisson arrivals served by the exit-aware preemptive loop (Algorithm 1; T_SLO
+    infinite unless --slo-ms sets the SLO of the preemption criterion, Eq. 3-4) on the wall clock; request r carries
+    image r mod 256 of a fixed pool."""
     import torch
 
     from paper_2209_13443_b200 import binding as eb

@@ -15,7 +15,8 @@ Driver functions and the passages they follow:
                        batched or refilled schedule has to reproduce per sample id, because
                        samples finish out of order and are re-associated by id (Section III-B,
                        Overhead)
-  serve_trace          Algorithm 1 with T_SLO = infinity on a virtual clock
+  serve_trace          Algorithm 1 on a virtual clock, with the SLO-aware preemption criterion (Eq. 3-4;
+                       T_SLO = infinity by default)
 """
 from __future__ import annotations
 
