@@ -95,6 +95,7 @@ def measure(spec, batches, verbose=True):
                                 continue       # cluster split-K of the one-CTA kernel: up to four ranges
                             m.set_layer_variant(s, i, 1, spec.max_batch, v)
                             us = time_layer(m, s, i, x, res, out, B, ws)
+                            m.check()          # a device-side fault stops the sweep here, not minutes later
                             rows.append({"stage": s, "layer": i, "splits": sp, "batch": B, "variant": v, "us": us,
                                          "default_splits": default_splits,
                                          "geom": [l.kh, l.cin, l.cout, l.stride, oshape[0], oshape[1]]})
