@@ -507,7 +507,12 @@ def run_trace(args):
     if args.slo_ms is not None:       # the scheduler's N_exits x B_max latency table, measured on this device
         lut = srv.measure_latency_table()
         latency = lambda s, b: float(lut[s, b - 1])   # noqa: E731
-    out = srv.serve(arrivals, image_of, pool, slo=slo, latency=latency)
+    if args.policy == "serial":
+        out = srv.serve_serial(arrivals, image_of, pool)
+    elif args.policy == "adaptb":
+        out = srv.serve_adaptive_batching(arrivals, image_of, pool, max_batch=args.batch, timeout=args.timeout_ms * 1e-3)
+    else:
+        out = srv.serve(arrivals, image_of, pool, slo=slo, latency=latency)
     lat = (out["finish"] - arrivals) * 1e3
     span = float(out["finish"].max() - arrivals[0])
     sizes = [len(ids) for _, ids in out["launches"]]
@@ -516,7 +521,8 @@ def run_trace(args):
         "metric": METRIC, "value": n / span, "unit": UNIT, "n_gpus": 1, "steps": n, "warmup": 300, "ms_per_step": span / n * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": spec.dtype, "data": "synthetic",
         "config": {"workload": f"{spec.name} {spec.dtype} streaming trace, {n} requests, Poisson {args.trace_rate:g} req/s, B_max={args.batch}, "
-                               f"Algorithm 1 with T_SLO={'inf' if args.slo_ms is None else str(args.slo_ms) + ' ms'}, wall clock"},
+                               + {"fluid": f"Algorithm 1 with T_SLO={'inf' if args.slo_ms is None else str(args.slo_ms) + ' ms'}", "serial": "SERIAL policy",
+                                  "adaptb": f"adaptive batching <B_max, T_timeout={args.timeout_ms} ms>"}[args.policy] + ", wall clock"},
         "latency_ms": {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99)), "mean": float(lat.mean())},
         "slo_ms": args.slo_ms, "slo_violation_rate": None if args.slo_ms is None else float(np.mean(lat > args.slo_ms)),
         "preemptions": out["preemptions"], "declined": out["declined"],
@@ -540,6 +546,9 @@ def main():
     ap.add_argument("--trace-requests", type=int, default=2000)
     ap.add_argument("--slo-ms", type=float, default=None,
                     help="streaming trace: latency SLO in ms for the SLO-aware preemption criterion (Eq. 3-4); default: T_SLO = inf")
+    ap.add_argument("--policy", default="fluid", choices=["fluid", "serial", "adaptb"],
+                    help="streaming trace: the exit-aware preemptive scheduler (default), one request at a time, or adaptive batching <B_max, T_timeout>")
+    ap.add_argument("--timeout-ms", type=float, default=1.0, help="streaming trace, adaptive batching: T_timeout in ms")
     ap.add_argument("--cpu-samples", type=int, default=64)
     ap.add_argument("--report-layers", action="store_true", help="add a per-layer table (time, TFLOP/s, GB/s, roofline bound) to the JSON line")
     args = ap.parse_args()

@@ -61,6 +61,7 @@ def measure(spec, batches, verbose=True):
     from . import workloads as wl
 
     m = eb.EEModel(spec, apply_tables=False)
+    m.set_wait_limit(200_000_000)       # a wait that runs out should cost 0.1 s, not seconds, per launch of a sweep
     shapes = layer_shapes(spec)
     rows = []
     ws = m.workspace()

@@ -640,6 +640,45 @@ def test_streaming_trace_matches_oracle_schedule():
     assert launches_slo != launches
 
 
+def test_comparison_policies_serve_every_request_like_its_serial_run():
+    """SERIAL and adaptive batching <B_max, T_timeout> on the same calls: whatever the batches, every request leaves
+    at the exit and with the class of its own serial run through the oracle; SERIAL launches single samples in
+    arrival order; adaptive batching with a long time-out issues full batches and never refills one."""
+    from paper_2209_13443_b200.serving import FluidServer
+
+    spec = wl.tiny_ee_cnn(seed=0)
+    pool_np = wl.make_input(spec, 40, seed=9)
+    serial = [eo.run_sample_serial(spec, pool_np[i]) for i in range(len(pool_np))]
+    keep = [i for i, sref in enumerate(serial) if all(abs(c - 0.6) > 10 * util.BAND for c in sref[2][:2])][:24]
+    pool_np, serial = pool_np[keep], [serial[i] for i in keep]
+    n = 120
+    arrivals = wl.poisson_arrivals(3, n, 2000.0)
+    image_of = [r % len(keep) for r in range(n)]
+    stage_time = lambda s, b: 2e-4 * (s + 1) + 3e-5 * b      # noqa: E731
+    srv = FluidServer(spec)
+    pool = eb.to_device("f32", pool_np)
+    want_exit = np.array([serial[image_of[r]][0] for r in range(n)])
+    want_pred = [serial[image_of[r]][1] for r in range(n)]
+    got = srv.serve_serial(arrivals, image_of, pool, stage_time)
+    assert np.array_equal(got["exit_stage"], want_exit) and got["pred"].tolist() == want_pred
+    assert all(len(ids) == 1 for _, ids in got["launches"])
+    assert [ids[0] for s, ids in got["launches"] if s == 0] == list(range(n))          # arrival order
+    assert np.all(np.diff(got["finish"]) > 0) and np.all(got["finish"] > arrivals)
+    # service time of a request alone: the subnets up to its exit at batch 1
+    alone = np.array([sum(stage_time(s, 1) for s in range(e + 1)) for e in want_exit])
+    assert np.all(got["finish"] - arrivals >= alone - 1e-12)
+    got = srv.serve_adaptive_batching(arrivals, image_of, pool, max_batch=4, timeout=1.0, stage_time=stage_time)
+    assert np.array_equal(got["exit_stage"], want_exit) and got["pred"].tolist() == want_pred
+    first = [ids for s, ids in got["launches"] if s == 0]
+    assert all(len(ids) == 4 for ids in first[:-1]) and sum(len(ids) for ids in first) == n
+    for (s0, a), (s1, b) in zip(got["launches"], got["launches"][1:]):                  # a batch only ever shrinks
+        if s1 == s0 + 1:
+            assert set(b) <= set(a)
+    got0 = srv.serve_adaptive_batching(arrivals, image_of, pool, max_batch=8, timeout=0.0, stage_time=stage_time)
+    assert np.array_equal(got0["exit_stage"], want_exit)
+    assert np.mean(got0["finish"] - arrivals) < np.mean(got["finish"] - arrivals)       # waiting a second for full batches costs latency
+
+
 def test_stage_replay_as_graph_is_bit_identical():
     """On a side stream a stage is captured into a CUDA graph at its first call and replayed afterwards; the replay,
     and a replay on new input values in the same buffers, must equal plain launches bit for bit."""
