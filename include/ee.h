@@ -229,6 +229,15 @@ ee_status_t ee_model_set_graphs(ee_model_t* model, int enabled);
  * Errors: INVALID_ARG. */
 ee_status_t ee_model_set_branches(ee_model_t* model, int enabled);
 
+/* Multi-layer launches.  Off by default: a run of consecutive layers that the CTA-pair kernel covers (dense convolutions
+ * with more than 64 filters) can execute as ONE persistent kernel with a grid-wide barrier between layers in place of a
+ * kernel boundary; the layers' arithmetic, K ranges and results are those of the per-layer kernels, bit for bit.
+ * Measured on B200 the barrier (output stores complete, release, acquire on every SM, first activation tiles) costs more
+ * than a kernel boundary under programmatic dependent launch at every batch size, hence the default.
+ * `max_batch` > 0 restricts it to batches of at most that size (0 = no limit).  Per-layer timing switches it off.
+ * Errors: INVALID_ARG. */
+ee_status_t ee_model_set_stage_kernel(ee_model_t* model, int enabled, int max_batch);
+
 /* Per-layer device timing.  When enabled, ee_stage_run brackets every kernel with CUDA events on the
  * stream it launches on.  ee_model_get_timing synchronises those events and writes, for the last run
  * of `stage`, up to `cap` entries: the layers in order, then the head and the gather kernels.

@@ -79,6 +79,13 @@ inline bool same_call(const StageCallKey& a, const StageCallKey& b) {  // field 
 struct StagePlan {
   std::vector<LayerPlan> layers;
   std::vector<int> order;          // execution order of the layers (side layers hoisted to where their input is ready)
+  // Runs of consecutive layers (positions in `order`) that the CTA-pair kernel can execute in ONE launch, with a grid
+  // barrier instead of a kernel boundary between them (see conv_pair.cuh).
+  struct Segment {
+    int first, n, bn;
+  };
+  std::vector<Segment> segments;
+  std::vector<int> seg_at;         // position -> index into `segments` if a segment starts there, else -1
   std::vector<StageGraph> graphs;  // captured stage executions by call signature
   std::vector<cudaGraphExec_t> retired;   // evicted executables: they may still be in flight, destroyed later
   int in_h, in_w, in_c, out_h, out_w, out_c, out_slot;
@@ -142,6 +149,9 @@ struct ee_model {
   std::vector<void*> owned;  // device allocations
   int* err_flag = nullptr;   // device word set by kernels whose bounded waits ran out
   unsigned* pair_counters = nullptr;   // arrival counters of the pair kernel's split-K reduction; zero between launches
+  unsigned* grid_bar = nullptr;        // arrival counters of the barriers between the layers of a multi-layer launch
+  bool stage_kernel = false;           // run eligible layer runs as one launch (measured slower than per-layer launches: off)
+  int stage_kernel_max_batch = 1 << 30;
   size_t pair_counter_words = 0;
   long long wait_cycles = kTcWaitCycles;   // limit of the bounded device-side waits of the pair kernel and the self-test
   int device = -1;           // the GPU the model lives on
@@ -348,6 +358,34 @@ ee_status_t append_launch_t(const void* src, void* dst, size_t bytes, const int3
   return EE_OK;
 }
 
+bool stage_kernel_active(const ee_model* m, const StagePlan& sp, int B) {
+  return m->dtype == EE_BF16 && m->stage_kernel && !m->timing && !sp.segments.empty() && B <= m->stage_kernel_max_batch;
+}
+
+// One launch for a run of layers (positions seg.first .. seg.first + seg.n - 1 of the execution order).
+ee_status_t launch_segment(ee_model* m, StagePlan& sp, const StagePlan::Segment& seg, const ee_stage_in_t* in, char* ws, int B,
+                           cudaStream_t st) {
+  static thread_local PairStageArgs args;
+  args.n_layers = seg.n;
+  for (int j = 0; j < seg.n; ++j) {
+    const int i = sp.order[seg.first + j];
+    const LayerPlan& L = sp.layers[i];
+    const void* src = L.src_slot < 0 ? in->features : ws + sp.slot_off[L.src_slot];
+    const void* res = L.res_slot == -2 ? nullptr : (L.res_slot == -1 ? in->features : ws + sp.slot_off[L.res_slot]);
+    void* dst = ws + sp.slot_off[L.out_slot];
+    // the residual operand is "late" when the layer right before this one in the same launch writes it
+    bool res_late = false;
+    if (res && j > 0 && L.d.residual_from >= 0) res_late = sp.order[seg.first + j - 1] == L.d.residual_from;
+    ee_status_t s = pair_fill_layer(m->tc, L.tc, seg.bn, src, res, dst, B, L.scale_dev, L.bias_dev, (float*)(ws + sp.split_off), sp.split_bytes,
+                                    m->pair_counters, res_late, &args, j);
+    if (s != EE_OK) return s;
+  }
+  ee_status_t s = pair_launch_args(m->tc, args, seg.bn, m->err_flag, m->grid_bar, m->wait_cycles, st);
+  if (s != EE_OK) return s;
+  EE_CUDA(cudaGetLastError());
+  return EE_OK;
+}
+
 // Everything one stage launches, in stream order (also the body of a captured graph).
 ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, char* ws, const ee_stage_out_t* out, cudaStream_t st) {
   const int B = in->batch;
@@ -357,8 +395,15 @@ ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, c
   // the layers run in execution order with the shortcut layers on the branch stream.
   // Measured on B200 (ResNet-50-shaped model): the overlap gains 8 us per pass at batch 1-4 and costs 6 us at batch 64,
   // where every kernel fills the machine by itself and the two cross-stream edges per shortcut are pure overhead.
-  const bool par = m->branches && !m->timing && B <= kBranchMaxBatch;
+  const bool mega = stage_kernel_active(m, sp, B);
+  const bool par = m->branches && !m->timing && B <= kBranchMaxBatch && !mega;
   for (size_t k = 0; k < sp.layers.size(); ++k) {
+    if (mega && sp.seg_at[k] >= 0) {
+      ee_status_t s = launch_segment(m, sp, sp.segments[sp.seg_at[k]], in, ws, B, st);
+      if (s != EE_OK) return s;
+      k += sp.segments[sp.seg_at[k]].n - 1;
+      continue;
+    }
     const size_t i = m->timing ? k : (size_t)sp.order[k];
     const LayerPlan& L = sp.layers[i];
     const void* src = L.src_slot < 0 ? in->features : ws + sp.slot_off[L.src_slot];
@@ -729,6 +774,34 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
         L.kind = KK_SIMT;
       }
     }
+    // Layer runs for the multi-layer launch: consecutive positions of the execution order whose layers the CTA-pair kernel
+    // covers with one tile width (256 columns if every layer has more than 128 filters, else 128).
+    {
+      const int nl = sd.n_layers;
+      sp.seg_at.assign(nl, -1);
+      auto ok_for = [&](int i, int variant) {
+        const LayerPlan& L = sp.layers[i];
+        return L.kind == KK_TC && L.tc.cin == L.d.cin && pair_supported(L.tc, variant);
+      };
+      int k = 0;
+      while (k < nl) {
+        if (!ok_for(sp.order[k], TCV_PAIR128)) {
+          ++k;
+          continue;
+        }
+        int e = k;
+        bool all256 = true;
+        while (e < nl && e - k < kPairMaxLayers && ok_for(sp.order[e], TCV_PAIR128)) {
+          all256 = all256 && ok_for(sp.order[e], TCV_PAIR256);
+          ++e;
+        }
+        if (e - k >= 2) {
+          sp.seg_at[k] = (int)sp.segments.size();
+          sp.segments.push_back({k, e - k, all256 ? 256 : 128});
+        }
+        k = e;
+      }
+    }
     // Walk directions.  Feature maps of a large batch exceed the L2, so a kernel that walks its input from the first
     // row finds the rows its producer wrote first already evicted, and evicts the newest ones before it reaches them.
     // Every kernel therefore walks opposite to the kernel that last touched its largest operand: it starts on the rows
@@ -756,6 +829,13 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
     if ((rc = upload_bytes(m, sd.fc_weight, (size_t)sd.n_classes * sp.out_c * es, ondev, st, &sp.fc_w)) != EE_OK) return fail(rc);
     if ((rc = upload<float>(m, sd.fc_bias, sd.n_classes, ondev, st, &sp.fc_b)) != EE_OK) return fail(rc);
     h = sp.out_h, w = sp.out_w, c = sp.out_c;
+  }
+  {
+    void* p = nullptr;
+    if (cudaMalloc(&p, 256) != cudaSuccess) return fail(EE_ERR_CUDA);
+    m->owned.push_back(p);
+    m->grid_bar = (unsigned*)p;
+    if (cudaMemsetAsync(p, 0, 256, st) != cudaSuccess) return fail(EE_ERR_CUDA);
   }
   if (m->pair_counter_words) {
     void* p = nullptr;
@@ -1045,6 +1125,17 @@ ee_status_t ee_model_set_branches(ee_model_t* m, int enabled) {
   return EE_OK;
 }
 
+ee_status_t ee_model_set_stage_kernel(ee_model_t* m, int enabled, int max_batch) {
+  if (!m || max_batch < 0) return EE_ERR_INVALID_ARG;
+  m->stage_kernel = enabled != 0;
+  m->stage_kernel_max_batch = max_batch == 0 ? (1 << 30) : max_batch;
+  for (auto& sp : m->stages) {
+    for (auto& g : sp.graphs) sp.retired.push_back(g.exec);
+    sp.graphs.clear();
+  }
+  return EE_OK;
+}
+
 ee_status_t ee_model_set_timing(ee_model_t* m, int enabled) {
   if (!m) return EE_ERR_INVALID_ARG;
   m->timing = enabled != 0;
@@ -1088,6 +1179,10 @@ ee_status_t ee_model_plan(const ee_model_t* m, int stage, int batch, int cap, ee
     p.bytes = in_b + out_b + w_b + (L.res_slot != -2 ? out_b : 0.0);
     p.launches = 1;
   }
+  if (stage_kernel_active(m, sp, batch))   // a run of layers is one launch: its first layer carries it
+    for (const auto& seg : sp.segments)
+      for (int j = 1; j < seg.n; ++j)
+        if (sp.order[seg.first + j] < *n) out[sp.order[seg.first + j]].launches = 0;
   return EE_OK;
 }
 
@@ -1166,6 +1261,7 @@ ee_status_t ee_model_check(ee_model_t* m, void* cuda_stream) {
   if (flag) {
     // a kernel that gave up may have left arrival counters of a split-K reduction behind
     if (m->pair_counters) EE_CUDA(cudaMemsetAsync(m->pair_counters, 0, m->pair_counter_words * sizeof(unsigned), st));
+    if (m->grid_bar) EE_CUDA(cudaMemsetAsync(m->grid_bar, 0, 256, st));
     EE_CUDA(cudaMemsetAsync(m->err_flag, 0, sizeof(int), st));
     EE_CUDA(cudaStreamSynchronize(st));
     return EE_ERR_TIMEOUT;

@@ -46,7 +46,7 @@ struct PairParams {
   int rev;              // 1: walk the units from the last one down
   float* partial;       // split-K partial tiles (splits > 1)
   unsigned* counters;   // per (tile, CTA of the pair, epilogue warp); zero between launches
-  long long wait_cycles;
+  int res_late;         // the residual operand is written by the layer just before this one in the same launch
 };
 
 template <int BN>
@@ -133,10 +133,44 @@ __host__ __device__ constexpr uint32_t umma2_idesc(int n) {   // bf16 x bf16 -> 
 
 // ----------------------------------------------------------------------------- kernel
 
+constexpr int kPairMaxLayers = 20;
+
+// Everything the kernel needs for a run of consecutive layers (one layer in the plain case).  Passed as one
+// __grid_constant__ argument: the tensor maps are used in place from the parameter space.
+struct PairStageArgs {
+  int n_layers;
+  unsigned* grid_bar;       // [kPairMaxLayers + 1] arrival counters of the barriers between layers; zero between launches
+  int* err_flag;
+  long long wait_cycles;
+  PairParams layer[kPairMaxLayers];
+  CUtensorMap tmA[kPairMaxLayers], tmW[kPairMaxLayers], tmR[kPairMaxLayers], tmO[kPairMaxLayers];
+};
+
+// Bounded spin on a global arrival counter (acquire at GPU scope).
+__device__ __forceinline__ bool grid_bar_wait(const unsigned* ctr, unsigned target, int* err_flag, long long limit) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+  if (v >= target) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+    if (v >= target) return true;
+    if (clock64() - t0 > limit) {
+      atomicExch(err_flag, (int)EE_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
+
+// A run of layers in one launch.  Layer l + 1 reads what layer l wrote, so between two layers every CTA's epilogue
+// warps wait for their own output stores to complete and the CTA arrives on a global counter; a CTA's producer
+// requests the first weight tiles of the next layer at once (nobody writes weights) and spins on the counter only
+// before its first activation tile.  The ring, the accumulator parity and the staging chunks carry on across layers.
+// All CTAs of the grid must be resident together (the grid is never larger than one CTA per SM); the spin is bounded
+// like every other wait.  With n_layers = 1 there is no barrier at all.
 template <int BN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
-conv_igemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
-                               const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmO, PairParams p) {
+conv_igemm_tcgen05_pair_kernel(const __grid_constant__ PairStageArgs A) {
   extern __shared__ uint8_t smem_raw[];
   using S = PairSmem<BN>;
   constexpr int kStages = S::kStages;
@@ -155,10 +189,9 @@ conv_igemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();        // 0: leader (issues the MMAs), 1: peer
   const int pair = (int)(blockIdx.x >> 1), n_pairs = (int)(gridDim.x >> 1);
-  const int num_kb_all = p.taps * p.cblocks;
-  const int total_units = p.m_tiles * p.n_tiles * p.splits;
-  const int my_units = pair < total_units ? (total_units - 1 - pair) / n_pairs + 1 : 0;
-  const long long limit = p.wait_cycles;
+  const long long limit = A.wait_cycles;
+  const int L = A.n_layers;
+  int* const err_flag = A.err_flag;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -173,10 +206,9 @@ conv_igemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0 && lane == 0) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmO) : "memory");
-    if (p.has_res) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmR) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&A.tmA[0]) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&A.tmW[0]) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&A.tmO[0]) : "memory");
   }
   if (warp == 1) {  // two accumulators of BN fp32 columns, allocated in both CTAs of the pair
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(2 * BN) : "memory");
@@ -189,9 +221,14 @@ conv_igemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-  // unit i of this pair -> (tile, K range)
-  auto unit_of = [&](int i, int& mt, int& nt, int& z) {
-    const int uf = pair + i * n_pairs, u = p.rev ? total_units - 1 - uf : uf;
+  // units of this pair in layer `l`: unit i -> (tile, K range)
+  auto units_of = [&](const PairParams& p) {
+    const int total = p.m_tiles * p.n_tiles * p.splits;
+    return pair < total ? (total - 1 - pair) / n_pairs + 1 : 0;
+  };
+  auto unit_of = [&](const PairParams& p, int i, int& mt, int& nt, int& z) {
+    const int total = p.m_tiles * p.n_tiles * p.splits;
+    const int uf = pair + i * n_pairs, u = p.rev ? total - 1 - uf : uf;
     const int t = u / p.splits;
     z = u - t * p.splits;
     mt = t / p.n_tiles;
@@ -200,42 +237,71 @@ conv_igemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __
 
   if (warp == 0) {
     if (lane == 0) {
-      int g = 0;   // K blocks issued so far, across units: the ring never drains at a unit boundary
+      int g = 0;   // K blocks issued so far, across units and layers: the ring never drains at a boundary
       bool ok = true;
-      for (int i = 0; i < my_units && ok; ++i) {
-        int mt, nt, z;
-        unit_of(i, mt, nt, z);
-        const int m0 = mt * 256 + (int)rank * kTcBM;       // this CTA's rows
-        const int nb0 = nt * BN + (int)rank * HALF;        // this CTA's weight rows
-        const bool rows = m0 < p.M;                        // a peer whose rows all lie past M loads no A tile
-        const bool peer_rows = mt * 256 + kTcBM < p.M;
-        const int kb_begin = z * p.kb_per, kb_end = min(num_kb_all, kb_begin + p.kb_per);
-        int cw = 0, ch = 0, cn = 0;
-        if (p.im2col && rows) {
-          const int hw = p.Ho * p.Wo;
-          cn = m0 / hw;
-          const int rem = m0 - cn * hw;
-          const int ho = rem / p.Wo;
-          cw = (rem - ho * p.Wo) * p.stride - p.pad;
-          ch = ho * p.stride - p.pad;
-        }
-        for (int kb = kb_begin; kb < kb_end; ++kb, ++g) {
-          const int s = g % kStages;
-          const uint32_t ph = (uint32_t)(g / kStages) & 1u;
-          const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
-          const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
-          ok = mbar_wait_for(empty_bar(s), ph ^ 1u, p.err_flag, limit);
-          if (!ok) break;
-          const uint32_t fb = map_to_rank(full_bar(s), 0);   // the leader's barrier collects all four loads
-          if (rank == 0) mbar_expect_tx(full_bar(s), (uint32_t)(2 * S::kBBytes + S::kABytes + (peer_rows ? S::kABytes : 0)));
-          tma2_load_3d(sb, &tmW, fb, cb * kTcBK, tap, nb0);
-          if (rows) {
+      for (int l = 0; l < L && ok; ++l) {
+        const PairParams& p = A.layer[l];
+        const CUtensorMap* tmA = &A.tmA[l];
+        const CUtensorMap* tmW = &A.tmW[l];
+        const int num_kb_all = p.taps * p.cblocks;
+        const int my_units = units_of(p);
+        bool inputs_ready = l == 0;   // layer 0: the dependency wait above
+        for (int i = 0; i < my_units && ok; ++i) {
+          int mt, nt, z;
+          unit_of(p, i, mt, nt, z);
+          const int m0 = mt * 256 + (int)rank * kTcBM;       // this CTA's rows
+          const int nb0 = nt * BN + (int)rank * HALF;        // this CTA's weight rows
+          const bool rows = m0 < p.M;                        // a peer whose rows all lie past M loads no A tile
+          const bool peer_rows = mt * 256 + kTcBM < p.M;
+          const int kb_begin = z * p.kb_per, kb_end = min(num_kb_all, kb_begin + p.kb_per);
+          int cw = 0, ch = 0, cn = 0;
+          if (p.im2col && rows) {
+            const int hw = p.Ho * p.Wo;
+            cn = m0 / hw;
+            const int rem = m0 - cn * hw;
+            const int ho = rem / p.Wo;
+            cw = (rem - ho * p.Wo) * p.stride - p.pad;
+            ch = ho * p.stride - p.pad;
+          }
+          auto arm_and_load_w = [&](int kb, int gg) -> bool {
+            const int s = gg % kStages;
+            const uint32_t ph = (uint32_t)(gg / kStages) & 1u;
+            const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
+            if (!mbar_wait_for(empty_bar(s), ph ^ 1u, err_flag, limit)) return false;
+            if (rank == 0) mbar_expect_tx(full_bar(s), (uint32_t)(2 * S::kBBytes + S::kABytes + (peer_rows ? S::kABytes : 0)));
+            tma2_load_3d(base + (uint32_t)s * S::kStage + S::kABytes, tmW, map_to_rank(full_bar(s), 0), cb * kTcBK, tap, nb0);
+            return true;
+          };
+          auto load_a = [&](int kb, int gg) {
+            if (!rows) return;
+            const int s = gg % kStages;
+            const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
+            const uint32_t sa = base + (uint32_t)s * S::kStage, fb = map_to_rank(full_bar(s), 0);
             if (p.im2col) {
               const int r = tap / p.kw;
-              tma2_load_im2col_4d(sa, &tmA, fb, cb * kTcBK, cw, ch, cn, (uint16_t)(tap - r * p.kw), (uint16_t)r);
+              tma2_load_im2col_4d(sa, tmA, fb, cb * kTcBK, cw, ch, cn, (uint16_t)(tap - r * p.kw), (uint16_t)r);
             } else {
-              tma2_load_2d(sa, &tmA, fb, cb * kTcBK, m0);
+              tma2_load_2d(sa, tmA, fb, cb * kTcBK, m0);
             }
+          };
+          int kb = kb_begin;
+          if (!inputs_ready) {
+            // first unit of a later layer: weight tiles of the first ring slots now, activation tiles once every CTA
+            // of the grid has finished the layer before
+            const int ahead = min(kStages, kb_end - kb_begin);
+            for (int j = 0; j < ahead && ok; ++j) ok = arm_and_load_w(kb_begin + j, g + j);
+            if (ok) ok = grid_bar_wait(A.grid_bar + (l - 1), gridDim.x, err_flag, limit);
+            if (!ok) break;
+            asm volatile("fence.proxy.async.global;" ::: "memory");   // the acquire above orders the TMA reads below
+            for (int j = 0; j < ahead; ++j) load_a(kb_begin + j, g + j);
+            kb += ahead;
+            g += ahead;
+            inputs_ready = true;
+          }
+          for (; kb < kb_end; ++kb, ++g) {
+            ok = arm_and_load_w(kb, g);
+            if (!ok) break;
+            load_a(kb, g);
           }
         }
       }
@@ -243,32 +309,37 @@ conv_igemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __
   } else if (warp == 1) {
     if (lane == 0 && rank == 0) {
       constexpr uint32_t idesc = umma2_idesc(BN);
-      int g = 0;
+      int g = 0, ui = 0;   // K blocks and units so far, across layers
       bool ok = true;
-      for (int i = 0; i < my_units && ok; ++i) {
-        int mt, nt, z;
-        unit_of(i, mt, nt, z);
-        const int kb_begin = z * p.kb_per, kb_end = min(num_kb_all, kb_begin + p.kb_per);
-        const int b = i & 1;
-        if (i >= 2) {  // the epilogue warps of both CTAs must have drained this accumulator (unit i - 2)
-          ok = mbar_wait_for(acc_empty(b), (uint32_t)((i >> 1) - 1) & 1u, p.err_flag, limit);
-          if (!ok) break;
-          tc_fence_after();
-        }
-        const uint32_t acc = tmem_base + (uint32_t)(b * BN);
-        for (int kb = kb_begin; kb < kb_end; ++kb, ++g) {
-          const int s = g % kStages;
-          const uint32_t ph = (uint32_t)(g / kStages) & 1u;
-          ok = mbar_wait_for(full_bar(s), ph, p.err_flag, limit);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
+      for (int l = 0; l < L && ok; ++l) {
+        const PairParams& p = A.layer[l];
+        const int num_kb_all = p.taps * p.cblocks;
+        const int my_units = units_of(p);
+        for (int i = 0; i < my_units && ok; ++i, ++ui) {
+          int mt, nt, z;
+          unit_of(p, i, mt, nt, z);
+          const int kb_begin = z * p.kb_per, kb_end = min(num_kb_all, kb_begin + p.kb_per);
+          const int b = ui & 1;
+          if (ui >= 2) {  // the epilogue warps of both CTAs must have drained this accumulator (unit ui - 2)
+            ok = mbar_wait_for(acc_empty(b), (uint32_t)((ui >> 1) - 1) & 1u, err_flag, limit);
+            if (!ok) break;
+            tc_fence_after();
+          }
+          const uint32_t acc = tmem_base + (uint32_t)(b * BN);
+          for (int kb = kb_begin; kb < kb_end; ++kb, ++g) {
+            const int s = g % kStages;
+            const uint32_t ph = (uint32_t)(g / kStages) & 1u;
+            ok = mbar_wait_for(full_bar(s), ph, err_flag, limit);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
 #pragma unroll
-          for (int k = 0; k < kTcBK / 16; ++k)
-            umma2_bf16(acc, umma_desc(sa + k * 32), umma_desc(sb + k * 32), idesc, (uint32_t)((kb > kb_begin) | (k != 0)));
-          umma2_commit_both(empty_bar(s));   // frees the slot in both CTAs once these MMAs have read it
+            for (int k = 0; k < kTcBK / 16; ++k)
+              umma2_bf16(acc, umma_desc(sa + k * 32), umma_desc(sb + k * 32), idesc, (uint32_t)((kb > kb_begin) | (k != 0)));
+            umma2_commit_both(empty_bar(s));   // frees the slot in both CTAs once these MMAs have read it
+          }
+          if (ok) umma2_commit_both(acc_full(b));
         }
-        if (ok) umma2_commit_both(acc_full(b));
       }
     }
   } else {
@@ -280,147 +351,183 @@ conv_igemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __
     const uint32_t io_s = base + S::kIoOff + ew * S::kWarpIo;
     const uint32_t acc_empty_leader0 = map_to_rank(acc_empty(0), 0), acc_empty_leader1 = map_to_rank(acc_empty(1), 0);
     bool ok = true;
-    int sc_n0 = -1;
-    bool pending = false;      // lane 0: a bulk store group of this warp may still be reading the staging chunks
+    bool pending = false;      // lane 0: a bulk store group of this warp may still be in flight
     uint32_t res_phase = 0;
-    for (int i = 0; i < my_units; ++i) {
-      int mt, nt, z;
-      unit_of(i, mt, nt, z);
-      const int m0 = mt * 256 + (int)rank * kTcBM, n0 = nt * BN, c_base = n0 + h * HALF;   // this warp's first column
-      const int b = i & 1;
-      const bool live = m0 + q * 32 < p.M && c_base < p.N;    // this warp has something to store
-      const bool split = p.splits > 1;
-      if (c_base != sc_n0) {
+    int ui = 0;
+    int prev_units = 0;
+    for (int l = 0; l < L; ++l) {   // a warp whose wait ran out skips the work but still meets the others at the layer's end
+      const PairParams& p = A.layer[l];
+      const CUtensorMap* tmR = &A.tmR[l];
+      const CUtensorMap* tmO = &A.tmO[l];
+      const int my_units = units_of(p);
+      int sc_n0 = -1;
+      for (int i = 0; i < my_units && ok; ++i, ++ui) {
+        int mt, nt, z;
+        unit_of(p, i, mt, nt, z);
+        const int m0 = mt * 256 + (int)rank * kTcBM, n0 = nt * BN, c_base = n0 + h * HALF;   // this warp's first column
+        const int b = ui & 1;
+        const bool live = m0 + q * 32 < p.M && c_base < p.N;    // this warp has something to store
+        const bool split = p.splits > 1;
+        if (c_base != sc_n0) {
+          __syncwarp();
+          for (int j = lane; j < HALF; j += 32) {
+            const bool in = c_base + j < p.N;
+            sc[j] = (p.scale && in) ? p.scale[c_base + j] : 1.f;
+            sc[HALF + j] = (p.bias && in) ? p.bias[c_base + j] : 0.f;
+          }
+          sc_n0 = c_base;
+        }
         __syncwarp();
-        for (int j = lane; j < HALF; j += 32) {
-          const bool in = c_base + j < p.N;
-          sc[j] = (p.scale && in) ? p.scale[c_base + j] : 1.f;
-          sc[HALF + j] = (p.bias && in) ? p.bias[c_base + j] : 0.f;
+        // the staging chunks are about to be rewritten (residual load or output): the previous store must have read them
+        if (lane == 0 && pending) {
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          pending = false;
         }
-        sc_n0 = c_base;
-      }
-      __syncwarp();
-      // the staging chunks are about to be rewritten (residual load or output): the previous store must have read them
-      if (lane == 0 && pending) {
-        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-        pending = false;
-      }
-      __syncwarp();
-      auto fetch_residual = [&]() {   // this warp's 32 rows x HALF columns of the residual operand, into the staging chunks
-        if (lane == 0) {
-          int chunks = 0;
-          for (int c = 0; c < S::kChunks; ++c)
-            if (c_base + c * 64 < p.N) ++chunks;
-          mbar_expect_tx(res_bar(ew), (uint32_t)(chunks * 4096));
-          for (int c = 0; c < S::kChunks; ++c)
-            if (c_base + c * 64 < p.N) tma_load_2d(io_s + c * 4096, &tmR, res_bar(ew), c_base + c * 64, m0 + q * 32);
+        __syncwarp();
+        auto fetch_residual = [&]() {   // this warp's 32 rows x HALF columns of the residual operand, into the staging chunks
+          if (lane == 0) {
+            int chunks = 0;
+            for (int c = 0; c < S::kChunks; ++c)
+              if (c_base + c * 64 < p.N) ++chunks;
+            mbar_expect_tx(res_bar(ew), (uint32_t)(chunks * 4096));
+            for (int c = 0; c < S::kChunks; ++c)
+              if (c_base + c * 64 < p.N) tma_load_2d(io_s + c * 4096, tmR, res_bar(ew), c_base + c * 64, m0 + q * 32);
+          }
+        };
+        // res_late: the residual operand was written by the layer just before this one in the same launch, so it may
+        // only be requested once this unit's accumulator is complete (its activation tiles came after the grid barrier)
+        // Early request only when the layer that wrote the residual operand is known to be complete on the whole grid:
+        // in layer 0, behind this layer's first unit (its accumulator implies the barrier before this layer), or
+        // when this CTA worked in the layer before and the operand is older than that layer.
+        const bool res_early = l == 0 || i > 0 || (prev_units > 0 && !p.res_late);
+        const bool res_now = p.has_res && live && !split && res_early;
+        if (res_now) fetch_residual();
+        ok = __all_sync(0xffffffffu, mbar_wait_for(acc_full(b), (uint32_t)(ui >> 1) & 1u, err_flag, limit));
+        if (!ok) break;
+        tc_fence_after();
+        if (p.has_res && live && !split && !res_early) {
+          asm volatile("fence.proxy.async.global;" ::: "memory");
+          fetch_residual();
         }
-      };
-      const bool res_now = p.has_res && live && !split;
-      if (res_now) fetch_residual();
-      ok = __all_sync(0xffffffffu, mbar_wait_for(acc_full(b), (uint32_t)(i >> 1) & 1u, p.err_flag, limit));
-      if (!ok) break;
-      tc_fence_after();
-      const uint32_t acc = tmem_base + (uint32_t)(b * BN + h * HALF) + ((uint32_t)(q * 32) << 16);
-      bool reduce = !split;
-      float* part = nullptr;
-      if (split) {
-        // region of this warp in the partial tile of (tile, range z, CTA rank): [HALF / 4 column groups][32 lanes][4] fp32
-        const size_t region = (size_t)32 * HALF;
-        const size_t tile = (size_t)mt * p.n_tiles + nt;
-        part = p.partial + (((tile * p.splits) * 2 + rank) * kPairEpiWarps + ew) * region;   // range 0; range z at + z * 2 * 8 * region
-        float* mine = part + (size_t)z * 2 * kPairEpiWarps * region;
+        const uint32_t acc = tmem_base + (uint32_t)(b * BN + h * HALF) + ((uint32_t)(q * 32) << 16);
+        bool reduce = !split;
+        float* part = nullptr;
+        if (split) {
+          // region of this warp in the partial tile of (tile, range z, CTA rank): [HALF / 4 column groups][32 lanes][4] fp32
+          const size_t region = (size_t)32 * HALF;
+          const size_t tile = (size_t)mt * p.n_tiles + nt;
+          part = p.partial + (((tile * p.splits) * 2 + rank) * kPairEpiWarps + ew) * region;   // range 0; range z at + z * 2 * 8 * region
+          float* mine = part + (size_t)z * 2 * kPairEpiWarps * region;
+#pragma unroll 1
+          for (int c = 0; c < S::kChunks; ++c) {
+            float va[32], vb[32];
+            tmem_ld32_issue(acc + (uint32_t)(c * 64), va);
+            tmem_ld32_issue(acc + (uint32_t)(c * 64 + 32), vb);
+            tmem_ld_wait(va, vb);
+            if (live) {
+#pragma unroll
+              for (int g4 = 0; g4 < 8; ++g4) {
+                __stcg(reinterpret_cast<float4*>(mine) + (size_t)(c * 16 + g4) * 32 + lane, make_float4(va[4 * g4], va[4 * g4 + 1], va[4 * g4 + 2], va[4 * g4 + 3]));
+                __stcg(reinterpret_cast<float4*>(mine) + (size_t)(c * 16 + 8 + g4) * 32 + lane, make_float4(vb[4 * g4], vb[4 * g4 + 1], vb[4 * g4 + 2], vb[4 * g4 + 3]));
+              }
+            }
+          }
+          tc_fence_before();
+          __threadfence();
+          __syncwarp();
+          unsigned old = 0;
+          if (lane == 0) {
+            mbar_arrive_cluster(b ? acc_empty_leader1 : acc_empty_leader0);   // accumulator drained
+            if (live) old = atomicAdd(p.counters + (tile * 2 + rank) * kPairEpiWarps + ew, 1u);
+          }
+          old = __shfl_sync(0xffffffffu, old, 0);
+          reduce = live && old == (unsigned)(p.splits - 1);
+          if (reduce) {
+            __threadfence();
+            if (lane == 0) p.counters[(tile * 2 + rank) * kPairEpiWarps + ew] = 0u;   // ready for the next launch
+            if (p.has_res) {
+              asm volatile("fence.proxy.async.global;" ::: "memory");
+              fetch_residual();
+            }
+          }
+        }
+        if (reduce && (p.has_res && live)) {
+          ok = __all_sync(0xffffffffu, mbar_wait_for(res_bar(ew), res_phase, err_flag, limit));
+          res_phase ^= 1u;
+          if (!ok) break;
+        }
 #pragma unroll 1
         for (int c = 0; c < S::kChunks; ++c) {
           float va[32], vb[32];
-          tmem_ld32_issue(acc + (uint32_t)(c * 64), va);
-          tmem_ld32_issue(acc + (uint32_t)(c * 64 + 32), vb);
-          tmem_ld_wait(va, vb);
-          if (live) {
+          if (!split) {
+            tmem_ld32_issue(acc + (uint32_t)(c * 64), va);
+            tmem_ld32_issue(acc + (uint32_t)(c * 64 + 32), vb);
+            tmem_ld_wait(va, vb);
+            if (c == S::kChunks - 1) {  // this warp's share of the accumulator is in registers: the MMA warp may refill it
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive_cluster(b ? acc_empty_leader1 : acc_empty_leader0);
+            }
+          } else if (reduce) {
+            // partials of ranges 0, 1, ... in ascending order (range 0 first, so the sum starts from it)
+            const size_t zs = (size_t)2 * kPairEpiWarps * 32 * HALF / 4;   // float4 stride between ranges
+            const float4* p4 = reinterpret_cast<const float4*>(part) + (size_t)(c * 16) * 32 + lane;
 #pragma unroll
             for (int g4 = 0; g4 < 8; ++g4) {
-              __stcg(reinterpret_cast<float4*>(mine) + (size_t)(c * 16 + g4) * 32 + lane, make_float4(va[4 * g4], va[4 * g4 + 1], va[4 * g4 + 2], va[4 * g4 + 3]));
-              __stcg(reinterpret_cast<float4*>(mine) + (size_t)(c * 16 + 8 + g4) * 32 + lane, make_float4(vb[4 * g4], vb[4 * g4 + 1], vb[4 * g4 + 2], vb[4 * g4 + 3]));
+              const float4 x = __ldcg(p4 + (size_t)g4 * 32), y = __ldcg(p4 + (size_t)(8 + g4) * 32);
+              va[4 * g4] = x.x, va[4 * g4 + 1] = x.y, va[4 * g4 + 2] = x.z, va[4 * g4 + 3] = x.w;
+              vb[4 * g4] = y.x, vb[4 * g4 + 1] = y.y, vb[4 * g4 + 2] = y.z, vb[4 * g4 + 3] = y.w;
+            }
+            for (int zz = 1; zz < p.splits; ++zz) {
+#pragma unroll
+              for (int g4 = 0; g4 < 8; ++g4) {
+                const float4 x = __ldcg(p4 + zz * zs + (size_t)g4 * 32), y = __ldcg(p4 + zz * zs + (size_t)(8 + g4) * 32);
+                va[4 * g4] += x.x, va[4 * g4 + 1] += x.y, va[4 * g4 + 2] += x.z, va[4 * g4 + 3] += x.w;
+                vb[4 * g4] += y.x, vb[4 * g4 + 1] += y.y, vb[4 * g4 + 2] += y.z, vb[4 * g4 + 3] += y.w;
+              }
+            }
+          }
+          if (!reduce || !live || c_base + c * 64 >= p.N) continue;
+          uint8_t* line = io + c * 4096 + lane * 128;   // this thread's 128-byte row of the chunk, 16-byte groups XOR-swizzled with the row
+#pragma unroll
+          for (int sub = 0; sub < 2; ++sub) {
+            const float* v = sub ? vb : va;
+#pragma unroll
+            for (int gq = 0; gq < 4; ++gq) {
+              const int col = c * 64 + sub * 32 + gq * 8;    // within this warp's HALF columns
+              if (c_base + col >= p.N) break;
+              uint4* chunk = reinterpret_cast<uint4*>(line + (((sub * 4 + gq) ^ (lane & 7)) << 4));
+              if (p.has_res)
+                *chunk = epilogue8_act<true>(p.act, v + gq * 8, sc + col, sc + HALF + col, *chunk);
+              else
+                *chunk = epilogue8_act<false>(p.act, v + gq * 8, sc + col, sc + HALF + col, make_uint4(0u, 0u, 0u, 0u));
             }
           }
         }
-        tc_fence_before();
+        if (reduce && live) {
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the TMA unit
+          __syncwarp();
+          if (lane == 0) {
+            for (int c = 0; c < S::kChunks; ++c)
+              if (c_base + c * 64 < p.N) tma_store_2d(tmO, io_s + c * 4096, c_base + c * 64, m0 + q * 32);   // rows past M, columns past N: clipped
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            pending = true;
+          }
+        }
+      }
+      prev_units = my_units;
+      if (l + 1 < L) {
+        // end of a layer: this warp's stores must be complete (not merely read from shared memory) before the CTA tells
+        // the grid that its part of the layer's output is in place
+        if (lane == 0) {
+          asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+          pending = false;
+        }
         __threadfence();
-        __syncwarp();
-        unsigned old = 0;
-        if (lane == 0) {
-          mbar_arrive_cluster(b ? acc_empty_leader1 : acc_empty_leader0);   // accumulator drained
-          if (live) old = atomicAdd(p.counters + (tile * 2 + rank) * kPairEpiWarps + ew, 1u);
-        }
-        old = __shfl_sync(0xffffffffu, old, 0);
-        reduce = live && old == (unsigned)(p.splits - 1);
-        if (reduce) {
-          __threadfence();
-          if (lane == 0) p.counters[(tile * 2 + rank) * kPairEpiWarps + ew] = 0u;   // ready for the next launch
-          if (p.has_res) fetch_residual();
-        }
-      }
-      if (reduce && (p.has_res && live)) {
-        ok = __all_sync(0xffffffffu, mbar_wait_for(res_bar(ew), res_phase, p.err_flag, limit));
-        res_phase ^= 1u;
-        if (!ok) break;
-      }
-#pragma unroll 1
-      for (int c = 0; c < S::kChunks; ++c) {
-        float va[32], vb[32];
-        if (!split) {
-          tmem_ld32_issue(acc + (uint32_t)(c * 64), va);
-          tmem_ld32_issue(acc + (uint32_t)(c * 64 + 32), vb);
-          tmem_ld_wait(va, vb);
-          if (c == S::kChunks - 1) {  // this warp's share of the accumulator is in registers: the MMA warp may refill it
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(b ? acc_empty_leader1 : acc_empty_leader0);
-          }
-        } else if (reduce) {
-          // partials of ranges 0, 1, ... in ascending order (range 0 first, so the sum starts from it)
-          const size_t zs = (size_t)2 * kPairEpiWarps * 32 * HALF / 4;   // float4 stride between ranges
-          const float4* p4 = reinterpret_cast<const float4*>(part) + (size_t)(c * 16) * 32 + lane;
-#pragma unroll
-          for (int g4 = 0; g4 < 8; ++g4) {
-            const float4 x = __ldcg(p4 + (size_t)g4 * 32), y = __ldcg(p4 + (size_t)(8 + g4) * 32);
-            va[4 * g4] = x.x, va[4 * g4 + 1] = x.y, va[4 * g4 + 2] = x.z, va[4 * g4 + 3] = x.w;
-            vb[4 * g4] = y.x, vb[4 * g4 + 1] = y.y, vb[4 * g4 + 2] = y.z, vb[4 * g4 + 3] = y.w;
-          }
-          for (int zz = 1; zz < p.splits; ++zz) {
-#pragma unroll
-            for (int g4 = 0; g4 < 8; ++g4) {
-              const float4 x = __ldcg(p4 + zz * zs + (size_t)g4 * 32), y = __ldcg(p4 + zz * zs + (size_t)(8 + g4) * 32);
-              va[4 * g4] += x.x, va[4 * g4 + 1] += x.y, va[4 * g4 + 2] += x.z, va[4 * g4 + 3] += x.w;
-              vb[4 * g4] += y.x, vb[4 * g4 + 1] += y.y, vb[4 * g4 + 2] += y.z, vb[4 * g4 + 3] += y.w;
-            }
-          }
-        }
-        if (!reduce || !live || c_base + c * 64 >= p.N) continue;
-        uint8_t* line = io + c * 4096 + lane * 128;   // this thread's 128-byte row of the chunk, 16-byte groups XOR-swizzled with the row
-#pragma unroll
-        for (int sub = 0; sub < 2; ++sub) {
-          const float* v = sub ? vb : va;
-#pragma unroll
-          for (int gq = 0; gq < 4; ++gq) {
-            const int col = c * 64 + sub * 32 + gq * 8;    // within this warp's HALF columns
-            if (c_base + col >= p.N) break;
-            uint4* chunk = reinterpret_cast<uint4*>(line + (((sub * 4 + gq) ^ (lane & 7)) << 4));
-            if (p.has_res)
-              *chunk = epilogue8_act<true>(p.act, v + gq * 8, sc + col, sc + HALF + col, *chunk);
-            else
-              *chunk = epilogue8_act<false>(p.act, v + gq * 8, sc + col, sc + HALF + col, make_uint4(0u, 0u, 0u, 0u));
-          }
-        }
-      }
-      if (reduce && live) {
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the TMA unit
-        __syncwarp();
-        if (lane == 0) {
-          for (int c = 0; c < S::kChunks; ++c)
-            if (c_base + c * 64 < p.N) tma_store_2d(&tmO, io_s + c * 4096, c_base + c * 64, m0 + q * 32);   // rows past M, columns past N: clipped
-          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-          pending = true;
+        asm volatile("bar.sync 2, 256;" ::: "memory");   // the eight epilogue warps of this CTA
+        if (ew == 0 && lane == 0) {
+          asm volatile("fence.proxy.async.global;" ::: "memory");
+          asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(A.grid_bar + l) : "memory");
         }
       }
     }
@@ -432,6 +539,15 @@ conv_igemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * BN) : "memory");
+  }
+  // the last CTA to leave puts the barrier counters back to zero for the next launch
+  if (L > 1 && threadIdx.x == 0) {
+    __threadfence();
+    const unsigned done = atomicAdd(A.grid_bar + kPairMaxLayers, 1u);
+    if (done == gridDim.x - 1) {
+      for (int l = 0; l <= kPairMaxLayers; ++l) A.grid_bar[l] = 0u;
+      __threadfence();
+    }
   }
 }
 
@@ -475,23 +591,24 @@ inline size_t pair_counter_words(const TcLayer& L, int B) {   // BN = 128 has th
   return (size_t)cdiv((long)B * L.out_h * L.out_w, 256) * cdiv(L.cout, 128) * 2 * kPairEpiWarps;
 }
 
-inline ee_status_t pair_launch(TcContext& c, const TcLayer& L, int variant, const void* src, const void* res, void* dst, int B,
-                               const float* scale, const float* bias, int* err_flag, float* partial, size_t partial_bytes,
-                               unsigned* counters, long long wait_cycles, cudaStream_t st) {
+// Fills layer slot `slot` of `args` for one layer at batch B.
+inline ee_status_t pair_fill_layer(TcContext& c, const TcLayer& L, int bn, const void* src, const void* res, void* dst, int B,
+                                   const float* scale, const float* bias, float* partial, size_t partial_bytes, unsigned* counters,
+                                   bool res_late, PairStageArgs* args, int slot) {
   if (((uintptr_t)src & 15) || ((uintptr_t)dst & 15) || ((uintptr_t)res & 15)) return EE_ERR_INVALID_ARG;
-  const int bn = variant == TCV_PAIR256 ? 256 : 128;
   const CUtensorMap* t = nullptr;
   ee_status_t s = tc_buffer_map(c, L, dst, B, 1, &t);
   if (s != EE_OK) return s;
-  const CUtensorMap tmO = *t;
+  args->tmO[slot] = *t;
   if ((s = tc_buffer_map(c, L, src, B, 0, &t)) != EE_OK) return s;
-  const CUtensorMap tmA = *t;
-  CUtensorMap tmR = tmO;
+  args->tmA[slot] = *t;
+  args->tmR[slot] = args->tmO[slot];
   if (res) {
     if ((s = tc_buffer_map(c, L, res, B, 1, &t)) != EE_OK) return s;
-    tmR = *t;
+    args->tmR[slot] = *t;
   }
-  PairParams p;
+  args->tmW[slot] = bn == 256 ? L.tm_w_half[0] : L.tm_w_half[1];
+  PairParams& p = args->layer[slot];
   p.M = B * L.out_h * L.out_w;
   p.N = L.cout;
   p.taps = L.kh * L.kw;
@@ -502,16 +619,27 @@ inline ee_status_t pair_launch(TcContext& c, const TcLayer& L, int variant, cons
   p.act = L.act;
   p.has_res = res ? 1 : 0;
   p.scale = scale, p.bias = bias;
-  p.err_flag = err_flag;
+  p.err_flag = nullptr;
   p.splits = L.splits, p.kb_per = L.kb_per;
   p.m_tiles = cdiv(p.M, 256), p.n_tiles = cdiv(p.N, bn);
   p.rev = L.rev ? 1 : 0;
   p.partial = partial;
   p.counters = counters;
-  p.wait_cycles = wait_cycles;
+  p.res_late = res_late ? 1 : 0;
   if (p.splits > 1 && (!partial || !counters || partial_bytes < pair_partial_bytes(L, B, bn))) return EE_ERR_CAPACITY;
-  const long units = (long)p.m_tiles * p.n_tiles * p.splits;
-  const int pairs = (int)std::min<long>(units, c.sm_count / 2);
+  return EE_OK;
+}
+
+// Launches the layers filled into `args` (n_layers of them) as one kernel.
+inline ee_status_t pair_launch_args(TcContext& c, PairStageArgs& args, int bn, int* err_flag, unsigned* grid_bar, long long wait_cycles,
+                                    cudaStream_t st) {
+  if (args.n_layers < 1 || args.n_layers > kPairMaxLayers || (args.n_layers > 1 && !grid_bar)) return EE_ERR_INTERNAL;
+  args.err_flag = err_flag;
+  args.grid_bar = grid_bar;
+  args.wait_cycles = wait_cycles;
+  long units = 0;
+  for (int l = 0; l < args.n_layers; ++l) units = std::max(units, (long)args.layer[l].m_tiles * args.layer[l].n_tiles * args.layer[l].splits);
+  const int pairs = (int)std::min<long>(units, c.sm_count / 2);   // never more than one CTA per SM: the grid is co-resident
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs);
   cfg.blockDim = dim3(kPairThreads);
@@ -522,10 +650,20 @@ inline ee_status_t pair_launch(TcContext& c, const TcLayer& L, int variant, cons
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const CUtensorMap& tmW = bn == 256 ? L.tm_w_half[0] : L.tm_w_half[1];
-  cudaError_t e = bn == 256 ? cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_pair_kernel<256>, tmA, tmW, tmR, tmO, p)
-                            : cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_pair_kernel<128>, tmA, tmW, tmR, tmO, p);
+  cudaError_t e = bn == 256 ? cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_pair_kernel<256>, args)
+                            : cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_pair_kernel<128>, args);
   return e == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+}
+
+inline ee_status_t pair_launch(TcContext& c, const TcLayer& L, int variant, const void* src, const void* res, void* dst, int B,
+                               const float* scale, const float* bias, int* err_flag, float* partial, size_t partial_bytes,
+                               unsigned* counters, long long wait_cycles, cudaStream_t st) {
+  const int bn = variant == TCV_PAIR256 ? 256 : 128;
+  static thread_local PairStageArgs args;   // 13 KB: kept off the stack
+  args.n_layers = 1;
+  ee_status_t s = pair_fill_layer(c, L, bn, src, res, dst, B, scale, bias, partial, partial_bytes, counters, false, &args, 0);
+  if (s != EE_OK) return s;
+  return pair_launch_args(c, args, bn, err_flag, nullptr, wait_cycles, st);
 }
 
 }  // namespace ee

@@ -745,6 +745,40 @@ def test_branch_execution_of_shortcut_layers_is_bit_identical():
     m.check()
 
 
+@pytest.mark.parametrize("B", [1, 3, 7])
+def test_multi_layer_launch_is_bit_identical_to_layer_by_layer(B):
+    """Runs of layers executed as one persistent kernel with grid barriers between layers (an option) against the
+    same stages launched layer by layer: logits and survivors' features must agree bit for bit, on plain launches and
+    on replayed graphs, twice in a row (the barrier counters must return to zero)."""
+    spec = wl.resnet50_ee(seed=1, in_hw=96, n_classes=100, max_batch=7, alphas=[0.01] * 4)
+    run = util.GpuRunner(spec)
+    m, ws = run.m, run.ws
+    x = wl.make_input(spec, B, seed=4)
+    side = torch.cuda.Stream()
+    xd = eb.to_device("bf16", x)
+    for s in range(m.n_stages):
+        snaps = []
+        for mega, stream in ((False, None), (True, None), (True, side), (True, side), (True, None)):
+            m.set_stage_kernel(mega)
+            run.bufs[s].logits.fill_(0)
+            run.bufs[s].features_out.fill_(0)
+            with torch.cuda.stream(stream or torch.cuda.current_stream()):
+                m.stage_run(s, xd, B, run.bufs[s], ws)
+            torch.cuda.synchronize()
+            m.check()
+            n = int(run.bufs[s].n_surv_host[0])
+            snaps.append((n, run.bufs[s].logits[:B].clone(), run.bufs[s].features_out[:n].clone()))
+        for n, z, f in snaps[1:]:
+            assert n == snaps[0][0] and torch.equal(z, snaps[0][1]) and torch.equal(f, snaps[0][2]), f"stage {s}"
+        xd = run.bufs[s].features_out[:B].clone() if s + 1 < m.n_stages else xd
+    run.check_guards()
+    m.set_stage_kernel(True)
+    launches_on = sum(pl["launches"] for s in range(m.n_stages) for pl in m.plan(s, B))
+    m.set_stage_kernel(False)
+    launches_off = sum(pl["launches"] for s in range(m.n_stages) for pl in m.plan(s, B))
+    assert launches_on < launches_off
+
+
 def test_count_reaches_the_host_without_a_stream_sync():
     """B_exit is copied to the pinned word beside the gather (plain launches and graph replay): ee_wait_count returns it
     without synchronising the stream, and it equals the count of the synchronised run."""
