@@ -181,6 +181,8 @@ def run_ours(args):
     B, K, W = args.batch, args.steps, max(args.warmup, 3)
     spec, seed = make_spec(args.workload, B, flat_heads=args.exit_rate is not None)
     model = eb.EEModel(spec)
+    if args.device_sized:
+        model.set_chain(B)      # ee_run_until_exit as one graph: every next stage is sized on the device
     nst = model.n_stages
     bufs = [eb.StageBuffers(model, s, with_logits=False) for s in range(nst)]
     ws = model.workspace()
@@ -455,7 +457,8 @@ def run_ours(args):
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": spec.dtype, "data": "synthetic",
         "config": {"workload": workload_name(spec, B, args.exit_rate), "global_batch": world * B, "parallelism": f"replicas x{world}",
-                   "l2": "flushed between timed steps (256 MB write)", "batch_per_stage": sizes_last},
+                   "l2": "flushed between timed steps (256 MB write)", "batch_per_stage": sizes_last,
+                   "stage_chain": "device-sized (one graph, switch nodes)" if (args.device_sized and args.exit_rate is None) else "host-sized"},
         "clocks": clocks,
         "e2e": {"value": replicas.job_throughput(world, B, K, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / K},
@@ -549,6 +552,9 @@ def main():
     ap.add_argument("--policy", default="fluid", choices=["fluid", "serial", "adaptb"],
                     help="streaming trace: the exit-aware preemptive scheduler (default), one request at a time, or adaptive batching <B_max, T_timeout>")
     ap.add_argument("--timeout-ms", type=float, default=1.0, help="streaming trace, adaptive batching: T_timeout in ms")
+    ap.add_argument("--device-sized", action="store_true",
+                    help="run the stage chain as one graph whose switch nodes size every next stage on the device (measured slower "
+                         "than the default, in which the host reads each count from its pinned word and launches the next stage)")
     ap.add_argument("--cpu-samples", type=int, default=64)
     ap.add_argument("--report-layers", action="store_true", help="add a per-layer table (time, TFLOP/s, GB/s, roofline bound) to the JSON line")
     args = ap.parse_args()

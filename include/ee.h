@@ -299,6 +299,17 @@ ee_status_t ee_run_until_exit(ee_model_t* model, int first_stage, const ee_stage
                               size_t workspace_bytes, const ee_stage_out_t* outs, int32_t* batch_per_stage,
                               double timeout_s, void* cuda_stream);
 
+/* Device-sized stage chain.  With max_batch > 0, ee_run_until_exit on a batch of up to max_batch samples runs as ONE CUDA
+ * graph: the first stage at the caller's batch, then for every later stage a switch node with one body per possible
+ * survivor count (body b = that stage at batch b, count 0 = nothing), selected on the device from the count the stage
+ * before left in n_surv_dev (Section III, steps 3-4: B_exit sizes the next launch -- here without the host in the loop).
+ * The counts still travel to the pinned words, so ee_run_until_exit returns the same batch_per_stage; results are
+ * identical to the host-sized chain.  The graph of a (first stage, buffers, batch) signature is built at its first use
+ * (one capture per stage and possible count: tens of milliseconds at batch 64) and cached (16 signatures).  Needs a
+ * capturable stream and stage replay on; otherwise, and for larger batches, the host sizes every stage as before.
+ * max_batch = 0 (the default) switches it off.  Errors: INVALID_ARG. */
+ee_status_t ee_model_set_chain(ee_model_t* model, int max_batch);
+
 /* Host-side wait for a survivor count without synchronising the stream (Section III, step 4: the scheduler needs
  * B_exit, not the features, to size its next launch).  Protocol: the caller stores `sentinel` (a negative value) in
  * its pinned word, passes the word as n_surv_host to ee_stage_run, then calls this: it polls the word until it differs

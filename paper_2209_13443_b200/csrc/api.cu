@@ -162,6 +162,17 @@ struct ee_model {
   cudaStream_t side = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   cudaStream_t branch = nullptr;   // shortcut layers run here, beside the main chain of their block
+  cudaStream_t cap = nullptr;      // the bodies of a device-sized stage chain are captured on this stream
+  int chain_max_batch = 0;         // ee_run_until_exit runs as ONE graph for batches up to this size (0 = host-sized stages)
+  struct ChainGraph {
+    int first;
+    ee_stage_in_t in;
+    void* ws;
+    std::vector<ee_stage_out_t> outs;
+    cudaGraph_t graph;
+    cudaGraphExec_t exec;
+  };
+  std::vector<ChainGraph> chains;
   bool branches = true;
 };
 
@@ -450,6 +461,122 @@ ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, c
   return EE_OK;
 }
 
+// Device-sized stage chain (Section III, steps 3-4: B_exit decides how many samples the next subnet processes).  The
+// whole chain from `first` on is ONE graph: the first stage at its batch, and for every later stage a switch node with one
+// body per possible survivor count (body b = that stage captured at batch b; count 0 = nothing).  A one-thread kernel in
+// front of each switch reads the survivor count the stage before left in device memory and sets the switch: the device
+// sizes its own next launch, the host only reads the counts that still travel to its pinned words.
+__global__ void chain_select_kernel(cudaGraphConditionalHandle handle, const int32_t* n_surv) {
+  const int32_t n = *n_surv;
+  cudaGraphSetConditional(handle, n > 0 ? (unsigned)n : 0u);
+}
+
+bool same_chain(const ee_model::ChainGraph& c, int first, const ee_stage_in_t* in, void* ws, const ee_stage_out_t* outs, int n_stages) {
+  if (c.first != first || c.ws != ws || c.in.features != in->features || c.in.ids != in->ids || c.in.batch != in->batch ||
+      c.in.logit_shift != in->logit_shift || c.in.shift_class != in->shift_class)
+    return false;
+  for (int s = first; s < n_stages; ++s) {
+    StageCallKey a, b;
+    a.out = c.outs[s];
+    b.out = outs[s];
+    a.in = b.in = *in;
+    a.ws = b.ws = ws;
+    if (!same_call(a, b)) return false;
+  }
+  return true;
+}
+
+ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, char* ws, const ee_stage_out_t* out, cudaStream_t st);
+
+ee_status_t build_chain(ee_model* m, int first, const ee_stage_in_t* in, char* ws, const ee_stage_out_t* outs, ee_model::ChainGraph* out) {
+  const int n_stages = (int)m->stages.size();
+  cudaGraph_t g = nullptr;
+  EE_CUDA(cudaGraphCreate(&g, 0));
+  auto fail = [&](ee_status_t s) {
+    cudaGraphDestroy(g);
+    return s;
+  };
+  std::vector<cudaGraphNode_t> deps;
+  for (int s = first; s < n_stages; ++s) {   // a stage that never runs leaves a zero count behind
+    cudaMemsetParams mp = {};
+    mp.dst = outs[s].n_surv_dev;
+    mp.value = 0;
+    mp.elementSize = 4;
+    mp.width = 1;
+    mp.height = 1;
+    mp.pitch = 4;
+    cudaGraphNode_t node;
+    if (cudaGraphAddMemsetNode(&node, g, nullptr, 0, &mp) != cudaSuccess) return fail(EE_ERR_CUDA);
+    deps.push_back(node);
+  }
+  // the first stage, at the caller's batch
+  cudaGraph_t sub = nullptr;
+  if (cudaStreamBeginCapture(m->cap, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return fail(EE_ERR_CUDA);
+  ee_status_t es = enqueue_stage(m, m->stages[first], in, ws, &outs[first], m->cap);
+  cudaError_t ce = cudaStreamEndCapture(m->cap, &sub);
+  if (es != EE_OK || ce != cudaSuccess || !sub) {
+    if (sub) cudaGraphDestroy(sub);
+    return fail(es != EE_OK ? es : EE_ERR_CUDA);
+  }
+  cudaGraphNode_t prev;
+  ce = cudaGraphAddChildGraphNode(&prev, g, deps.data(), deps.size(), sub);
+  cudaGraphDestroy(sub);
+  if (ce != cudaSuccess) return fail(EE_ERR_CUDA);
+  for (int s = first + 1; s < n_stages; ++s) {
+    cudaGraphConditionalHandle handle;
+    if (cudaGraphConditionalHandleCreate(&handle, g, 0, cudaGraphCondAssignDefault) != cudaSuccess) return fail(EE_ERR_CUDA);
+    const int32_t* count = outs[s - 1].n_surv_dev;
+    void* kargs[2] = {(void*)&handle, (void*)&count};
+    cudaKernelNodeParams kp = {};
+    kp.func = (void*)chain_select_kernel;
+    kp.gridDim = dim3(1);
+    kp.blockDim = dim3(1);
+    kp.kernelParams = kargs;
+    cudaGraphNode_t sel;
+    if (cudaGraphAddKernelNode(&sel, g, &prev, 1, &kp) != cudaSuccess) return fail(EE_ERR_CUDA);
+    cudaGraphNodeParams np = {};
+    np.type = cudaGraphNodeTypeConditional;
+    np.conditional.handle = handle;
+    np.conditional.type = cudaGraphCondTypeSwitch;
+    np.conditional.size = (unsigned)in->batch + 1;
+    cudaGraphNode_t cond;
+    if (cudaGraphAddNode(&cond, g, &sel, 1, &np) != cudaSuccess) return fail(EE_ERR_CUDA);
+    for (int b = 1; b <= in->batch; ++b) {   // body b: this stage on b survivors of the stage before
+      ee_stage_in_t cur = {};
+      cur.features = outs[s - 1].features_out;
+      cur.ids = (in->ids && outs[s - 1].ids_out) ? outs[s - 1].ids_out : nullptr;
+      cur.batch = b;
+      cudaGraph_t body = np.conditional.phGraph_out[b];
+      if (cudaStreamBeginCaptureToGraph(m->cap, body, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return fail(EE_ERR_CUDA);
+      es = enqueue_stage(m, m->stages[s], &cur, ws, &outs[s], m->cap);
+      cudaGraph_t ended = nullptr;
+      ce = cudaStreamEndCapture(m->cap, &ended);
+      if (es != EE_OK || ce != cudaSuccess) return fail(es != EE_OK ? es : EE_ERR_CUDA);
+    }
+    prev = cond;
+  }
+  cudaGraphExec_t exec = nullptr;
+  if (cudaGraphInstantiate(&exec, g, 0) != cudaSuccess) {
+    g_cuda_err = std::string("device-sized stage chain: graph instantiation failed: ") + cudaGetErrorString(cudaGetLastError());
+    return fail(EE_ERR_CUDA);
+  }
+  out->first = first;
+  out->in = *in;
+  out->ws = ws;
+  out->outs.assign(outs, outs + n_stages);
+  out->graph = g;
+  out->exec = exec;
+  return EE_OK;
+}
+
+void drop_chains(ee_model* m) {   // whole-chain graphs hold the kernel choices they were captured with
+  for (auto& c : m->chains) {
+    cudaGraphExecDestroy(c.exec);
+    cudaGraphDestroy(c.graph);
+  }
+  m->chains.clear();
+}
+
 // The GPU that is current must be the one the model lives on: kernels launched elsewhere would dereference this
 // model's weights from another device.
 bool on_model_device(const ee_model* m) {
@@ -494,6 +621,11 @@ ee_status_t ee_model_destroy(ee_model_t* m) {
   if (m->ev_join) cudaEventDestroy(m->ev_join);
   if (m->side) cudaStreamDestroy(m->side);
   if (m->branch) cudaStreamDestroy(m->branch);
+  if (m->cap) cudaStreamDestroy(m->cap);
+  for (auto& c : m->chains) {
+    cudaGraphExecDestroy(c.exec);
+    cudaGraphDestroy(c.graph);
+  }
   for (auto& sp : m->stages)
     for (auto& L : sp.layers) {
       if (L.ev_fork) cudaEventDestroy(L.ev_fork);
@@ -534,7 +666,8 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
     m->err_flag = (int*)p;
     if (cudaMemsetAsync(p, 0, 256, st) != cudaSuccess) return fail(EE_ERR_CUDA);
   }
-  if (cudaStreamCreateWithFlags(&m->branch, cudaStreamNonBlocking) != cudaSuccess ||
+  if (cudaStreamCreateWithFlags(&m->cap, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&m->branch, cudaStreamNonBlocking) != cudaSuccess ||
       cudaStreamCreateWithFlags(&m->side, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&m->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming) != cudaSuccess)
@@ -878,6 +1011,48 @@ ee_status_t ee_run_until_exit(ee_model_t* m, int first_stage, const ee_stage_in_
     if (!outs[s].n_surv_host) return EE_ERR_INVALID_ARG;
   if (batch_per_stage)
     for (int s = 0; s < n_stages; ++s) batch_per_stage[s] = 0;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const bool legacy = st == nullptr || st == cudaStreamLegacy || st == cudaStreamPerThread;
+  if (in->batch >= 1 && in->batch <= m->chain_max_batch && first_stage + 1 < n_stages && m->graphs && !m->timing && !legacy &&
+      in->batch <= m->max_batch && in->features && workspace && !((uintptr_t)workspace & 255) && on_model_device(m)) {
+    // Device-sized chain: one graph launch; the host then only collects the counts as they arrive.
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) == cudaSuccess && cs == cudaStreamCaptureStatusNone) {
+      size_t need = 0;
+      for (int s = first_stage; s < n_stages; ++s) {
+        need = std::max(need, m->stages[s].ws_bytes);
+        if (!valid_out(&outs[s], true)) return EE_ERR_INVALID_ARG;
+      }
+      if (workspace_bytes < need) return EE_ERR_CAPACITY;
+      ee_model::ChainGraph* cg = nullptr;
+      for (auto& c : m->chains)
+        if (same_chain(c, first_stage, in, workspace, outs, n_stages)) cg = &c;
+      if (!cg) {
+        ee_model::ChainGraph fresh;
+        ee_status_t rc = build_chain(m, first_stage, in, (char*)workspace, outs, &fresh);
+        if (rc != EE_OK) return rc;
+        if (m->chains.size() >= 16) {   // bounded: the oldest chain goes once the stream has passed it
+          cudaStreamSynchronize(st);
+          cudaGraphExecDestroy(m->chains.front().exec);
+          cudaGraphDestroy(m->chains.front().graph);
+          m->chains.erase(m->chains.begin());
+        }
+        m->chains.push_back(std::move(fresh));
+        cg = &m->chains.back();
+      }
+      for (int s = first_stage; s + 1 < n_stages; ++s) *(volatile int32_t*)outs[s].n_surv_host = -1;
+      EE_CUDA(cudaGraphLaunch(cg->exec, st));
+      int32_t n = in->batch;
+      for (int s = first_stage; s < n_stages; ++s) {
+        if (batch_per_stage) batch_per_stage[s] = n;
+        if (s + 1 == n_stages) break;
+        ee_status_t rc = ee_wait_count(outs[s].n_surv_host, -1, timeout_s, &n);
+        if (rc != EE_OK) return rc;
+        if (n <= 0) break;
+      }
+      return EE_OK;
+    }
+  }
   ee_stage_in_t cur = *in;
   for (int s = first_stage; s < n_stages; ++s) {
     const bool last = s + 1 == n_stages;
@@ -1118,6 +1293,7 @@ ee_status_t ee_model_set_graphs(ee_model_t* m, int enabled) {
 ee_status_t ee_model_set_branches(ee_model_t* m, int enabled) {
   if (!m) return EE_ERR_INVALID_ARG;
   m->branches = enabled != 0;
+  drop_chains(m);
   for (auto& sp : m->stages) {
     for (auto& g : sp.graphs) sp.retired.push_back(g.exec);
     sp.graphs.clear();
@@ -1129,10 +1305,17 @@ ee_status_t ee_model_set_stage_kernel(ee_model_t* m, int enabled, int max_batch)
   if (!m || max_batch < 0) return EE_ERR_INVALID_ARG;
   m->stage_kernel = enabled != 0;
   m->stage_kernel_max_batch = max_batch == 0 ? (1 << 30) : max_batch;
+  drop_chains(m);
   for (auto& sp : m->stages) {
     for (auto& g : sp.graphs) sp.retired.push_back(g.exec);
     sp.graphs.clear();
   }
+  return EE_OK;
+}
+
+ee_status_t ee_model_set_chain(ee_model_t* m, int max_batch) {
+  if (!m || max_batch < 0) return EE_ERR_INVALID_ARG;
+  m->chain_max_batch = max_batch;
   return EE_OK;
 }
 
@@ -1198,6 +1381,7 @@ ee_status_t ee_model_set_layer_variant(ee_model_t* m, int stage, int layer, int 
   for (int b = batch_lo; b <= batch_hi; ++b) L.variant[b] = (uint8_t)variant;
   for (auto& g : sp.graphs) cudaGraphExecDestroy(g.exec);   // captured stages hold the old choice
   sp.graphs.clear();
+  drop_chains(m);
   return EE_OK;
 }
 
@@ -1216,6 +1400,7 @@ ee_status_t ee_model_set_layer_splits(ee_model_t* m, int stage, int layer, int s
   layout_stage_tail(m, sp);
   for (auto& g : sp.graphs) cudaGraphExecDestroy(g.exec);
   sp.graphs.clear();
+  drop_chains(m);
   return EE_OK;
 }
 

@@ -805,6 +805,46 @@ def test_count_reaches_the_host_without_a_stream_sync():
 
 
 @pytest.mark.parametrize("which", ["tiny", "resnet"])
+def test_device_sized_chain_matches_the_host_sized_chain(which):
+    """ee_run_until_exit as one graph whose switch nodes pick every next stage's batch on the device, against the
+    same call with the host sizing every stage: same batch per stage, and every output of every stage bit for bit.
+    tiny: samples leave at every exit (varying counts, including runs that end early); resnet: nobody leaves early."""
+    spec = wl.tiny_ee_cnn(seed=0) if which == "tiny" else wl.resnet50_ee(seed=1, in_hw=64, n_classes=100, max_batch=8, alphas=[0.01] * 4)
+    run = util.GpuRunner(spec)
+    m, ws = run.m, run.ws
+    bufs_h = [eb.StageBuffers(m, s) for s in range(m.n_stages)]
+    bufs_d = [eb.StageBuffers(m, s) for s in range(m.n_stages)]
+    side = torch.cuda.Stream()
+    seen = set()
+    with torch.cuda.stream(side):
+        for B, seed in ((8, 5), (8, 6), (3, 7), (1, 8), (8, 5)):
+            x = eb.to_device(spec.dtype, wl.make_input(spec, 8, seed=seed))
+            ids = torch.arange(100, 108, dtype=torch.int32, device="cuda")
+            m.set_chain(0)
+            sizes_h = m.run_until_exit(0, x, B, bufs_h, ws, ids)
+            torch.cuda.synchronize()
+            m.set_chain(spec.max_batch)
+            for b in bufs_d:
+                b.exit_mask.fill_(9)
+            sizes_d = m.run_until_exit(0, x, B, bufs_d, ws, ids)
+            torch.cuda.synchronize()
+            m.check()
+            assert sizes_d == sizes_h, (B, seed, sizes_d, sizes_h)
+            seen.add(tuple(sizes_h))
+            for s, n in enumerate(sizes_h):
+                if n == 0:
+                    break
+                h, d = bufs_h[s], bufs_d[s]
+                ns = int(h.n_surv_host[0])
+                assert int(d.n_surv_host[0]) == ns == int(d.n_surv_dev.cpu()[0])
+                assert torch.equal(d.exit_mask[:n], h.exit_mask[:n]) and torch.equal(d.pred[:n], h.pred[:n]) and torch.equal(d.conf[:n], h.conf[:n])
+                assert torch.equal(d.logits[:n], h.logits[:n]) and torch.equal(d.survivor_idx[:ns], h.survivor_idx[:ns])
+                assert torch.equal(d.ids_out[:ns], h.ids_out[:ns]) and torch.equal(d.features_out[:ns], h.features_out[:ns])
+    assert len(seen) >= (3 if which == "tiny" else 2)
+    run.check_guards()
+
+
+@pytest.mark.parametrize("which", ["tiny", "resnet"])
 def test_run_until_exit_matches_the_stage_by_stage_loop(which):
     """ee_run_until_exit chains the stages inside the library; it must leave exactly what a caller's own loop of
     ee_stage_run + count read-back leaves: same batch per stage, same masks, predictions, ids and survivors.
