@@ -54,6 +54,19 @@ template <> struct Vec16<bf16> {
   }
 };
 
+// Accumulator type of the CUDA-core kernels: the fp32 model sums in fp64 (products of two floats are exact in a double,
+// so a sum is rounded once, to fp32, at the store: the 1e-5 parity bar then holds for every element, however small
+// against its tensor); bf16 models sum in fp32 (their bar is the bf16 rounding of the result).
+template <typename T> struct Accum { typedef float type; };
+template <> struct Accum<float> { typedef double type; };
+__device__ __forceinline__ float acc_fma(float a, float b, float c) { return fmaf(a, b, c); }
+__device__ __forceinline__ double acc_fma(float a, float b, double c) { return fma((double)a, (double)b, c); }
+__device__ __forceinline__ double apply_act(double v, int act) {
+  if (act == EE_ACT_RELU) return fmax(v, 0.0);
+  if (act == EE_ACT_RELU6) return fmin(fmax(v, 0.0), 6.0);
+  return v;
+}
+
 __device__ __forceinline__ float apply_act(float v, int act) {
   if (act == EE_ACT_RELU) return fmaxf(v, 0.f);
   if (act == EE_ACT_RELU6) return fminf(fmaxf(v, 0.f), 6.f);

@@ -3,8 +3,8 @@
 //
 // The convolution is the product of the implicit Toeplitz matrix A [M = B*Ho*Wo][K = kh*kw*Cin]
 // with the weight matrix W [N = Cout][K] (paper Section II-C); A is never materialised.
-// Every output sums its K terms in ascending k with fp32 FMAs, independent of the batch size,
-// so a sample's result does not depend on which batch it rides in.
+// Every output sums its K terms in ascending k (fp32 FMAs for bf16 models, fp64 for the fp32 model: see Accum),
+// independent of the batch size, so a sample's result does not depend on which batch it rides in.
 #pragma once
 #include "common.cuh"
 
@@ -50,11 +50,12 @@ conv_igemm_simt_kernel(const T* __restrict__ x, const T* __restrict__ w, const f
   }
 
   const int tx = t & 15, ty = t >> 4;
-  float acc[4][4];
+  typedef typename Accum<T>::type A;
+  A acc[4][4];
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int j = 0; j < 4; ++j) acc[i][j] = (A)0;
 
   for (int k0 = 0; k0 < K; k0 += kSimtBK) {
     const int k = k0 + kk;
@@ -89,7 +90,7 @@ conv_igemm_simt_kernel(const T* __restrict__ x, const T* __restrict__ w, const f
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        for (int j = 0; j < 4; ++j) acc[i][j] = acc_fma(av[i], bv[j], acc[i][j]);
     }
     __syncthreads();
   }
@@ -102,9 +103,9 @@ conv_igemm_simt_kernel(const T* __restrict__ x, const T* __restrict__ w, const f
     for (int j = 0; j < 4; ++j) {
       const int n = n0 + tx * 4 + j;
       if (n >= N) continue;
-      float v = fmaf(scale ? scale[n] : 1.f, acc[i][j], bias ? bias[n] : 0.f);
-      if (residual) v += Elem<T>::ld(residual + m * N + n);
-      Elem<T>::st(y + m * N + n, apply_act(v, g.act));
+      A v = (A)(scale ? scale[n] : 1.f) * acc[i][j] + (A)(bias ? bias[n] : 0.f);   // float: one FMA; double: exact product, one add
+      if (residual) v += (A)Elem<T>::ld(residual + m * N + n);
+      Elem<T>::st(y + m * N + n, (float)apply_act(v, g.act));
     }
   }
 }
@@ -124,9 +125,10 @@ dwconv_kernel(const T* __restrict__ x, const T* __restrict__ w, const float* __r
     p /= g.Wo;
     const int ho = (int)(p % g.Ho);
     const long b = p / g.Ho;
-    float acc[VEC];
+    typedef typename Accum<T>::type A;
+    A acc[VEC];
 #pragma unroll
-    for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+    for (int e = 0; e < VEC; ++e) acc[e] = (A)0;
     for (int r = 0; r < g.kh; ++r) {
       const int hi = ho * g.stride - g.pad + r;
       if (hi < 0 || hi >= g.H) continue;
@@ -138,9 +140,9 @@ dwconv_kernel(const T* __restrict__ x, const T* __restrict__ w, const float* __r
           Vec16<T> xv;
           xv.load(xp);
 #pragma unroll
-          for (int e = 0; e < VEC; ++e) acc[e] = fmaf(xv.v[e], Elem<T>::ld(w + ((long)(c + e) * g.kh + r) * g.kw + s), acc[e]);
+          for (int e = 0; e < VEC; ++e) acc[e] = acc_fma(xv.v[e], Elem<T>::ld(w + ((long)(c + e) * g.kh + r) * g.kw + s), acc[e]);
         } else {
-          acc[0] = fmaf(Elem<T>::ld(xp), Elem<T>::ld(w + ((long)c * g.kh + r) * g.kw + s), acc[0]);
+          acc[0] = acc_fma(Elem<T>::ld(xp), Elem<T>::ld(w + ((long)c * g.kh + r) * g.kw + s), acc[0]);
         }
       }
     }
@@ -148,10 +150,11 @@ dwconv_kernel(const T* __restrict__ x, const T* __restrict__ w, const float* __r
     if constexpr (VEC > 1) {
       Vec16<T> o;
 #pragma unroll
-      for (int e = 0; e < VEC; ++e) o.v[e] = apply_act(fmaf(scale ? scale[c + e] : 1.f, acc[e], bias ? bias[c + e] : 0.f), g.act);
+      for (int e = 0; e < VEC; ++e)
+        o.v[e] = (float)apply_act((A)(scale ? scale[c + e] : 1.f) * acc[e] + (A)(bias ? bias[c + e] : 0.f), g.act);
       o.store(yp);
     } else {
-      Elem<T>::st(yp, apply_act(fmaf(scale ? scale[c] : 1.f, acc[0], bias ? bias[c] : 0.f), g.act));
+      Elem<T>::st(yp, (float)apply_act((A)(scale ? scale[c] : 1.f) * acc[0] + (A)(bias ? bias[c] : 0.f), g.act));
     }
   }
 }

@@ -30,7 +30,8 @@ template <typename T, int VEC>
 __global__ void __launch_bounds__(kGapThreads)
 gap_kernel(const T* __restrict__ x, int HW, int C, int lanes, float* __restrict__ gap, unsigned* __restrict__ zero_me, int n_zero,
            int rev) {
-  __shared__ float red[kGapThreads * VEC];
+  typedef typename Accum<T>::type A;   // fp64 sums for the fp32 model
+  __shared__ A red[kGapThreads * VEC];
   const int tid = threadIdx.x, b = rev ? (int)(gridDim.y - 1 - blockIdx.y) : (int)blockIdx.y;   // rev: last sample first
   const int cv = C / VEC;
   const int groups = kGapThreads / lanes;
@@ -40,9 +41,9 @@ gap_kernel(const T* __restrict__ x, int HW, int C, int lanes, float* __restrict_
   pdl_launch_dependents();
   if (blockIdx.x == 0 && blockIdx.y == 0)
     for (int i = tid; i < n_zero; i += kGapThreads) zero_me[i] = 0u;
-  float acc[VEC];
+  A acc[VEC];
 #pragma unroll
-  for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+  for (int e = 0; e < VEC; ++e) acc[e] = (A)0;
   if (v < cv) {
     const T* p0 = x + (size_t)b * HW * C + (size_t)v * VEC;
     int r = grp;
@@ -75,9 +76,9 @@ gap_kernel(const T* __restrict__ x, int HW, int C, int lanes, float* __restrict_
   if (tid < lanes * VEC) {
     const int c = blockIdx.x * lanes * VEC + tid;   // red[q][lv][e] with lv * VEC + e == tid
     if (c < cv * VEC) {
-      float sum = 0.f;
+      A sum = (A)0;
       for (int q = 0; q < groups; ++q) sum += red[q * lanes * VEC + tid];
-      gap[(size_t)b * C + c] = sum * (1.0f / (float)HW);
+      gap[(size_t)b * C + c] = (float)(sum / (A)HW);
     }
   }
 }
@@ -275,11 +276,12 @@ fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float*
 
   pdl_wait();
   pdl_launch_dependents();
-  float acc[kFcClassesPerWarp][S];
+  typedef typename Accum<T>::type A;   // fp64 sums for the fp32 model
+  A acc[kFcClassesPerWarp][S];
 #pragma unroll
   for (int q = 0; q < kFcClassesPerWarp; ++q)
 #pragma unroll
-    for (int s2 = 0; s2 < S; ++s2) acc[q][s2] = 0.f;
+    for (int s2 = 0; s2 < S; ++s2) acc[q][s2] = (A)0;
   if constexpr (ALIGNED) {
 #pragma unroll
     for (int s0 = 0; s0 < STAGES - 1; ++s0) {
@@ -312,7 +314,7 @@ fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float*
 #pragma unroll
       for (int q = 0; q < kFcClassesPerWarp; ++q)
 #pragma unroll
-        for (int e = 0; e < PER; ++e) acc[q][s2] = fmaf(wv[q][e], gv[e], acc[q][s2]);
+        for (int e = 0; e < PER; ++e) acc[q][s2] = acc_fma(wv[q][e], gv[e], acc[q][s2]);
     }
   }
 #pragma unroll
@@ -321,10 +323,10 @@ fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float*
     const float bk = (bfc && k < K) ? bfc[k] : 0.f;
 #pragma unroll
     for (int s2 = 0; s2 < S; ++s2) {
-      float v = acc[q][s2];
+      A v = acc[q][s2];
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      if (lane == 0 && k < K && b0 + s2 < B) z[(size_t)(b0 + s2) * K + k] = v + bk;
+      if (lane == 0 && k < K && b0 + s2 < B) z[(size_t)(b0 + s2) * K + k] = (float)(v + (A)bk);
     }
   }
   __threadfence();
