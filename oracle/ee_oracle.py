@@ -50,6 +50,8 @@ def lib():
         L.eo_round_bf16.argtypes = [C.c_double]
         L.eo_conv2d.argtypes = [fp, C.c_int, C.c_int, C.c_int, C.c_int, fp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                 C.c_int, fp, fp, fp, C.c_int, C.c_int, fp]
+        L.eo_conv2d_hw.argtypes = [fp, C.c_int, C.c_int, C.c_int, C.c_int, fp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                   C.c_int, fp, fp, fp, C.c_int, C.c_int, fp]
         L.eo_maxpool.argtypes = [fp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, fp]
         L.eo_exit_head.argtypes = [fp, C.c_int, C.c_int, C.c_int, fp, fp, C.c_int, fp, ip, C.c_float, C.c_int,
                                    dp, dp, dp, ip, up]
@@ -83,17 +85,19 @@ def round_bf16(v: float) -> float:
 OP_CONV, OP_DWCONV, OP_MAXPOOL = 0, 1, 2
 
 
-def conv2d(x, w, stride=1, pad=0, groups=1, scale=None, bias=None, residual=None, act=0, bf16=False):
+def conv2d(x, w, stride=1, pad=0, groups=1, scale=None, bias=None, residual=None, act=0, bf16=False, pad_w=None):
+    """``pad`` pads the rows and, unless ``pad_w`` is given, the columns too."""
     x = _c32(x); w = _c32(w); scale = _c32(scale); bias = _c32(bias); residual = _c32(residual)
     B, H, W, Cin = x.shape
     Cout, kh, kw, cpg = w.shape
     assert cpg * groups == Cin
-    Ho, Wo = (H + 2 * pad - kh) // stride + 1, (W + 2 * pad - kw) // stride + 1
+    pad_w = pad if pad_w is None or pad_w < 0 else pad_w
+    Ho, Wo = (H + 2 * pad - kh) // stride + 1, (W + 2 * pad_w - kw) // stride + 1
     y = np.empty((B, Ho, Wo, Cout), dtype=np.float32)
     if B == 0:
         return y
-    rc = lib().eo_conv2d(_f(x), B, H, W, Cin, _f(w), Cout, kh, kw, stride, pad, groups, _f(scale), _f(bias),
-                         _f(residual), act, 1 if bf16 else 0, _f(y))
+    rc = lib().eo_conv2d_hw(_f(x), B, H, W, Cin, _f(w), Cout, kh, kw, stride, pad, pad_w, groups, _f(scale), _f(bias),
+                            _f(residual), act, 1 if bf16 else 0, _f(y))
     assert rc == 0
     return y
 
@@ -179,7 +183,7 @@ def run_layers(model, stage: int, x, keep_all: bool = False):
         elif l.residual_from >= 0:
             res = outs[l.residual_from]
         groups = l.cin if l.op == OP_DWCONV else 1
-        outs.append(conv2d(src, l.weight, l.stride, l.pad, groups, l.scale, l.bias, res, l.act, bf16))
+        outs.append(conv2d(src, l.weight, l.stride, l.pad, groups, l.scale, l.bias, res, l.act, bf16, getattr(l, "pad_w", None)))
     return outs if keep_all else outs[st.out_layer]
 
 

@@ -52,14 +52,16 @@ static double eo_round(double v, int mode) {
     return mode == EO_ROUND_BF16 ? eo_round_bf16(v) : (double)(float)v;
 }
 
-/* y[b,ho,wo,co] = act(scale[co] * sum_{r,s,ci} x[b, ho*st-pad+r, wo*st-pad+s, g*cpg+ci] * w[co,r,s,ci]
- *                     + bias[co] + residual[b,ho,wo,co]),  rounded once to the storage type. */
-int eo_conv2d(const float* x, int B, int H, int W, int Cin,
-              const float* w, int Cout, int kh, int kw, int stride, int pad, int groups,
-              const float* scale, const float* bias, const float* residual, int act, int rounding,
-              float* y) {
+/* y[b,ho,wo,co] = act(scale[co] * sum_{r,s,ci} x[b, ho*st-pad_h+r, wo*st-pad_w+s, g*cpg+ci] * w[co,r,s,ci]
+ *                     + bias[co] + residual[b,ho,wo,co]),  rounded once to the storage type.
+ * Padding per axis: the factorised 1x7 / 7x1 convolutions of the paper's second benchmark network (Section IV,
+ * Benchmarks: Inception-v3) keep the map size by padding only the axis the filter extends along. */
+int eo_conv2d_hw(const float* x, int B, int H, int W, int Cin,
+                 const float* w, int Cout, int kh, int kw, int stride, int pad_h, int pad_w, int groups,
+                 const float* scale, const float* bias, const float* residual, int act, int rounding,
+                 float* y) {
     if (groups < 1 || Cin % groups || Cout % groups) return 1;
-    const int Ho = (H + 2 * pad - kh) / stride + 1, Wo = (W + 2 * pad - kw) / stride + 1;
+    const int Ho = (H + 2 * pad_h - kh) / stride + 1, Wo = (W + 2 * pad_w - kw) / stride + 1;
     const int cpg = Cin / groups, opg = Cout / groups;
     if (Ho < 1 || Wo < 1) return 1;
     const long rows = (long)B * Ho;
@@ -71,10 +73,10 @@ int eo_conv2d(const float* x, int B, int H, int W, int Cin,
                 const int g = co / opg;
                 double acc = 0.0;
                 for (int r = 0; r < kh; ++r) {
-                    const int hi = ho * stride - pad + r;
+                    const int hi = ho * stride - pad_h + r;
                     if (hi < 0 || hi >= H) continue;
                     for (int s = 0; s < kw; ++s) {
-                        const int wi = wo * stride - pad + s;
+                        const int wi = wo * stride - pad_w + s;
                         if (wi < 0 || wi >= W) continue;
                         const float* xp = x + (((size_t)b * H + hi) * W + wi) * Cin + (size_t)g * cpg;
                         const float* wp = w + (((size_t)co * kh + r) * kw + s) * cpg;
@@ -91,6 +93,14 @@ int eo_conv2d(const float* x, int B, int H, int W, int Cin,
         }
     }
     return 0;
+}
+
+/* The same padding on both axes. */
+int eo_conv2d(const float* x, int B, int H, int W, int Cin,
+              const float* w, int Cout, int kh, int kw, int stride, int pad, int groups,
+              const float* scale, const float* bias, const float* residual, int act, int rounding,
+              float* y) {
+    return eo_conv2d_hw(x, B, H, W, Cin, w, Cout, kh, kw, stride, pad, pad, groups, scale, bias, residual, act, rounding, y);
 }
 
 /* Window maximum over the taps that fall inside the image. */

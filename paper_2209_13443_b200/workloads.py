@@ -72,6 +72,7 @@ class Layer:
     weight: Optional[np.ndarray] = None   # [cout][kh][kw][cin/groups]; None for maxpool
     scale: Optional[np.ndarray] = None    # [cout] folded-BN scale
     bias: Optional[np.ndarray] = None     # [cout] folded-BN bias
+    pad_w: int = -1                       # padding of the columns; -1 = the same as ``pad`` (which pads the rows)
 
     @property
     def groups(self) -> int:
@@ -102,7 +103,8 @@ class Model:
 
 
 def out_hw(h: int, w: int, l: Layer):
-    return (h + 2 * l.pad - l.kh) // l.stride + 1, (w + 2 * l.pad - l.kw) // l.stride + 1
+    pw = l.pad if l.pad_w < 0 else l.pad_w
+    return (h + 2 * l.pad - l.kh) // l.stride + 1, (w + 2 * pw - l.kw) // l.stride + 1
 
 
 def stage_shapes(model: Model):
@@ -144,6 +146,18 @@ def _conv(rng, op, cin, cout, k, stride, pad, act, *, gamma=1.0, jitter=True, bf
     if bf16:
         w = to_bf16_grid(w)
     return Layer(op, cin, cout, k, k, stride, pad, act, input_from, residual_from, w, scale, bias)
+
+
+def _conv_hw(rng, cin, cout, kh, kw, stride, pad_h, pad_w, act, *, gamma=1.0, bf16=False, input_from=FROM_PREV,
+             residual_from=NO_RESIDUAL) -> Layer:
+    """A dense convolution with a kh x kw filter and per-axis padding (the factorised 1 x n / n x 1 filters of
+    Inception-style towers)."""
+    w = rng.standard_normal((cout, kh, kw, cin), dtype=np.float32) * np.float32(np.sqrt(2.0 / (kh * kw * cin)))
+    scale = (gamma * rng.uniform(0.8, 1.2, size=cout)).astype(np.float32)
+    bias = (0.05 * rng.standard_normal(cout)).astype(np.float32)
+    if bf16:
+        w = to_bf16_grid(w)
+    return Layer(OP_CONV, cin, cout, kh, kw, stride, pad_h, act, input_from, residual_from, w, scale, bias, pad_w)
 
 
 def head_weights(seed: int, stream: int, c: int, n_classes: int, alpha: float, bf16: bool):
@@ -308,6 +322,41 @@ def benchmark_model(workload: str, max_batch: int, flat_heads: bool = False):
     if workload == "tiny":
         return tiny_ee_cnn(seed=0, max_batch=max_batch), 0
     raise ValueError(f"unknown workload {workload}")
+
+
+def factorised_tower_ee(seed: int = 5, max_batch: int = 32, in_hw: int = 68, width: int = 192, n_classes: int = 1000,
+                        blocks=(2, 2), dtype: str = "bf16", alphas=None, threshold: float = 0.6) -> Model:
+    """A backbone in the shape of the 17 x 17 towers of Inception-v3 (the paper's second benchmark network, Section IV):
+    a strided 3x3 stem pair brings the image to in_hw / 4, then every stage is a run of residual blocks
+    1x1 -> 1x7 -> 7x1 -> 1x1 (+ block input), the 1 x 7 and 7 x 1 filters padded only along their own axis.  The
+    branches of the original (concatenated towers, pooled branch) are not modelled: this workload exists for the
+    asymmetric filters.  Exit heads (GAP + FC) after every stage, the last one always taken."""
+    bf16 = dtype == "bf16"
+    alphas = alphas or [6.0] * len(blocks)
+    stages = []
+    cin = 3
+    for s, nb in enumerate(blocks):
+        rng = _rng(seed, 400 + s)
+        layers: List[Layer] = []
+        idx = FROM_STAGE_INPUT
+        if s == 0:
+            layers.append(_conv(rng, OP_CONV, 3, 32, 3, 2, 1, ACT_RELU, bf16=bf16))
+            layers.append(_conv(rng, OP_CONV, 32, width, 3, 2, 1, ACT_RELU, bf16=bf16))
+            idx, cin = 1, width
+        elif cin != width << s:
+            layers.append(_conv(rng, OP_CONV, cin, width << s, 1, 2, 0, ACT_RELU, bf16=bf16, input_from=idx))
+            idx, cin = len(layers) - 1, width << s
+        mid = cin // 2
+        for _ in range(nb):
+            layers.append(_conv_hw(rng, cin, mid, 1, 1, 1, 0, 0, ACT_RELU, bf16=bf16, input_from=idx))
+            layers.append(_conv_hw(rng, mid, mid, 1, 7, 1, 0, 3, ACT_RELU, bf16=bf16))
+            layers.append(_conv_hw(rng, mid, mid, 7, 1, 1, 3, 0, ACT_RELU, bf16=bf16))
+            layers.append(_conv_hw(rng, mid, cin, 1, 1, 1, 0, 0, ACT_RELU, gamma=0.3, bf16=bf16, residual_from=idx))
+            idx = len(layers) - 1
+        last = s == len(blocks) - 1
+        fw, fb = head_weights(seed, 400 + s, cin, n_classes, alphas[s], bf16)
+        stages.append(Stage(layers, n_classes, fw, fb, 1.0 if last else threshold, last))
+    return Model("factorised_tower_ee", dtype, in_hw, in_hw, 3, stages, max_batch, {"seed": seed})
 
 
 # ----------------------------------------------------------------------------- inputs

@@ -143,6 +143,28 @@ def test_conv_matches_torch_fp64(groups, stride, pad, k):
         np.testing.assert_allclose(got, fn(ref).numpy(), rtol=2e-7, atol=1e-6)
 
 
+@pytest.mark.parametrize("kh,kw,ph,pw,stride", [(1, 7, 0, 3, 1), (7, 1, 3, 0, 1), (3, 5, 1, 2, 2), (1, 3, 0, 0, 1), (5, 1, 0, 0, 2)])
+def test_conv_with_per_axis_padding_matches_torch_fp64_and_closed_forms(kh, kw, ph, pw, stride):
+    """Filters that are not square and pad only along their own axis (the factorised 1 x 7 / 7 x 1 convolutions of
+    Inception-v3, Section IV Benchmarks): torch fp64 with padding=(ph, pw), and an all-ones closed form that tells the
+    axes apart (a transposed pad or filter changes the count of in-range taps at the borders)."""
+    rng = np.random.default_rng(kh * 10 + kw)
+    x = rng.standard_normal((2, 9, 11, 4)).astype(np.float32)
+    w = rng.standard_normal((3, kh, kw, 4)).astype(np.float32)
+    got = eo.conv2d(x, w, stride, ph, pad_w=pw)
+    ref = F.conv2d(torch.from_numpy(x).double().permute(0, 3, 1, 2), torch.from_numpy(w).double().permute(0, 3, 1, 2),
+                   stride=stride, padding=(ph, pw)).permute(0, 2, 3, 1).numpy()
+    assert got.shape == ref.shape
+    np.testing.assert_allclose(got, ref, rtol=2e-7, atol=1e-6)
+    ones = eo.conv2d(np.ones((1, 9, 11, 2), np.float32), np.ones((1, kh, kw, 2), np.float32), 1, ph, pad_w=pw)
+    rows_in = lambda c, n, k, p: sum(0 <= c - p + t < n for t in range(k))     # noqa: E731
+    for (ho, wo) in [(0, 0), (0, ones.shape[2] - 1), (ones.shape[1] - 1, 0), (ones.shape[1] // 2, ones.shape[2] // 2)]:
+        assert ones[0, ho, wo, 0] == 2 * rows_in(ho, 9, kh, ph) * rows_in(wo, 11, kw, pw)
+    # pad_w left out or negative: the same padding on both axes, i.e. the square-padding routine
+    if kh == kw:
+        np.testing.assert_array_equal(eo.conv2d(x, w, stride, ph), eo.conv2d(x, w, stride, ph, pad_w=ph))
+
+
 def test_epilogue_order_and_bf16_store():
     # residual is added BEFORE the activation; ReLU6 clamps at 6; the store rounds once to bf16
     x = np.array([[[[1.0]]]], np.float32)
