@@ -57,6 +57,7 @@ typedef enum { EE_ACT_NONE = 0, EE_ACT_RELU = 1, EE_ACT_RELU6 = 2 } ee_act_t;
 #define EE_FROM_PREV (-1)         /* input_from: output of the previous layer (stage input for layer 0) */
 #define EE_FROM_STAGE_INPUT (-2)  /* the stage's input tensor */
 #define EE_NO_RESIDUAL (-1)       /* residual_from: no residual operand */
+#define EE_PAD_W_SAME (-1)        /* pad_w: the columns are padded like the rows */
 
 /* One layer of a stage.  y = act(scale[c] * conv(x, weight) + bias[c] (+ residual)), stored in
  * the model dtype with one round-to-nearest-even.  BN is folded into scale/bias by the caller.
@@ -71,6 +72,9 @@ typedef struct {
   const void* weight; /* HOST or DEVICE (see ee_model_desc_t.weights_on_device); copied at create */
   const float* scale; /* [cout] fp32, may be NULL (= 1) */
   const float* bias;  /* [cout] fp32, may be NULL (= 0) */
+  int pad_w;          /* padding of the columns; EE_PAD_W_SAME (-1): `pad` pads rows and columns alike, otherwise `pad`
+                         pads the rows only (filters that are not square, such as 1 x 7 and 7 x 1, pad along their own
+                         axis); dense convolutions only */
 } ee_layer_desc_t;
 
 /* One stage = a subnet followed by its exit head (global average pool, one FC layer, softmax;

@@ -35,7 +35,7 @@ class EEError(RuntimeError):
 class LayerDesc(C.Structure):
     _fields_ = [("op", C.c_int), ("cin", C.c_int), ("cout", C.c_int), ("kh", C.c_int), ("kw", C.c_int), ("stride", C.c_int),
                 ("pad", C.c_int), ("act", C.c_int), ("input_from", C.c_int), ("residual_from", C.c_int),
-                ("weight", C.c_void_p), ("scale", C.c_void_p), ("bias", C.c_void_p)]
+                ("weight", C.c_void_p), ("scale", C.c_void_p), ("bias", C.c_void_p), ("pad_w", C.c_int)]
 
 
 class StageDesc(C.Structure):
@@ -208,7 +208,7 @@ class EEModel:
             self._keep.append(layers)
             for li, l in enumerate(st.layers):
                 layers[li] = LayerDesc(l.op, l.cin, l.cout, l.kh, l.kw, l.stride, l.pad, l.act, l.input_from, l.residual_from,
-                                       host(l.weight, True), host(l.scale, False), host(l.bias, False))
+                                       host(l.weight, True), host(l.scale, False), host(l.bias, False), int(getattr(l, "pad_w", -1)))
             stage_structs[si] = StageDesc(len(st.layers), layers, st.out_layer, st.n_classes, host(st.fc_weight, True),
                                           host(st.fc_bias, False), float(st.threshold), int(bool(st.always_exit)))
         desc = ModelDesc(1 if self.dtype == "bf16" else 0, spec.in_h, spec.in_w, spec.in_c, self.n_stages, stage_structs,

@@ -221,7 +221,7 @@ void layout_stage_tail(ee_model* m, StagePlan& sp) {
 template <typename T>
 ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const void* res, void* dst, int B, float* partial,
                          size_t partial_bytes, cudaStream_t st) {
-  ConvGeom g{B, L.in_h, L.in_w, L.d.cin, L.out_h, L.out_w, L.d.cout, L.d.kh, L.d.kw, L.d.stride, L.d.pad, L.d.act};
+  ConvGeom g{B, L.in_h, L.in_w, L.d.cin, L.out_h, L.out_w, L.d.cout, L.d.kh, L.d.kw, L.d.stride, L.d.pad, L.d.pad_w, L.d.act};
   constexpr int V = Elem<T>::kVec;
   switch (L.kind) {
     case KK_SIMT: {
@@ -698,6 +698,9 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
       const ee_layer_desc_t& d = sd.layers[i];
       LayerPlan& L = sp.layers[i];
       L.d = d;
+      if (d.pad_w < EE_PAD_W_SAME) return fail(EE_ERR_INVALID_ARG);
+      if (L.d.pad_w == EE_PAD_W_SAME) L.d.pad_w = d.pad;              // from here on pad = rows, pad_w = columns
+      if (d.op != EE_OP_CONV && L.d.pad_w != d.pad) return fail(EE_ERR_UNSUPPORTED);
       if (d.op < EE_OP_CONV || d.op > EE_OP_MAXPOOL || d.kh < 1 || d.kw < 1 || d.stride < 1 || d.pad < 0 || d.cin < 1 ||
           d.cout < 1 || d.act < EE_ACT_NONE || d.act > EE_ACT_RELU6 || d.input_from < EE_FROM_STAGE_INPUT ||
           d.input_from >= i || d.residual_from < EE_FROM_STAGE_INPUT || d.residual_from >= i)
@@ -716,8 +719,8 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
       L.in_h = ih;
       L.in_w = iw;
       L.out_h = (ih + 2 * d.pad - d.kh) / d.stride + 1;
-      L.out_w = (iw + 2 * d.pad - d.kw) / d.stride + 1;
-      if (ih + 2 * d.pad < d.kh || iw + 2 * d.pad < d.kw || L.out_h < 1 || L.out_w < 1) return fail(EE_ERR_SHAPE);
+      L.out_w = (iw + 2 * L.d.pad_w - d.kw) / d.stride + 1;
+      if (ih + 2 * d.pad < d.kh || iw + 2 * L.d.pad_w < d.kw || L.out_h < 1 || L.out_w < 1) return fail(EE_ERR_SHAPE);
       oh[i] = L.out_h, ow[i] = L.out_w, oc[i] = d.cout;
       L.src_slot = src;  // layer index for now; mapped to slots below
       int rs = d.residual_from;
@@ -879,7 +882,7 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
         }
         if (rc != EE_OK) return fail(rc);
         L.tc.halo = halo_supported(d, L.in_w);
-      } else if (desc->dtype == EE_BF16 && d.cout % 8 == 0 && d.kh * d.kw * d.cin <= 1024) {
+      } else if (desc->dtype == EE_BF16 && d.cout % 8 == 0 && d.kh * d.kw * d.cin <= 1024 && d.pad_w == d.pad) {
         // pixel rows are not 16-byte units (e.g. a 3-channel stem): explicit Toeplitz rows, then the tensor-core GEMM
         L.kind = KK_TC_GATHER;
         const bool stem7 = stem_supported(d, L.in_h, L.in_w, L.out_w) && d.residual_from == EE_NO_RESIDUAL;
@@ -895,7 +898,7 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
           pack_weights_kernel<<<cdiv((long)d.cout * kp, 256), 256, 0, st>>>((const bf16*)L.w_dev, (bf16*)wp, d.cout, d.kh, run, runp, kp);
         if (cudaGetLastError() != cudaSuccess) return fail(EE_ERR_CUDA);
         ee_layer_desc_t g = d;   // the GEMM view: a 1x1 layer over kp packed columns
-        g.cin = kp, g.kh = g.kw = 1, g.stride = 1, g.pad = 0;
+        g.cin = kp, g.kh = g.kw = 1, g.stride = 1, g.pad = g.pad_w = 0;
         rc = tc_plan_layer(m->tc, g, L.out_h, L.out_w, L.out_h, L.out_w, desc->max_batch, wp, &L.tc);
         if (rc != EE_OK) return fail(rc);
         L.tc.gather = true;

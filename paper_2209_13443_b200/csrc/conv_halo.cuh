@@ -209,7 +209,7 @@ conv3x3_halo_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
 // output channels, no residual operand, and an image row short enough that a ring slot holds 128 positions plus the
 // two rows and two pixels the last tap reaches past them.
 inline bool halo_supported(const ee_layer_desc_t& d, int in_w) {
-  return d.op == EE_OP_CONV && d.kh == 3 && d.kw == 3 && d.stride == 1 && d.pad == 1 && d.cin == 64 && d.cout <= 64 && d.cout % 8 == 0 &&
+  return d.op == EE_OP_CONV && d.kh == 3 && d.kw == 3 && d.stride == 1 && d.pad == 1 && d.pad_w == 1 && d.cin == 64 && d.cout <= 64 && d.cout % 8 == 0 &&
          d.residual_from == EE_NO_RESIDUAL && kTcBM + 2 * (in_w + 2) + 2 <= kHaloBlockRows;
 }
 

@@ -34,7 +34,7 @@ struct PairParams {
   int M, N;             // valid rows (B*Ho*Wo) and Cout
   int taps, kw;         // kh*kw and kw
   int cblocks;          // ceil(Cin / 64)
-  int Ho, Wo, stride, pad;
+  int Ho, Wo, stride, pad, pad_w;
   int im2col;           // 0: A is a plain [rows][Cin] matrix, 1: im2col tensor map
   int act;
   int has_res;
@@ -260,7 +260,7 @@ conv_igemm_tcgen05_pair_kernel(const __grid_constant__ PairStageArgs A) {
             cn = m0 / hw;
             const int rem = m0 - cn * hw;
             const int ho = rem / p.Wo;
-            cw = (rem - ho * p.Wo) * p.stride - p.pad;
+            cw = (rem - ho * p.Wo) * p.stride - p.pad_w;
             ch = ho * p.stride - p.pad;
           }
           auto arm_and_load_w = [&](int kb, int gg) -> bool {
@@ -614,7 +614,7 @@ inline ee_status_t pair_fill_layer(TcContext& c, const TcLayer& L, int bn, const
   p.taps = L.kh * L.kw;
   p.kw = L.kw;
   p.cblocks = cdiv(L.cin, kTcBK);
-  p.Ho = L.out_h, p.Wo = L.out_w, p.stride = L.stride, p.pad = L.pad;
+  p.Ho = L.out_h, p.Wo = L.out_w, p.stride = L.stride, p.pad = L.pad, p.pad_w = L.pad_w;
   p.im2col = L.im2col ? 1 : 0;
   p.act = L.act;
   p.has_res = res ? 1 : 0;

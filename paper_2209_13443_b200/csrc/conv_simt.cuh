@@ -11,7 +11,7 @@
 namespace ee {
 
 struct ConvGeom {
-  int B, H, W, Cin, Ho, Wo, Cout, kh, kw, stride, pad, act;
+  int B, H, W, Cin, Ho, Wo, Cout, kh, kw, stride, pad, pad_w, act;   // pad: rows, pad_w: columns (equal except for dense convolutions)
 };
 
 constexpr int kSimtBM = 64, kSimtBN = 64, kSimtBK = 16, kSimtThreads = 256, kSimtPad = 4;
@@ -42,7 +42,7 @@ conv_igemm_simt_kernel(const T* __restrict__ x, const T* __restrict__ w, const f
       const long b = q / g.Ho;
       a_base[i] = b * g.H * g.W;
       a_hi0[i] = ho * g.stride - g.pad;
-      a_wi0[i] = wo * g.stride - g.pad;
+      a_wi0[i] = wo * g.stride - g.pad_w;
     } else {
       a_base[i] = -1;
       a_hi0[i] = a_wi0[i] = 0;

@@ -288,7 +288,7 @@ __global__ void pack_stem_weights_kernel(const bf16* __restrict__ w, bf16* __res
 
 inline bool stem_supported(const ee_layer_desc_t& d, int in_h, int in_w, int out_w) {
   (void)in_h;
-  return d.op == EE_OP_CONV && d.cin == kStemCin && d.kh == kStemKh && d.kw == kStemKw && d.stride == kStemStride && d.pad == kStemPad &&
+  return d.op == EE_OP_CONV && d.cin == kStemCin && d.kh == kStemKh && d.kw == kStemKw && d.stride == kStemStride && d.pad == kStemPad && d.pad_w == kStemPad &&
          d.cout % 8 == 0 && d.cout <= 64 && in_w % 8 == 0 && out_w <= kStemMaxWo;
 }
 

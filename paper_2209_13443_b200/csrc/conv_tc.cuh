@@ -37,7 +37,7 @@ struct TcParams {
   int M, N;             // valid rows (B*Ho*Wo) and Cout
   int taps, kw;         // kh*kw and kw
   int cblocks;          // ceil(Cin / 64); the TMA unit zero-fills channels past Cin in both operands
-  int Ho, Wo, stride, pad;
+  int Ho, Wo, stride, pad, pad_w;   // pad: rows, pad_w: columns
   int im2col;           // 0: A is a plain [rows][Cin] matrix, 1: im2col tensor map
   int act;
   const float* scale;
@@ -446,7 +446,7 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
         cn = m0 / hw;
         const int rem = m0 - cn * hw;
         const int ho = rem / p.Wo;
-        cw = (rem - ho * p.Wo) * p.stride - p.pad;
+        cw = (rem - ho * p.Wo) * p.stride - p.pad_w;
         ch = ho * p.stride - p.pad;
       }
       for (int i = 0; i < num_kb; ++i) {
@@ -767,7 +767,7 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
           cn = m0 / hw;
           const int rem = m0 - cn * hw;
           const int ho = rem / p.Wo;
-          cw = (rem - ho * p.Wo) * p.stride - p.pad;
+          cw = (rem - ho * p.Wo) * p.stride - p.pad_w;
           ch = ho * p.stride - p.pad;
         }
         for (int kb = 0; kb < num_kb; ++kb, ++g) {
@@ -932,7 +932,7 @@ __global__ void replicate_kernel(const float* __restrict__ src, float* __restric
 // Pixels per row for a 1x1 / stride 1 / pad 0 layer on hw pixels per sample: the largest g with g * Cin <= 64 that
 // divides hw (so no row straddles two samples); 1 = leave the layer as it is.
 inline int pixel_group(const ee_layer_desc_t& d, int hw) {
-  if (!(d.kh == 1 && d.kw == 1 && d.stride == 1 && d.pad == 0) || d.cin > 32) return 1;
+  if (!(d.kh == 1 && d.kw == 1 && d.stride == 1 && d.pad == 0 && d.pad_w == 0) || d.cin > 32) return 1;
   int g = kTcBK / d.cin;
   while (g > 1 && hw % g != 0) --g;
   return g;
@@ -965,7 +965,7 @@ struct TcContext {
 };
 
 struct TcLayer {
-  int cin = 0, cout = 0, kh = 1, kw = 1, stride = 1, pad = 0, act = 0;
+  int cin = 0, cout = 0, kh = 1, kw = 1, stride = 1, pad = 0, pad_w = 0, act = 0;
   int in_h = 0, in_w = 0, out_h = 0, out_w = 0, max_batch = 0;
   int bn = 128;
   bool im2col = false;
@@ -1033,16 +1033,16 @@ inline ee_status_t tc_context_init(TcContext& c) {
 inline bool tc_supported(const ee_layer_desc_t& d, int in_h, int in_w) {
   (void)in_h;
   (void)in_w;
-  return d.op == EE_OP_CONV && d.cin % 8 == 0 && d.cout % 8 == 0 && d.kh == d.kw && d.kh <= 7 && d.stride <= 8 &&
-         d.pad < d.kh && d.pad <= 127;
+  return d.op == EE_OP_CONV && d.cin % 8 == 0 && d.cout % 8 == 0 && d.kh <= 7 && d.kw <= 7 && d.stride <= 8 &&
+         d.pad < d.kh && d.pad_w < d.kw;   // filters need not be square: the im2col map takes one corner pair per axis
 }
 
 inline ee_status_t tc_plan_layer(TcContext& c, const ee_layer_desc_t& d, int in_h, int in_w, int out_h, int out_w, int max_batch,
                                  const void* w_dev, TcLayer* L) {
-  L->cin = d.cin, L->cout = d.cout, L->kh = d.kh, L->kw = d.kw, L->stride = d.stride, L->pad = d.pad, L->act = d.act;
+  L->cin = d.cin, L->cout = d.cout, L->kh = d.kh, L->kw = d.kw, L->stride = d.stride, L->pad = d.pad, L->pad_w = d.pad_w, L->act = d.act;
   L->in_h = in_h, L->in_w = in_w, L->out_h = out_h, L->out_w = out_w, L->max_batch = max_batch;
   L->bn = d.cout > 64 ? 128 : 64;
-  L->im2col = !(d.kh == 1 && d.stride == 1 && d.pad == 0);
+  L->im2col = !(d.kh == 1 && d.kw == 1 && d.stride == 1 && d.pad == 0 && d.pad_w == 0);
   // Split-K: a lone CTA cannot pull operands faster than its SM's L2 port (about 126 GB/s: a 32 KB K block of a
   // 128x128 tile takes 0.26 us in tile mode and 0.36 us in im2col mode, against 0.13 us of MMA time), so a layer
   // whose grid leaves SMs idle spreads the K range of a tile over a cluster of 2..4 CTAs.  A split costs about
@@ -1159,8 +1159,8 @@ inline ee_status_t tc_buffer_map(const TcContext& c, const TcLayer& L, const voi
     // NHWC as (C, W, H, N).  Base pixels (filter tap 0,0) range over [-pad, dim - 1 + pad - (k - 1)] in steps of `stride`.
     const cuuint64_t dims[4] = {(cuuint64_t)L.cin, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)batch};
     const cuuint64_t strides[3] = {(cuuint64_t)L.cin * 2, (cuuint64_t)L.cin * 2 * L.in_w, (cuuint64_t)L.cin * 2 * L.in_w * L.in_h};
-    const int lower[2] = {-L.pad, -L.pad};
-    const int upper[2] = {L.pad - (L.kw - 1), L.pad - (L.kh - 1)};
+    const int lower[2] = {-L.pad_w, -L.pad};                                 // (W, H) corners
+    const int upper[2] = {L.pad_w - (L.kw - 1), L.pad - (L.kh - 1)};
     const cuuint32_t es[4] = {1, (cuuint32_t)L.stride, (cuuint32_t)L.stride, 1};
     r = c.encode_im2col(&e.tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, lower, upper, kTcBK,
                         kTcBM, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1261,7 +1261,7 @@ inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, co
   p.taps = L.kh * L.kw;
   p.kw = L.kw;
   p.cblocks = cdiv(L.cin, kTcBK);
-  p.Ho = L.out_h, p.Wo = L.out_w, p.stride = L.stride, p.pad = L.pad;
+  p.Ho = L.out_h, p.Wo = L.out_w, p.stride = L.stride, p.pad = L.pad, p.pad_w = L.pad_w;
   p.im2col = L.im2col ? 1 : 0;
   p.act = L.act;
   p.scale = scale, p.bias = bias;
@@ -1273,7 +1273,7 @@ inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, co
   p.rev = L.rev ? 1 : 0;
   p.gx = (const bf16*)src;
   p.gH = L.g_h, p.gW = L.g_w, p.gCin = L.g_cin, p.gkh = L.g_kh, p.grun = L.g_kw * L.g_cin, p.grunp = L.g_runp;
-  if (L.gather) p.stride = L.g_stride, p.pad = L.g_pad;
+  if (L.gather) p.stride = L.g_stride, p.pad = p.pad_w = L.g_pad;
   dim3 grid(cdiv(p.M, kTcBM), cdiv(L.cout, L.bn), split ? L.splits : 1);
   // At most one CTA per SM anyway: take the deep operand ring.  A cluster grid close to the SM count does not: its
   // clusters need all their CTAs inside one GPC, a 192 KB CTA owns its SM, and the last clusters then wait for a second

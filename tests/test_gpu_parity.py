@@ -240,6 +240,50 @@ def test_maxpool_layer(dtype):
     assert np.array_equal(g["features_out"], o["features_out"])
 
 
+# filters that are not square, padded along their own axis (the factorised convolutions of Inception-style towers)
+ASYM_GEOMS = [
+    # H, W, cin, cout, kh, kw, stride, pad_h, pad_w, act, variant
+    (17, 17, 96, 96, 1, 7, 1, 0, 3, wl.ACT_RELU, 0),
+    (17, 17, 96, 96, 7, 1, 1, 3, 0, wl.ACT_RELU, 0),
+    (13, 9, 24, 40, 3, 5, 2, 1, 2, wl.ACT_RELU6, 0),
+    (9, 12, 16, 32, 1, 3, 1, 0, 0, wl.ACT_NONE, 0),          # no padding: the map shrinks along one axis only
+    (17, 17, 192, 192, 1, 7, 1, 0, 3, wl.ACT_RELU, 1),        # the same on the CTA-pair kernel
+    (17, 17, 192, 192, 7, 1, 1, 3, 0, wl.ACT_RELU, 2),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("geom", ASYM_GEOMS)
+def test_conv_layer_with_a_filter_that_is_not_square(dtype, geom):
+    H, W, cin, cout, kh, kw, stride, ph, pw, act, variant = geom
+    if dtype == "f32" and variant:
+        pytest.skip("the CTA-pair kernel is a bf16 kernel")
+    bf16 = dtype == "bf16"
+    rng = wl._rng(hash(geom) % 1000, 904)
+    layer = wl._conv_hw(rng, cin, cout, kh, kw, stride, ph, pw, act, bf16=bf16)
+    fw, fb = wl._head(rng, cout, 7, 1.0, bf16)
+    spec = wl.Model("asym", dtype, H, W, cin, [wl.Stage([layer], 7, fw, fb, 2.0, False)], 5)
+
+    def configure(m):
+        if variant:
+            m.set_layer_splits(0, 0, 2)
+            m.set_layer_variant(0, 0, 1, 5, variant)
+
+    run = util.GpuRunner(spec, configure)
+    for B in (1, 5):
+        x = wl.random_features((B, H, W, cin), seed=B, bf16=bf16, relu=False)
+        o = util.oracle_stage(spec, 0, x)
+        g = run.stage(0, x)
+        assert g["features_out"].shape == o["features_out"].shape
+        util.check_stage(spec, g, o, f"{dtype} {geom} B={B}", elementwise=True)
+
+
+@pytest.mark.parametrize("B", [1, 4])
+def test_factorised_tower_shaped_small(B):
+    spec = wl.factorised_tower_ee(seed=5, in_hw=36, width=64, n_classes=50, max_batch=4)
+    _stagewise(spec, B, seed=5)
+
+
 # ----------------------------------------------------------------------------- configs 2-3 at reduced size
 
 def _stagewise(spec, B, seed, tol=None):
