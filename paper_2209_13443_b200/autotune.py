@@ -3,14 +3,20 @@
 The paper's design-space exploration picks, offline, the configuration that maximises a throughput objective
 summed over the batch sizes the device will see (Section III-D, Eq. 2) and stores the per-(layer, batch) choice in a
 look-up table the hardware addresses at run time (Section III-C).  This script is the counterpart for the kernels
-of this library: for every tensor-core layer it times every kernel variant (one-CTA tiles, CTA pairs with 256- or
-128-wide tiles) for every candidate number of K ranges and every batch size on the GPU at hand, picks the number
-of K ranges per layer that minimises sum_b w_b T(b) with every batch taking its fastest variant (the K ranges must not
-depend on the batch: they fix the grouping of the sums), then the variant per (layer, batch), and writes the table as JSON:
+of this library.  Everything is timed IN CONTEXT: the quantity measured is the device time of a whole ee_stage_run
+(replayed back to back as a CUDA graph), because a kernel's choice also moves the time of its neighbours (a CTA-pair
+kernel owns its SMs' shared memory, so the kernels before and after it cannot overlap with it); timing layers alone
+picked variants that made the stages slower.
 
-  python -m paper_2209_13443_b200.autotune --workload resnet50 --max-batch 64 [--out FILE] [--raw FILE]
+  phase 1, K ranges:  for every tensor-core layer, greedily, the number of K ranges (1, 2, 3, 4, 6, 8; one value per
+                      layer for all batch sizes, because the ranges fix the grouping of every sum) that minimises
+                      sum_b w_b T_stage(b) over a few batch sizes, all layers on the one-CTA kernels;
+  phase 2, variants:  for every measured batch size and every layer, greedily, the kernel variant (0 one-CTA tiles,
+                      1 CTA pairs 256 x 256, 2 CTA pairs 256 x 128) that lowers the stage's time by more than 3 %, twice.
 
-``EEModel`` applies a table written for (workload, max_batch) at creation (see ``binding.apply_table``).
+  python -m paper_2209_13443_b200.autotune --workload resnet50 --max-batch 64 [--out FILE]
+
+``EEModel`` applies a table written for (workload, input, max_batch) at creation (see ``binding.apply_table``).
 """
 from __future__ import annotations
 
@@ -22,125 +28,122 @@ import torch
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 SPLITS = (1, 2, 3, 4, 6, 8)
-VARIANTS = (0, 1, 2)
+VARIANTS = (1, 2)
 
 
 def table_path(name: str, max_batch: int) -> str:
     return os.path.join(HERE, "tables", f"{name}_b{max_batch}.json")
 
 
-def layer_shapes(spec):
-    from . import workloads as wl
+class StageTimer:
+    """Device time of ee_stage_run for one stage at a batch: `reps` runs captured into one CUDA graph, best of `rounds`."""
 
-    return wl.stage_shapes(spec)
+    def __init__(self, m, spec, reps=8, rounds=3):
+        from . import binding as eb
+
+        self.m, self.spec, self.reps, self.rounds = m, spec, reps, rounds
+        self.bufs = [eb.StageBuffers(m, s, with_logits=False) for s in range(m.n_stages)]
+        self.ws = m.workspace()
+        self.x = []
+        td = eb.torch_dtype(spec.dtype)
+        for s in range(m.n_stages):
+            q = m.query(s)
+            self.x.append((torch.randn(spec.max_batch, q["in_h"], q["in_w"], q["in_c"], device="cuda") * 0.5).to(td))
+
+    def ensure_workspace(self):
+        need = max(self.m.query(s)["workspace_bytes"] for s in range(self.m.n_stages))
+        if self.ws.numel() < need + 256:
+            self.ws = torch.empty(need + 256, dtype=torch.uint8, device="cuda")
+
+    def time(self, s, B) -> float:
+        self.ensure_workspace()
+        st = torch.cuda.current_stream()
+        m = self.m
+        m.stage_run(s, self.x[s], B, self.bufs[s], self.ws)      # tensor maps cached before the capture
+        st.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            for _ in range(self.reps):
+                m.stage_run(s, self.x[s], B, self.bufs[s], self.ws)
+        best = float("inf")
+        for _ in range(self.rounds + 1):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            g.replay()
+            b.record()
+            b.synchronize()
+            best = min(best, a.elapsed_time(b) * 1e3 / self.reps)
+        m.check()          # a device-side fault stops the sweep here, not minutes later
+        return best
 
 
-def time_layer(m, s, i, x, res, out, B, ws, reps=20, rounds=3):
-    """Device time (us) of one launch of a layer: `reps` back-to-back launches replayed as one CUDA graph (so that the
-    host's launch cost does not bound the measurement), best of `rounds` replays."""
-    st = torch.cuda.current_stream()
-    m.layer_run(s, i, x, res, B, out, ws)           # tensor maps cached, lazy module loading done before the capture
-    st.synchronize()
-    g = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(g, stream=st):
-        for _ in range(reps):
-            m.layer_run(s, i, x, res, B, out, ws)
-    best = float("inf")
-    for _ in range(rounds + 1):
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        g.replay()
-        b.record()
-        b.synchronize()
-        best = min(best, a.elapsed_time(b) * 1e3 / reps)
-    return best
-
-
-def measure(spec, batches, verbose=True):
+def tune(spec, batches, split_batches, verbose=True):
     from . import binding as eb
-    from . import workloads as wl
 
     m = eb.EEModel(spec, apply_tables=False)
     m.set_wait_limit(200_000_000)       # a wait that runs out should cost 0.1 s, not seconds, per launch of a sweep
-    shapes = layer_shapes(spec)
-    rows = []
-    ws = m.workspace()
+    timer = StageTimer(m, spec)
+    layers = []                          # (stage, layer, support mask, default K ranges)
+    for s, st in enumerate(spec.stages):
+        for i in range(len(st.layers)):
+            cfg = m.layer_config(s, i, 1)
+            if cfg["tensor_core"] >= 0:
+                layers.append((s, i, cfg["tensor_core"], cfg["splits"]))
     side = torch.cuda.Stream()
+    table = {(s, i): {"splits": d, "variants": {}} for s, i, _, d in layers}
+    log = []
     with torch.cuda.stream(side):
-        for s, st in enumerate(spec.stages):
-            sh = shapes[s]
-            for i, l in enumerate(st.layers):
-                cfg = m.layer_config(s, i, 1)
-                if cfg["tensor_core"] < 0:
+        # phase 1: K ranges, one-CTA kernels, objective sum over split_batches of the stage's time
+        for s, i, _, default in layers:
+            def cost():
+                return sum(timer.time(s, b) for b in split_batches)
+            best_sp, best_cost = default, cost()
+            for sp in SPLITS:
+                if sp == default or sp > 4:          # the cluster reduce-scatter of the one-CTA kernel takes up to four ranges
                     continue
-                src = l.input_from
-                ishape = sh["in"] if (src == wl.FROM_STAGE_INPUT or (src == wl.FROM_PREV and i == 0)) else sh["layers"][i - 1 if src == wl.FROM_PREV else src]
-                oshape = sh["layers"][i]
-                default_splits = cfg["splits"]
-                for sp in SPLITS:
-                    try:
-                        m.set_layer_splits(s, i, sp)
-                    except eb.EEError:
-                        continue
-                    need = m.query(s)["workspace_bytes"]
-                    if ws.numel() < need + 256:
-                        ws = torch.empty(need + 256, dtype=torch.uint8, device="cuda")
-                    for B in batches:
-                        x = torch.randn((B,) + tuple(ishape), device="cuda").to(torch.bfloat16)
-                        res = torch.randn((B,) + tuple(oshape), device="cuda").to(torch.bfloat16) if l.residual_from != wl.NO_RESIDUAL else None
-                        out = torch.empty((B,) + tuple(oshape), dtype=torch.bfloat16, device="cuda")
-                        for v in VARIANTS:
-                            if v > 0 and not (cfg["tensor_core"] >> (v - 1)) & 1:
-                                continue
-                            if v == 0 and sp > 4:
-                                continue       # cluster split-K of the one-CTA kernel: up to four ranges
-                            m.set_layer_variant(s, i, 1, spec.max_batch, v)
-                            us = time_layer(m, s, i, x, res, out, B, ws)
-                            m.check()          # a device-side fault stops the sweep here, not minutes later
-                            rows.append({"stage": s, "layer": i, "splits": sp, "batch": B, "variant": v, "us": us,
-                                         "default_splits": default_splits,
-                                         "geom": [l.kh, l.cin, l.cout, l.stride, oshape[0], oshape[1]]})
-                    m.check()
-                    if verbose:
-                        last = [r for r in rows if r["stage"] == s and r["layer"] == i and r["splits"] == sp]
-                        print(f"stage {s} layer {i} {l.kh}x{l.kw} {l.cin}->{l.cout} splits {sp}: " +
-                              " ".join(f"B{r['batch']}v{r['variant']}={r['us']:.1f}" for r in last), flush=True)
-                m.set_layer_splits(s, i, default_splits)
-                m.set_layer_variant(s, i, 1, spec.max_batch, 0)
-    return rows
-
-
-def choose(rows, max_batch, weights=None):
-    """Per layer: the number of K ranges minimising sum_b w_b min_v T(b, splits, v); then the variant per batch
-    (measured batches are extended to the batches between them: batch b takes the choice of the nearest measured
-    batch at or above it)."""
-    layers = {}
-    for r in rows:
-        layers.setdefault((r["stage"], r["layer"]), []).append(r)
-    table = []
-    for (s, i), rs in sorted(layers.items()):
-        batches = sorted({r["batch"] for r in rs})
-        best_sp, best_cost = None, float("inf")
-        for sp in sorted({r["splits"] for r in rs}):
-            cost = 0.0
-            for b in batches:
-                ts = [r["us"] for r in rs if r["splits"] == sp and r["batch"] == b]
-                if not ts:
-                    cost = float("inf")
-                    break
-                cost += (weights or {}).get(b, 1.0) * min(ts)
-            if cost < best_cost:
-                best_sp, best_cost = sp, cost
-        per_b = {}
-        for b in batches:
-            cand = [(r["us"], r["variant"]) for r in rs if r["splits"] == best_sp and r["batch"] == b]
-            per_b[b] = min(cand)[1]
+                try:
+                    m.set_layer_splits(s, i, sp)
+                except eb.EEError:
+                    continue
+                c = cost()
+                if c < best_cost * 0.98 and cost() < best_cost * 0.98:              # a gain has to show twice
+                    best_sp, best_cost = sp, c
+            m.set_layer_splits(s, i, best_sp)
+            table[(s, i)]["splits"] = best_sp
+            log.append({"phase": "splits", "stage": s, "layer": i, "default": default, "chosen": best_sp, "cost_us": best_cost})
+            if verbose:
+                print(f"stage {s} layer {i}: K ranges {default} -> {best_sp} (sum of stage times {best_cost:.1f} us)", flush=True)
+        # phase 2: variants per batch
+        for s in range(m.n_stages):
+            mine = [(i, mask) for ss, i, mask, _ in layers if ss == s and mask]
+            for B in batches:
+                base = timer.time(s, B)
+                for i, mask in mine:
+                    pick = 0
+                    for v in VARIANTS:
+                        if not (mask >> (v - 1)) & 1:
+                            continue
+                        m.set_layer_variant(s, i, B, B, v)
+                        t = timer.time(s, B)
+                        if t < base * 0.97 and timer.time(s, B) < base * 0.97:     # a gain has to show twice
+                            base, pick = t, v
+                    m.set_layer_variant(s, i, B, B, pick)
+                    table[(s, i)]["variants"][B] = pick
+                log.append({"phase": "variants", "stage": s, "batch": B, "stage_us": base,
+                            "pairs": [i for i, _ in mine if table[(s, i)]["variants"].get(B)]})
+                if verbose:
+                    print(f"stage {s} batch {B}: {base:.1f} us, pair kernel on layers {log[-1]['pairs']}", flush=True)
+    out = []
+    for s, i, _, _ in layers:
+        l = spec.stages[s].layers[i]
+        per_b = table[(s, i)]["variants"]
         variants = []
-        for b in range(1, max_batch + 1):
+        for b in range(1, spec.max_batch + 1):     # a batch between two measured ones takes the choice of the next measured batch above it
             nb = min([x for x in batches if x >= b] or [batches[-1]])
-            variants.append(per_b[nb])
-        table.append({"stage": s, "layer": i, "splits": best_sp, "variants": variants, "geom": rs[0]["geom"]})
-    return table
+            variants.append(per_b.get(nb, 0))
+        out.append({"stage": s, "layer": i, "splits": table[(s, i)]["splits"], "variants": variants,
+                    "geom": [l.kh, l.cin, l.cout, l.stride]})
+    return out, log
 
 
 def main():
@@ -151,19 +154,21 @@ def main():
     ap.add_argument("--max-batch", type=int, default=64)
     ap.add_argument("--batches", default="")
     ap.add_argument("--out", default=None)
-    ap.add_argument("--raw", default=None)
+    ap.add_argument("--log", default=None)
     args = ap.parse_args()
     spec, _ = wl.benchmark_model(args.workload, args.max_batch)
     if args.batches:
         batches = [int(b) for b in args.batches.split(",")]
     else:
-        batches = sorted({b for b in (1, 2, 3, 4, 6, 8, 12, 16, 24, 32, 48, 64, 96, 128) if b < args.max_batch} | {args.max_batch})
-    rows = measure(spec, batches)
-    if args.raw:
-        with open(args.raw, "w") as f:
-            json.dump(rows, f)
-    table = {"workload": spec.name, "max_batch": args.max_batch, "input": [spec.in_h, spec.in_w, spec.in_c], "gpu": torch.cuda.get_device_name(0), "batches_measured": batches,
-             "layers": choose(rows, args.max_batch)}
+        batches = sorted({b for b in (1, 2, 3, 4, 6, 8, 12, 16, 20, 24, 28, 32, 40, 48, 56, 64, 96, 128) if b < args.max_batch} | {args.max_batch})
+    mb = args.max_batch
+    split_batches = sorted({1, max(1, mb // 16), max(1, mb // 4), max(1, mb // 2), mb})
+    layers, log = tune(spec, batches, split_batches)
+    if args.log:
+        with open(args.log, "w") as f:
+            json.dump(log, f)
+    table = {"workload": spec.name, "max_batch": args.max_batch, "input": [spec.in_h, spec.in_w, spec.in_c], "gpu": torch.cuda.get_device_name(0),
+             "batches_measured": batches, "split_batches": split_batches, "layers": layers}
     out = args.out or table_path(spec.name, args.max_batch)
     os.makedirs(os.path.dirname(out), exist_ok=True)
     with open(out, "w") as f:
