@@ -362,7 +362,7 @@ def run_ours(args):
         for s in range(nst):
             run_stage(s, feat, n, ids)
             stream.synchronize()
-            plan = model.plan(s, n)
+            plan = [pl for pl in model.plan(s, n) if pl["launches"] > 0]   # a layer fused into its predecessor has no launch
             tm = model.get_timing(s)
             for i, (name, ms) in enumerate(tm):
                 f = fam.setdefault(name, {"ms": 0.0, "launches": 0, "flops": 0.0, "bytes": 0.0})

@@ -244,7 +244,8 @@ ee_status_t ee_model_set_stage_kernel(ee_model_t* model, int enabled, int max_ba
 
 /* Per-layer device timing.  When enabled, ee_stage_run brackets every kernel with CUDA events on the
  * stream it launches on.  ee_model_get_timing synchronises those events and writes, for the last run
- * of `stage`, up to `cap` entries: the layers in order, then the head and the gather kernels.
+ * of `stage`, up to `cap` entries: the layers that launch a kernel (ee_layer_plan_t.launches > 0) in order, then the
+ * head and the gather kernels.
  * names[i] points at a static string.  Errors: INVALID_ARG, STAGE, CUDA. */
 ee_status_t ee_model_set_timing(ee_model_t* model, int enabled);
 ee_status_t ee_model_get_timing(ee_model_t* model, int stage, int cap, float* ms, const char** names, int* n);
@@ -255,7 +256,9 @@ typedef struct {
   const char* kernel;
   int m, n, k;
   double flops, bytes;
-  int launches; /* kernels this layer launches at this batch size */
+  int launches; /* kernels this layer launches at this batch size; 0: an earlier layer's launch does its work (a layer
+                 * inside a multi-layer launch; a 3x3 stride-2 pad-1 max-pool read only from the 7x7 stride-2 3-channel
+                 * bf16 convolution right before it, which pools in its epilogue and never stores its own output) */
 } ee_layer_plan_t;
 ee_status_t ee_model_plan(const ee_model_t* model, int stage, int batch, int cap, ee_layer_plan_t* out, int* n);
 

@@ -54,6 +54,10 @@ struct LayerPlan {
   std::vector<uint8_t> variant;
   // Branch execution: a layer whose output is only ever a residual operand (the projection shortcut of a block) does
   // not depend on the layers between its input and its consumer, so it runs on a side stream beside them.
+  // A stem convolution read only by the 3x3 stride-2 pad-1 max-pool right behind it takes that pool into its epilogue
+  // inside ee_stage_run (the convolution's own output is then never written); ee_layer_run still runs either alone.
+  bool pool_next = false;     // this layer's launch also does the pooling of the next layer
+  bool fused_away = false;    // this (pooling) layer's work is done by the launch of the layer before it
   bool side = false;          // runs on the model's branch stream
   int wait_for = -1;          // layer index of a side layer whose result this layer consumes
   cudaEvent_t ev_fork = nullptr, ev_done = nullptr;
@@ -220,7 +224,7 @@ void layout_stage_tail(ee_model* m, StagePlan& sp) {
 
 template <typename T>
 ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const void* res, void* dst, int B, float* partial,
-                         size_t partial_bytes, cudaStream_t st) {
+                         size_t partial_bytes, cudaStream_t st, bool fuse_pool = false) {
   ConvGeom g{B, L.in_h, L.in_w, L.d.cin, L.out_h, L.out_w, L.d.cout, L.d.kh, L.d.kw, L.d.stride, L.d.pad, L.d.pad_w, L.d.act};
   constexpr int V = Elem<T>::kVec;
   switch (L.kind) {
@@ -246,7 +250,7 @@ ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const
     }
     case KK_TC_GATHER: {
       if constexpr (sizeof(T) == 2) {
-        ee_status_t s = L.tc.stem7 ? stem_launch(m->tc, L.tc, src, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st)
+        ee_status_t s = L.tc.stem7 ? stem_launch(m->tc, L.tc, src, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st, fuse_pool)
                                    : tc_launch(m->tc, L.tc, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st);
         if (s != EE_OK) return s;
       } else {
@@ -417,9 +421,10 @@ ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, c
     }
     const size_t i = m->timing ? k : (size_t)sp.order[k];
     const LayerPlan& L = sp.layers[i];
+    if (L.fused_away) continue;   // the launch of the convolution before it pools as well
     const void* src = L.src_slot < 0 ? in->features : ws + sp.slot_off[L.src_slot];
     const void* res = L.res_slot == -2 ? nullptr : (L.res_slot == -1 ? in->features : ws + sp.slot_off[L.res_slot]);
-    void* dst = ws + sp.slot_off[L.out_slot];
+    void* dst = ws + sp.slot_off[L.pool_next ? sp.layers[i + 1].out_slot : L.out_slot];
     float* partial = (float*)(ws + sp.split_off);
     cudaStream_t ls = st;
     if (par && L.side) {            // fork: everything enqueued so far (the producer of this layer's input) precedes it
@@ -428,7 +433,7 @@ ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, c
       ls = m->branch;
     }
     if (par && L.wait_for >= 0) EE_CUDA(cudaStreamWaitEvent(st, sp.layers[L.wait_for].ev_done, 0));   // join
-    ee_status_t s = m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, src, res, dst, B, partial, sp.split_bytes, ls)
+    ee_status_t s = m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, src, res, dst, B, partial, sp.split_bytes, ls, L.pool_next)
                                         : launch_layer<float>(m, L, src, res, dst, B, partial, sp.split_bytes, ls);
     if (s != EE_OK) return s;
     if (par && L.side) EE_CUDA(cudaEventRecord(L.ev_done, m->branch));
@@ -910,6 +915,15 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
         L.kind = KK_SIMT;
       }
     }
+    for (int i = 0; i + 1 < sd.n_layers; ++i) {
+      LayerPlan& L = sp.layers[i];
+      LayerPlan& P = sp.layers[i + 1];
+      if (L.kind != KK_TC_GATHER || !L.tc.stem7 || !stem_pool_supported(P.d) || i == out_layer) continue;
+      if (src_of[i + 1] != i || n_in_use[i] != 1 || n_res_use[i] != 0) continue;   // someone else reads the convolution's output
+      if (L.src_slot >= 0 && L.src_slot == P.out_slot) continue;                  // the pooled tensor would overwrite the input
+      L.pool_next = true;
+      P.fused_away = true;
+    }
     // Layer runs for the multi-layer launch: consecutive positions of the execution order whose layers the CTA-pair kernel
     // covers with one tile width (256 columns if every layer has more than 128 filters, else 128).
     {
@@ -1364,6 +1378,11 @@ ee_status_t ee_model_plan(const ee_model_t* m, int stage, int batch, int cap, ee
     const double w_b = L.d.op == EE_OP_MAXPOOL ? 0.0 : (double)L.d.cout * p.k * es;
     p.bytes = in_b + out_b + w_b + (L.res_slot != -2 ? out_b : 0.0);
     p.launches = 1;
+    if (L.pool_next) {   // the launch writes the pooled tensor instead of the convolution's output
+      const LayerPlan& P = sp.layers[i + 1];
+      p.bytes = in_b + w_b + (double)batch * P.out_h * P.out_w * P.d.cout * es;
+    }
+    if (L.fused_away) p.bytes = 0.0, p.launches = 0;   // done by the launch of the convolution before it
   }
   if (stage_kernel_active(m, sp, batch))   // a run of layers is one launch: its first layer carries it
     for (const auto& seg : sp.segments)

@@ -1139,6 +1139,16 @@ inline ee_status_t tc_buffer_map(const TcContext& c, const TcLayer& L, const voi
     r = c.encode_tiled(&e.tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else if (kind == 5) {
+    // stem output behind its fused 3x3 stride-2 pad-1 max-pool, as (Cout, Wp, B*Hp): a store is up to 32 pixels of a pooled row
+    const int hp = (L.out_h - 1) / 2 + 1, wp = (L.out_w - 1) / 2 + 1;
+    const cuuint64_t dims[3] = {(cuuint64_t)L.cout, (cuuint64_t)wp, (cuuint64_t)batch * hp};
+    const cuuint64_t strides[2] = {(cuuint64_t)L.cout * 2, (cuuint64_t)L.cout * 2 * wp};
+    const cuuint32_t box[3] = {64, 32, 1};
+    const cuuint32_t es[3] = {1, 1, 1};
+    r = c.encode_tiled(&e.tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else if (kind == 1) {
     const cuuint64_t dims[2] = {(cuuint64_t)L.cout, (cuuint64_t)batch * L.out_h * L.out_w};
     const cuuint64_t strides[1] = {(cuuint64_t)L.cout * 2};

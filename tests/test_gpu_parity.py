@@ -789,6 +789,46 @@ def test_branch_execution_of_shortcut_layers_is_bit_identical():
     m.check()
 
 
+STEM_POOL_CASES = [  # (H, W, cout, act, B): even and odd output heights and widths, rows past the tile, row ranges across images
+    (224, 224, 64, wl.ACT_RELU, 3), (222, 216, 64, wl.ACT_NONE, 2), (64, 64, 64, wl.ACT_RELU, 7), (30, 40, 32, wl.ACT_RELU6, 5),
+    (18, 8, 64, wl.ACT_NONE, 1), (226, 224, 48, wl.ACT_RELU, 4)]
+
+
+@pytest.mark.parametrize("case", STEM_POOL_CASES)
+def test_stem_with_the_pool_in_its_epilogue_equals_the_two_layers_run_apart(case):
+    """ee_stage_run lets the 7x7/2 stem kernel pool (3x3, stride 2, pad 1) in its epilogue; ee_layer_run runs the
+    convolution and the pooling as two kernels.  The maximum of bf16 values is exact, so the stage's features must
+    equal the two-kernel result bit for bit (and the oracle within the bf16 bar); the plan reports one launch."""
+    H, W, cout, act, B = case
+    rng = wl._rng(11, H, W, cout)
+    layers = [wl._conv(rng, wl.OP_CONV, 3, cout, 7, 2, 3, act, bf16=True), wl.Layer(wl.OP_MAXPOOL, cout, cout, 3, 3, 2, 1)]
+    fw, fb = wl._head(rng, cout, 5, 1.0, True)
+    spec = wl.Model("stem_pool", "bf16", H, W, 3, [wl.Stage(layers, 5, fw, fb, 2.0, False)], 7)
+    run = util.GpuRunner(spec)
+    m, ws, out = run.m, run.ws, run.bufs[0]
+    plan = m.plan(0, B)
+    assert [pl["launches"] for pl in plan] == [1, 0]
+    x = wl.make_input(spec, B, seed=5)
+    xd = eb.to_device("bf16", x)
+    ho, wo = (H - 1) // 2 + 1, (W - 1) // 2 + 1
+    hp, wp = (ho - 1) // 2 + 1, (wo - 1) // 2 + 1
+    conv = torch.empty((B, ho, wo, cout), dtype=torch.bfloat16, device="cuda")
+    apart = torch.empty((B, hp, wp, cout), dtype=torch.bfloat16, device="cuda")
+    m.layer_run(0, 0, xd, None, B, conv, ws)
+    m.layer_run(0, 1, conv, None, B, apart, ws)
+    for graphs in (False, True, True):
+        m.set_graphs(graphs)
+        out.features_out.fill_(0)
+        m.stage_run(0, xd, B, out, ws)
+        torch.cuda.synchronize()
+        m.check()
+        assert int(out.n_surv_host[0]) == B
+        assert torch.equal(out.features_out[:B], apart)
+    run.check_guards()
+    want = eo.run_layers(spec, 0, x)
+    assert util.rel_err(apart.float().cpu().numpy(), want, "bf16") <= util.TOL["bf16"]
+
+
 @pytest.mark.parametrize("B", [1, 3, 7])
 def test_multi_layer_launch_is_bit_identical_to_layer_by_layer(B):
     """Runs of layers executed as one persistent kernel with grid barriers between layers (an option) against the
