@@ -226,6 +226,21 @@ ee_status_t ee_gather_survivors(const void* feat, size_t bytes_per_sample, const
  * Errors: INVALID_ARG. */
 ee_status_t ee_model_set_graphs(ee_model_t* model, int enabled);
 
+/* One-launch exit head.  Off by default.  For bf16 models whose head has C % 8 == 0, C <= 2048 and K <= 1024 (16-byte
+ * aligned features and FC weights) global average pool, FC, softmax top-1, threshold and the survivor scan (Section II-B;
+ * Section III-B steps 2-3) can run as one kernel of 8-CTA thread-block clusters, one cluster per tile of 1, 2 or 4
+ * samples, that exchange the pooled vectors and the softmax partials through distributed shared memory.  Otherwise, and
+ * for other shapes and fp32 models: a pooling kernel and an FC + decision kernel.  Both orders of summation are fixed by
+ * the head's shape, so either way a sample's logits do not depend on its batch; between the two ways logits differ by
+ * the fp32 rounding of differently grouped sums.  Measured on B200 the cluster kernel wins only on large maps at batch 1
+ * (10 us against 14 us at 56x56x256): a cluster per sample tile leaves the pooling with one CTA per SM and eight SMs per
+ * tile to pull the FC weights, where the two kernels spread both over the whole GPU (54 against 32 us at batch 64 on
+ * 56x56x256, 25 against 20 us at batch 27 on 7x7x2048), hence the default.
+ * Applies to ee_stage_run, ee_exit_head and ee_exit_head_static alike.  Errors: INVALID_ARG. */
+ee_status_t ee_model_set_fused_head(ee_model_t* model, int enabled);
+/* Kernels the exit head of `stage` launches on 16-byte aligned features: 1 (one-launch head) or 2; 0 for a bad argument. */
+int ee_model_head_launches(const ee_model_t* model, int stage);
+
 /* Branch execution.  On by default for batches of up to 32 samples: a layer whose output is only a residual operand of a later layer (the projection
  * shortcut of a residual block) runs on a stream of the model's own, beside the layers between its input and its
  * consumer, forked from and joined to the caller's stream by events (also inside captured stages).  Results are

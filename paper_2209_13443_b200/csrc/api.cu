@@ -157,6 +157,8 @@ struct ee_model {
   bool stage_kernel = false;           // run eligible layer runs as one launch (measured slower than per-layer launches: off)
   int stage_kernel_max_batch = 1 << 30;
   size_t pair_counter_words = 0;
+  unsigned* head_done = nullptr;       // one arrival counter per stage for the one-launch exit head; zero between launches
+  bool fused_head = false;             // bf16 models: pool + FC + decision + scan as one cluster kernel where the shape allows (an option)
   long long wait_cycles = kTcWaitCycles;   // limit of the bounded device-side waits of the pair kernel and the self-test
   int device = -1;           // the GPU the model lives on
   bool timing = false;
@@ -310,6 +312,15 @@ ee_status_t launch_head(ee_model* m, StagePlan& sp, const void* x, int B, int hw
   unsigned* cnt = (unsigned*)(scratch + h.off_cnt);
   float* gap = (float*)(scratch + h.off_gap);
   float* z = out->logits ? out->logits : (float*)(scratch + h.off_z);
+  if constexpr (sizeof(T) == 2) {
+    if (m->fused_head && hc_supported(C, K, x, sp.fc_w)) {
+      DecideArgs da{shift, shift_cls, sp.threshold, sp.always_exit, out->conf, out->pred, out->exit_mask,
+                    in_ids ? in_ids->ids : nullptr, out->survivor_idx, out->ids_out, out->n_surv_dev, nullptr, m->head_done + (&sp - m->stages.data())};
+      EE_CUDA(hc_launch((const bf16*)x, hw, C, (const bf16*)sp.fc_w, sp.fc_b, B, K, z, da, st));
+      if (timed) record(m, sp, st, "head_gap_fc_softmax_scan");
+      return EE_OK;
+    }
+  }
   constexpr int V = Elem<T>::kVec;
   const bool vec = C % V == 0 && ((uintptr_t)x & 15) == 0;
   const int lanes = gap_lanes(hw);
@@ -682,6 +693,7 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
   if (rc == EE_OK) rc = halo_context_init();
   if (rc == EE_OK) rc = pair_context_init();
   if (rc == EE_OK) rc = dw_context_init();
+  if (rc == EE_OK && hc_context_init() != cudaSuccess) rc = EE_ERR_CUDA;
   if (rc != EE_OK) return fail(rc);
 
   int h = desc->in_h, w = desc->in_w, c = desc->in_c;
@@ -986,6 +998,13 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
     m->owned.push_back(p);
     m->grid_bar = (unsigned*)p;
     if (cudaMemsetAsync(p, 0, 256, st) != cudaSuccess) return fail(EE_ERR_CUDA);
+  }
+  {
+    void* p = nullptr;
+    if (cudaMalloc(&p, 256 + m->stages.size() * sizeof(unsigned)) != cudaSuccess) return fail(EE_ERR_CUDA);
+    m->owned.push_back(p);
+    m->head_done = (unsigned*)p;
+    if (cudaMemsetAsync(p, 0, 256 + m->stages.size() * sizeof(unsigned), st) != cudaSuccess) return fail(EE_ERR_CUDA);
   }
   if (m->pair_counter_words) {
     void* p = nullptr;
@@ -1307,6 +1326,23 @@ ee_status_t ee_model_set_graphs(ee_model_t* m, int enabled) {
   return EE_OK;
 }
 
+int ee_model_head_launches(const ee_model_t* m, int stage) {
+  if (!m || stage < 0 || stage >= (int)m->stages.size()) return 0;
+  const StagePlan& sp = m->stages[stage];
+  return m->dtype == EE_BF16 && m->fused_head && hc_supported(sp.out_c, sp.n_classes, nullptr, sp.fc_w) ? 1 : 2;
+}
+
+ee_status_t ee_model_set_fused_head(ee_model_t* m, int enabled) {
+  if (!m) return EE_ERR_INVALID_ARG;
+  m->fused_head = enabled != 0;
+  drop_chains(m);
+  for (auto& sp : m->stages) {
+    for (auto& g : sp.graphs) sp.retired.push_back(g.exec);
+    sp.graphs.clear();
+  }
+  return EE_OK;
+}
+
 ee_status_t ee_model_set_branches(ee_model_t* m, int enabled) {
   if (!m) return EE_ERR_INVALID_ARG;
   m->branches = enabled != 0;
@@ -1469,6 +1505,7 @@ ee_status_t ee_model_check(ee_model_t* m, void* cuda_stream) {
     // a kernel that gave up may have left arrival counters of a split-K reduction behind
     if (m->pair_counters) EE_CUDA(cudaMemsetAsync(m->pair_counters, 0, m->pair_counter_words * sizeof(unsigned), st));
     if (m->grid_bar) EE_CUDA(cudaMemsetAsync(m->grid_bar, 0, 256, st));
+    if (m->head_done) EE_CUDA(cudaMemsetAsync(m->head_done, 0, m->stages.size() * sizeof(unsigned), st));
     EE_CUDA(cudaMemsetAsync(m->err_flag, 0, sizeof(int), st));
     EE_CUDA(cudaStreamSynchronize(st));
     return EE_ERR_TIMEOUT;

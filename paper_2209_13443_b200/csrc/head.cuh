@@ -352,6 +352,317 @@ fc_kernel(const float* __restrict__ gap, const T* __restrict__ wfc, const float*
 // Samples per FC tile for a batch.
 inline int fc_tile_samples(int B) { return B <= 16 ? 4 : 8; }
 
+// ----------------------------------------------------------------------------- the whole exit head in one launch
+//
+// bf16 models: global average pool, FC, softmax top-1, threshold and the survivor scan as ONE kernel of 8-CTA
+// clusters, one cluster per tile of S samples (S = 1, 2 or 4 by the batch; no sum depends on S).
+//   1. Pool.  CTA r of a cluster pools the channels [r, r+1) * C/8 of the tile's samples (row groups in ascending order
+//      as in gap_kernel, the grouping a function of C only) and writes its slab of the pooled vectors into the shared
+//      memory of all eight CTAs (distributed shared memory); a cluster barrier publishes them.
+//   2. FC.  CTA r owns the classes [r, r+1) * ceil(K/8).  Their weights stream through a 4-deep cp.async ring of
+//      [64 classes][256 channels] blocks whose first three blocks are requested before the kernel waits for its
+//      predecessor in the stream (the weights are constants).  Warp w takes classes 8w..8w+7 of a block, a lane the
+//      channels 8 lane..8 lane+7: per (sample, class) a lane adds its channels in ascending order over the blocks, then
+//      a shuffle tree, so a logit is the same bits in every batch and at every position.
+//   3. Decision.  Every CTA reduces its classes to (max, lowest argmax, sum of exp(z - max)) per sample and writes the
+//      triple into the leader CTA's shared memory; after a second cluster barrier the leader combines the eight triples in
+//      rank order: conf = 1 / sum_r s_r exp(m_r - m), exit = always || conf >= thr.
+//   4. Scan.  The leader of the cluster that finishes last (one counter per launch, left at zero) runs the stable scan.
+// No wait in this kernel spins: cluster barriers and cp.async groups only.  Launched with programmatic stream
+// serialization.
+constexpr int kHcCluster = 8, kHcThreads = 256, kHcRing = 4, kHcBlockClasses = 64, kHcBlockCh = 256, kHcMaxKc = 128;
+
+__device__ __forceinline__ uint32_t hc_cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t hc_map(const void* smem_ptr, uint32_t rank) {   // the same variable in CTA `rank` of the cluster
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"((uint32_t)__cvta_generic_to_shared(smem_ptr)), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void hc_st_f32(uint32_t cluster_addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void hc_cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void hc_cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+struct HcShape {   // functions of the head's shape (C, K) only
+  int Cp;          // C rounded up to whole 256-channel blocks
+  int cvp;         // 16-byte channel vectors a CTA pools: ceil(C / 8 / 8)
+  int L;           // power of two >= cvp: vectors side by side in the pooling loop (256 / L row groups)
+  int kc;          // classes per CTA: ceil(K / 8)
+  int nchunk;      // channel blocks: Cp / 256
+  int ngroup;      // class blocks of a CTA: ceil(kc / 64)
+};
+inline HcShape hc_shape(int C, int K) {
+  HcShape h;
+  h.Cp = (C + kHcBlockCh - 1) / kHcBlockCh * kHcBlockCh;
+  h.cvp = (C / 8 + kHcCluster - 1) / kHcCluster;
+  h.L = 1;
+  while (h.L < h.cvp) h.L *= 2;
+  h.kc = (K + kHcCluster - 1) / kHcCluster;
+  h.nchunk = h.Cp / kHcBlockCh;
+  h.ngroup = (h.kc + kHcBlockClasses - 1) / kHcBlockClasses;
+  return h;
+}
+inline size_t hc_smem_bytes(int S, const HcShape& h) {
+  return (size_t)S * h.Cp * 4 + (size_t)kHcRing * kHcBlockClasses * kHcBlockCh * 2 + (size_t)S * kHcThreads * 8 * 4 +
+         (size_t)S * kHcMaxKc * 4 + (size_t)kHcCluster * S * 4 * 4 + 16;
+}
+inline int hc_tile_samples(int B) { return B <= 18 ? 1 : B <= 37 ? 2 : 4; }   // up to 18 clusters of 8 fill the 148 SMs
+inline bool hc_supported(int C, int K, const void* x, const void* wfc) {
+  if (C < 8 || C % 8 != 0 || C > 2048 || K < 1 || K > kHcCluster * kHcMaxKc) return false;
+  if (((uintptr_t)x & 15) || ((uintptr_t)wfc & 15)) return false;
+  return hc_shape(C, K).L <= kHcThreads;
+}
+
+template <int S>
+__global__ void __cluster_dims__(kHcCluster, 1, 1) __launch_bounds__(kHcThreads)
+head_cluster_kernel(const bf16* __restrict__ x, int HW, int C, const bf16* __restrict__ wfc, const float* __restrict__ bfc, int B, int K,
+                    float* z, DecideArgs d, HcShape h) {
+  extern __shared__ __align__(16) uint8_t hc_smem[];
+  float* gsm = reinterpret_cast<float*>(hc_smem);                                   // [S][Cp] pooled vectors of the tile
+  bf16* ring = reinterpret_cast<bf16*>(gsm + (size_t)S * h.Cp);                     // [4][64][256]
+  float* red = reinterpret_cast<float*>(ring + (size_t)kHcRing * kHcBlockClasses * kHcBlockCh);   // [S][256][8]
+  float* zs = red + (size_t)S * kHcThreads * 8;                                     // [S][128] this CTA's logits
+  float* part = zs + (size_t)S * kHcMaxKc;                                          // [8][S][4] (leader): max, argmax, sum
+  int* flag = reinterpret_cast<int*>(part + kHcCluster * S * 4);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t rank = hc_cluster_rank();
+  const int tile = (int)blockIdx.x / kHcCluster, b0 = tile * S;
+  const int k0 = (int)rank * h.kc, k1 = min(K, k0 + h.kc), nk = max(k1 - k0, 0);
+  const int T = h.ngroup * h.nchunk;   // ring blocks of this CTA, class block major
+
+  hc_cluster_arrive();   // #1: every CTA of the cluster runs (waited for before the first remote store)
+  auto block_load = [&](int t, int buf) {
+    const int g = t / h.nchunk, ch = t - g * h.nchunk;
+    bf16* dst = ring + (size_t)buf * kHcBlockClasses * kHcBlockCh;
+#pragma unroll
+    for (int i = 0; i < kHcBlockClasses * (kHcBlockCh / 8) / kHcThreads; ++i) {
+      const int idx = tid + i * kHcThreads, row = idx >> 5, c = ch * kHcBlockCh + (idx & 31) * 8;
+      const int k = k0 + g * kHcBlockClasses + row;
+      const bool in = k < k1 && c < C;
+      cp_async16(dst + row * kHcBlockCh + (idx & 31) * 8, in ? wfc + (size_t)k * C + c : wfc, in ? 16 : 0);
+    }
+  };
+#pragma unroll
+  for (int t = 0; t < kHcRing - 1; ++t) {
+    if (t < T) block_load(t, t);
+    cp_async_commit();
+  }
+  for (int i = tid; i < S * (h.Cp - C); i += kHcThreads) gsm[(i / (h.Cp - C)) * h.Cp + C + i % (h.Cp - C)] = 0.f;   // channel padding
+  pdl_wait();
+  pdl_launch_dependents();
+
+  // ---- 1. pool
+  {
+    const int groups = kHcThreads / h.L, grp = tid / h.L, lv = tid - grp * h.L;
+    const int v = (int)rank * h.cvp + lv;
+    const bool mine = lv < h.cvp && v < C / 8;
+#pragma unroll
+    for (int s = 0; s < S; ++s) {
+      float acc[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+      if (mine && b0 + s < B) {
+        const bf16* p0 = x + (size_t)(b0 + s) * HW * C + (size_t)v * 8;
+        int r = grp;
+        for (; r + 15 * groups < HW; r += 16 * groups) {   // sixteen 16-byte loads in flight per thread; added in row order
+          uint4 t[16];
+#pragma unroll
+          for (int u = 0; u < 16; ++u) t[u] = __ldg(reinterpret_cast<const uint4*>(p0 + (size_t)(r + u * groups) * C));
+#pragma unroll
+          for (int u = 0; u < 16; ++u) {
+            const uint32_t w4[4] = {t[u].x, t[u].y, t[u].z, t[u].w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              acc[2 * i] += __uint_as_float(w4[i] << 16);
+              acc[2 * i + 1] += __uint_as_float(w4[i] & 0xffff0000u);
+            }
+          }
+        }
+        for (; r < HW; r += groups) {
+          Vec16<bf16> t;
+          t.load(p0 + (size_t)r * C);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[e] += t.v[e];
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) red[((size_t)s * kHcThreads + grp * h.L + lv) * 8 + e] = acc[e];
+    }
+    __syncthreads();
+    hc_cluster_wait();   // #1
+    if (tid < h.L * 8) {
+      const int lv2 = tid >> 3, c = ((int)rank * h.cvp + lv2) * 8 + (tid & 7);
+      if (lv2 < h.cvp && c < C) {
+#pragma unroll
+        for (int s = 0; s < S; ++s) {
+          float sum = 0.f;
+          for (int q = 0; q < groups; ++q) sum += red[((size_t)s * kHcThreads + q * h.L) * 8 + tid];
+          const float mean = sum / (float)HW;
+#pragma unroll
+          for (uint32_t peer = 0; peer < (uint32_t)kHcCluster; ++peer) hc_st_f32(hc_map(gsm + (size_t)s * h.Cp + c, peer), mean);
+        }
+      }
+    }
+    hc_cluster_arrive();   // #2: the pooled vectors are complete in every CTA
+    hc_cluster_wait();
+  }
+
+  // ---- 2. FC
+  float acc[8][S];
+#pragma unroll
+  for (int q = 0; q < 8; ++q)
+#pragma unroll
+    for (int s = 0; s < S; ++s) acc[q][s] = 0.f;
+  for (int t = 0; t < T; ++t) {
+    const int buf = t % kHcRing;
+    cp_async_wait<kHcRing - 2>();
+    __syncthreads();   // block t landed for every thread; the buffer refilled below was read one iteration ago
+    if (t + kHcRing - 1 < T) block_load(t + kHcRing - 1, (t + kHcRing - 1) % kHcRing);
+    cp_async_commit();
+    const int g = t / h.nchunk, ch = t - g * h.nchunk;
+    float gv[S][8];
+#pragma unroll
+    for (int s = 0; s < S; ++s) {
+      const float4 a = *reinterpret_cast<const float4*>(gsm + (size_t)s * h.Cp + ch * kHcBlockCh + lane * 8);
+      const float4 b = *reinterpret_cast<const float4*>(gsm + (size_t)s * h.Cp + ch * kHcBlockCh + lane * 8 + 4);
+      gv[s][0] = a.x, gv[s][1] = a.y, gv[s][2] = a.z, gv[s][3] = a.w, gv[s][4] = b.x, gv[s][5] = b.y, gv[s][6] = b.z, gv[s][7] = b.w;
+    }
+    const bf16* wb = ring + (size_t)buf * kHcBlockClasses * kHcBlockCh + (warp * 8) * kHcBlockCh + lane * 8;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      Vec16<bf16> w;
+      w.load(wb + q * kHcBlockCh);
+#pragma unroll
+      for (int s = 0; s < S; ++s)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[q][s] = fmaf(w.v[e], gv[s][e], acc[q][s]);
+    }
+    if (ch == h.nchunk - 1) {   // the classes of this block are complete
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const int kl = g * kHcBlockClasses + warp * 8 + q;
+        const float bk = (bfc && kl < nk) ? bfc[k0 + kl] : 0.f;
+#pragma unroll
+        for (int s = 0; s < S; ++s) {
+          float v = acc[q][s];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+          if (lane == 0 && kl < nk) zs[s * kHcMaxKc + kl] = v + bk;
+          acc[q][s] = 0.f;
+        }
+      }
+    }
+  }
+  cp_async_wait<0>();
+  __syncthreads();
+
+  // ---- 3. decision
+  if (warp < S && b0 + warp < B) {
+    const int s = warp, b = b0 + s;
+    const int cls = (d.shift && d.shift_cls) ? d.shift_cls[b] : -1;
+    const float sh = cls >= 0 && cls < K ? d.shift[b] : 0.f;
+    float zr[kHcMaxKc / 32];
+    float m = -INFINITY;
+    int arg = 0x7fffffff;
+#pragma unroll
+    for (int i = 0; i < kHcMaxKc / 32; ++i) {
+      const int j = lane + 32 * i;
+      zr[i] = j < nk ? zs[s * kHcMaxKc + j] : -INFINITY;
+      if (j < nk) {
+        if (k0 + j == cls) zr[i] += sh;
+        if (z) z[(size_t)b * K + k0 + j] = zr[i];
+        if (zr[i] > m) m = zr[i], arg = k0 + j;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float om = __shfl_xor_sync(0xffffffffu, m, o);
+      const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
+      if (om > m || (om == m && oa < arg)) m = om, arg = oa;
+    }
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < kHcMaxKc / 32; ++i)
+      if (lane + 32 * i < nk) sum += expf(zr[i] - m);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) {
+      float* mine = part + ((size_t)rank * S + s) * 4;
+      hc_st_f32(hc_map(mine, 0), m);
+      hc_st_f32(hc_map(mine + 1, 0), __int_as_float(arg));
+      hc_st_f32(hc_map(mine + 2, 0), sum);
+    }
+  }
+  hc_cluster_arrive();   // #3: the leader holds every CTA's triple
+  hc_cluster_wait();
+  if (rank != 0) return;
+  if (tid < S && b0 + tid < B) {
+    const int s = tid, b = b0 + s;
+    float m = -INFINITY;
+    int arg = 0x7fffffff;
+    for (int r = 0; r < kHcCluster; ++r) {   // ranks hold ascending classes: strict > keeps the lowest argmax
+      const float mr = part[(r * S + s) * 4];
+      if (mr > m) m = mr, arg = __float_as_int(part[(r * S + s) * 4 + 1]);
+    }
+    float tot = 0.f;
+    for (int r = 0; r < kHcCluster; ++r) {
+      const float mr = part[(r * S + s) * 4];
+      if (mr != -INFINITY) tot += part[(r * S + s) * 4 + 2] * expf(mr - m);   // a rank without classes holds -inf
+    }
+    const float cf = 1.0f / tot;
+    if (d.conf) d.conf[b] = cf;
+    if (d.pred) d.pred[b] = arg == 0x7fffffff ? 0 : arg;
+    d.mask[b] = (uint8_t)((d.always_exit || cf >= d.thr) ? 1 : 0);
+  }
+  // ---- 4. scan, by the last tile
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) *flag = atomicAdd(d.done, 1u) == gridDim.x / kHcCluster - 1 ? 1 : 0;
+  __syncthreads();
+  if (!*flag) return;
+  __threadfence();
+  if (tid == 0) *d.done = 0;
+  exit_scan<kHcThreads>(B, d);
+}
+
+template <int S>
+inline cudaError_t hc_launch_t(const bf16* x, int HW, int C, const bf16* wfc, const float* bfc, int B, int K, float* z, const DecideArgs& d,
+                               cudaStream_t st) {
+  const HcShape h = hc_shape(C, K);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)((B + S - 1) / S * kHcCluster));
+  cfg.blockDim = dim3(kHcThreads);
+  cfg.dynamicSmemBytes = hc_smem_bytes(S, h);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, head_cluster_kernel<S>, x, HW, C, wfc, bfc, B, K, z, d, h);
+}
+// d.done must be zero when the kernel starts and is zero again when it ends; d.tile_done is not used.
+inline cudaError_t hc_launch(const bf16* x, int HW, int C, const bf16* wfc, const float* bfc, int B, int K, float* z, const DecideArgs& d,
+                             cudaStream_t st) {
+  switch (hc_tile_samples(B)) {
+    case 1: return hc_launch_t<1>(x, HW, C, wfc, bfc, B, K, z, d, st);
+    case 2: return hc_launch_t<2>(x, HW, C, wfc, bfc, B, K, z, d, st);
+    default: return hc_launch_t<4>(x, HW, C, wfc, bfc, B, K, z, d, st);
+  }
+}
+inline cudaError_t hc_context_init() {
+  const size_t most = hc_smem_bytes(4, hc_shape(2048, kHcCluster * kHcMaxKc));
+  cudaError_t e = cudaFuncSetAttribute(head_cluster_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(head_cluster_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(head_cluster_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most);
+  return e;
+}
+
 constexpr int kCopyThreads = 256, kCopyUnroll = 8;
 
 // feat_out[j] = feat[surv_idx[j]] for j < *n_surv, in vectors of type V (16 bytes whenever the row size

@@ -346,6 +346,53 @@ def test_exit_head_alone(dtype, B, HW, C, K):
     assert torch.equal(z1, out.logits[:B])
 
 
+@pytest.mark.parametrize("B,HW,C,K", [(27, 49, 2048, 1000), (5, 3136, 256, 1000), (37, 196, 1024, 1000), (7, 9, 72, 33), (1, 4, 8, 3),
+                                     (19, 16, 1280, 1000), (40, 25, 320, 10), (64, 49, 512, 1024), (18, 1, 264, 129)])
+def test_one_launch_head_against_the_two_kernel_head_and_the_oracle(B, HW, C, K):
+    """The cluster kernel (pool + FC + decision + scan in one launch; an option) and the pooling + FC kernels on the same inputs:
+    logits within fp32 rounding of each other and within the bf16 bar of the oracle, the same predictions and exit
+    decisions away from the threshold, a survivor list consistent with the decisions; each sample alone in a batch of
+    one gives the same bits as inside the batch (tile heights 1, 2 and 4 are all crossed by the batch sizes)."""
+    rng = wl._rng(B * 1000 + C, 905)
+    fw, fb = wl._head(rng, C, K, 8.0, True)
+    layers = [wl._conv(rng, wl.OP_CONV, C, C, 1, 1, 0, wl.ACT_NONE, bf16=True)]
+    spec = wl.Model("head", "bf16", 1, HW, C, [wl.Stage(layers, K, fw, fb, 0.5, False)], B)
+    m = eb.EEModel(spec)
+    out = eb.StageBuffers(m, 0)
+    scratch = torch.empty(m.exit_head_scratch_bytes(0) + 256, dtype=torch.uint8, device="cuda")
+    x = wl.random_features((B, HW, C), seed=HW + 1, bf16=True)
+    shift = (np.arange(B) % 3 == 0).astype(np.float32) * 9.0
+    cls = (np.arange(B) * 5 % K).astype(np.int32)
+    xd, sd, cd = eb.to_device("bf16", x), torch.as_tensor(shift, device="cuda"), torch.as_tensor(cls, device="cuda")
+    got = {}
+    for fused in (True, False, True):            # the last run: the arrival counter of the first must be back at zero
+        m.set_fused_head(fused)
+        assert m.head_launches(0) == (1 if fused else 2)
+        out.logits.fill_(float("nan"))
+        out.n_surv_dev.fill_(-1)
+        m.exit_head(0, xd, B, HW, out, scratch, sd, cd)
+        torch.cuda.synchronize()
+        n = int(out.n_surv_dev.cpu()[0])
+        got[fused] = {"z": out.logits[:B].cpu().numpy(), "conf": out.conf[:B].cpu().numpy(), "pred": out.pred[:B].cpu().numpy(),
+                      "exit": out.exit_mask[:B].cpu().numpy(), "idx": out.survivor_idx[:n].cpu().numpy(), "n": n}
+    one, two = got[True], got[False]
+    o = eo.exit_head(x, fw, fb, 0.5, False, shift, cls)
+    assert util.rel_err(one["z"], two["z"], "bf16", floor=util.LOGIT_FLOOR["bf16"]) <= 1e-3   # fp32 sums over up to 2048 terms, grouped differently
+    assert util.rel_err(one["z"], o["z"], "bf16", floor=util.LOGIT_FLOOR["bf16"]) <= 2e-3
+    assert np.max(np.abs(one["conf"] - o["conf"])) <= 1e-2
+    band = np.abs(o["conf"] - 0.5) < util.BAND
+    assert np.array_equal(one["exit"][~band], o["exit"][~band]) and np.array_equal(one["exit"][~band], two["exit"][~band])
+    top2 = np.sort(o["z"], axis=1)[:, -2:]
+    clear = (top2[:, 1] - top2[:, 0]) > 1e-2 * np.abs(top2[:, 1])
+    assert np.array_equal(one["pred"][clear], o["pred"][clear])
+    assert np.array_equal(one["idx"], np.nonzero(one["exit"] == 0)[0]) and one["n"] == len(one["idx"])
+    # batch invariance: every fourth sample alone
+    for b in range(0, B, 4):
+        m.exit_head(0, xd[b:b + 1].contiguous(), 1, HW, out, scratch, sd[b:b + 1].contiguous(), cd[b:b + 1].contiguous())
+        torch.cuda.synchronize()
+        assert np.array_equal(out.logits[:1].cpu().numpy()[0], one["z"][b]) and float(out.conf[0]) == float(one["conf"][b])
+
+
 def test_compaction_masks_and_gather_bit_exact():
     """Force every mask pattern of a small batch through the head (identity-like FC on 1x1 maps with a
     decisive logit) and check indices, ids, count and the gathered rows bit for bit."""
