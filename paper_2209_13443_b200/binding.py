@@ -20,7 +20,7 @@ EE_OK = 0
 STATUS_NAMES = ["EE_OK", "EE_ERR_INVALID_ARG", "EE_ERR_SHAPE", "EE_ERR_CAPACITY", "EE_ERR_STAGE", "EE_ERR_UNSUPPORTED",
                 "EE_ERR_CUDA", "EE_ERR_TIMEOUT", "EE_ERR_INTERNAL"]
 EXPORTS = ["ee_model_create", "ee_model_destroy", "ee_model_query", "ee_stage_run", "ee_layer_run", "ee_batch_refill", "ee_exit_head",
-           "ee_exit_head_scratch_bytes", "ee_exit_head_static", "ee_gather_survivors", "ee_model_set_graphs", "ee_model_set_branches", "ee_model_set_fused_head", "ee_model_head_launches", "ee_model_set_stage_kernel", "ee_model_set_chain", "ee_model_set_timing", "ee_model_get_timing",
+           "ee_exit_head_scratch_bytes", "ee_exit_head_static", "ee_gather_survivors", "ee_model_set_graphs", "ee_model_set_branches", "ee_model_set_fused_head", "ee_model_set_proj_fusion", "ee_model_head_launches", "ee_model_set_stage_kernel", "ee_model_set_chain", "ee_model_set_timing", "ee_model_get_timing",
            "ee_model_plan", "ee_model_check", "ee_model_set_layer_variant", "ee_model_set_layer_splits", "ee_model_get_layer_config",
            "ee_model_set_wait_limit", "ee_model_selftest_wait", "ee_wait_count", "ee_run_until_exit", "ee_status_string", "ee_last_cuda_error"]
 
@@ -97,6 +97,7 @@ def load_library() -> C.CDLL:
     L.ee_model_set_timing.argtypes = [vp, i]
     L.ee_model_set_branches.argtypes = [vp, i]
     L.ee_model_set_fused_head.argtypes = [vp, i]
+    L.ee_model_set_proj_fusion.argtypes = [vp, i]
     L.ee_model_head_launches.argtypes = [vp, i]
     L.ee_model_head_launches.restype = i
     L.ee_model_set_stage_kernel.argtypes = [vp, i, i]
@@ -313,6 +314,10 @@ class EEModel:
 
     def set_branches(self, enabled: bool):
         _check(self._L.ee_model_set_branches(self._h, int(enabled)), "ee_model_set_branches")
+
+    def set_proj_fusion(self, enabled: bool):
+        """Projection shortcuts computed inside the layer that adds them (bit-identical either way)."""
+        _check(self._L.ee_model_set_proj_fusion(self._h, int(enabled)), "ee_model_set_proj_fusion")
 
     def set_fused_head(self, enabled: bool):
         """One-launch exit head (cluster kernel) on / off; off = pooling kernel + FC/decision kernel."""

@@ -58,6 +58,10 @@ struct LayerPlan {
   // inside ee_stage_run (the convolution's own output is then never written); ee_layer_run still runs either alone.
   bool pool_next = false;     // this layer's launch also does the pooling of the next layer
   bool fused_away = false;    // this (pooling) layer's work is done by the launch of the layer before it
+  // A projection shortcut (1x1, no padding, read only as the residual operand of one later layer) can be computed inside
+  // that layer's launch whenever the layer runs on the persistent kernel at the batch at hand (see conv_tc.cuh, PROJ).
+  int proj_into = -1;         // projection: the layer that can absorb it
+  int proj_from = -1;         // absorbing layer: its projection
   bool side = false;          // runs on the model's branch stream
   int wait_for = -1;          // layer index of a side layer whose result this layer consumes
   cudaEvent_t ev_fork = nullptr, ev_done = nullptr;
@@ -158,6 +162,7 @@ struct ee_model {
   int stage_kernel_max_batch = 1 << 30;
   size_t pair_counter_words = 0;
   unsigned* head_done = nullptr;       // one arrival counter per stage for the one-launch exit head; zero between launches
+  bool proj_fusion = true;             // projection shortcuts computed inside the layer that adds them, where that applies
   bool fused_head = false;             // bf16 models: pool + FC + decision + scan as one cluster kernel where the shape allows (an option)
   long long wait_cycles = kTcWaitCycles;   // limit of the bounded device-side waits of the pair kernel and the self-test
   int device = -1;           // the GPU the model lives on
@@ -384,6 +389,16 @@ ee_status_t append_launch_t(const void* src, void* dst, size_t bytes, const int3
   return EE_OK;
 }
 
+// True when layer `l` of the stage absorbs its projection at batch B: it would run on the persistent kernel anyway and no
+// table entry sends either layer elsewhere.
+bool proj_absorbed(const ee_model* m, const StagePlan& sp, int l, int B) {
+  const LayerPlan& L = sp.layers[l];
+  if (!m->proj_fusion || m->dtype != EE_BF16 || L.proj_from < 0) return false;
+  const LayerPlan& P = sp.layers[L.proj_from];
+  auto plain = [&](const LayerPlan& q) { return q.variant.empty() || q.variant[B] == (uint8_t)TCV_AUTO; };
+  return plain(L) && plain(P) && L.tc.splits == 1 && P.tc.splits == 1 && tc_runs_persistent(m->tc, L.tc, B);
+}
+
 bool stage_kernel_active(const ee_model* m, const StagePlan& sp, int B) {
   return m->dtype == EE_BF16 && m->stage_kernel && !m->timing && !sp.segments.empty() && B <= m->stage_kernel_max_batch;
 }
@@ -433,6 +448,17 @@ ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, c
     const size_t i = m->timing ? k : (size_t)sp.order[k];
     const LayerPlan& L = sp.layers[i];
     if (L.fused_away) continue;   // the launch of the convolution before it pools as well
+    if (L.proj_into >= 0 && !mega && proj_absorbed(m, sp, L.proj_into, B)) continue;   // computed inside the layer that adds it
+    if (L.proj_from >= 0 && !mega && proj_absorbed(m, sp, (int)i, B)) {
+      const LayerPlan& P = sp.layers[L.proj_from];
+      const void* psrc = P.src_slot < 0 ? in->features : ws + sp.slot_off[P.src_slot];
+      const void* lsrc = L.src_slot < 0 ? in->features : ws + sp.slot_off[L.src_slot];
+      ee_status_t ps = tc_launch_proj(m->tc, L.tc, P.tc, lsrc, psrc, ws + sp.slot_off[L.out_slot], B, L.scale_dev, L.bias_dev, P.scale_dev,
+                                      P.bias_dev, m->err_flag, st);
+      if (ps != EE_OK) return ps;
+      record(m, sp, st, kKernelNames[L.kind]);
+      continue;
+    }
     const void* src = L.src_slot < 0 ? in->features : ws + sp.slot_off[L.src_slot];
     const void* res = L.res_slot == -2 ? nullptr : (L.res_slot == -1 ? in->features : ws + sp.slot_off[L.res_slot]);
     void* dst = ws + sp.slot_off[L.pool_next ? sp.layers[i + 1].out_slot : L.out_slot];
@@ -936,6 +962,16 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
       L.pool_next = true;
       P.fused_away = true;
     }
+    for (int i = 0; i < sd.n_layers; ++i) {
+      LayerPlan& P = sp.layers[i];
+      if (P.kind != KK_TC || P.tc.cin != P.d.cin || i == out_layer || n_in_use[i] != 0 || n_res_use[i] != 1 || P.res_slot != -2) continue;
+      LayerPlan& L = sp.layers[res_user[i]];
+      if (L.kind != KK_TC || L.tc.cin != L.d.cin || !tc_proj_supported(L.tc, P.tc)) continue;
+      if (P.src_slot >= 0 && P.src_slot == L.out_slot) continue;   // the layer's output would overwrite the projection's input
+      if (P.src_slot >= 0 && !P.side) continue;   // only a branch layer's input is kept alive until its consumer runs
+      P.proj_into = res_user[i];
+      L.proj_from = i;
+    }
     // Layer runs for the multi-layer launch: consecutive positions of the execution order whose layers the CTA-pair kernel
     // covers with one tile width (256 columns if every layer has more than 128 filters, else 128).
     {
@@ -1332,6 +1368,17 @@ int ee_model_head_launches(const ee_model_t* m, int stage) {
   return m->dtype == EE_BF16 && m->fused_head && hc_supported(sp.out_c, sp.n_classes, nullptr, sp.fc_w) ? 1 : 2;
 }
 
+ee_status_t ee_model_set_proj_fusion(ee_model_t* m, int enabled) {
+  if (!m) return EE_ERR_INVALID_ARG;
+  m->proj_fusion = enabled != 0;
+  drop_chains(m);
+  for (auto& sp : m->stages) {
+    for (auto& g : sp.graphs) sp.retired.push_back(g.exec);
+    sp.graphs.clear();
+  }
+  return EE_OK;
+}
+
 ee_status_t ee_model_set_fused_head(ee_model_t* m, int enabled) {
   if (!m) return EE_ERR_INVALID_ARG;
   m->fused_head = enabled != 0;
@@ -1419,6 +1466,9 @@ ee_status_t ee_model_plan(const ee_model_t* m, int stage, int batch, int cap, ee
       p.bytes = in_b + w_b + (double)batch * P.out_h * P.out_w * P.d.cout * es;
     }
     if (L.fused_away) p.bytes = 0.0, p.launches = 0;   // done by the launch of the convolution before it
+    if (L.proj_into >= 0 && !stage_kernel_active(m, sp, batch) && proj_absorbed(m, sp, L.proj_into, batch))
+      p.bytes = in_b + w_b, p.launches = 0;            // its GEMM runs inside the layer that adds it; its output is never stored
+    if (L.proj_from >= 0 && !stage_kernel_active(m, sp, batch) && proj_absorbed(m, sp, (int)i, batch)) p.bytes = in_b + out_b + w_b;
   }
   if (stage_kernel_active(m, sp, batch))   // a run of layers is one launch: its first layer carries it
     for (const auto& seg : sp.segments)

@@ -51,6 +51,11 @@ struct TcParams {
   // gather mode (layers whose pixel rows are not 16-byte units, e.g. a 3-channel stem): the epilogue warps build the A tile
   const bf16* gx;       // input feature map [B][gH][gW][gCin]
   int gH, gW, gCin, gkh, grun, grunp;  // run = kw*Cin contiguous taps of one filter row, zero-padded to runp columns
+  // projection mode of the persistent kernel: the residual operand is itself a 1x1 convolution (stride stride2, no
+  // padding, scale2 / bias2 / act2) of a second input with the same output geometry, computed into a second accumulator
+  int cblocks2, im2col2, stride2, act2;
+  const float* scale2;
+  const float* bias2;
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -655,7 +660,7 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
 // Staged outputs leave through TMA stores; a staging tile is rewritten only after the warp has seen its previous store
 // finish reading it.  Residual tiles are prefetched by the producer into two buffers of their own, which return to it
 // (res_free) as soon as all four epilogue warps have read them.
-template <int BN, bool RES>
+template <int BN, bool RES, bool PROJ = false>
 struct TcPersistSmem {
   // without a residual: a longer ring and two output staging tiles; with one: two residual tiles the producer
   // prefetches (free again as soon as the epilogue has read them) and a single staging tile
@@ -670,23 +675,31 @@ struct TcPersistSmem {
   static constexpr int kROff = kTiles;
   static constexpr int kOOff = kTiles + (RES ? 2 * kIoBytes : 0);
   static constexpr int kAfter = kOOff + (RES ? 1 : 2) * kIoBytes;
-  static constexpr int kBytes = kAfter + kEpiWarps * 2 * BN * 4 + 256 + 1024;  // + one scale/bias copy per epilogue warp, barriers, slack
+  static constexpr int kSb = (PROJ ? 4 : 2) * BN;   // floats per epilogue warp: scale | bias (| scale2 | bias2)
+  static constexpr int kBytes = kAfter + kEpiWarps * kSb * 4 + 256 + 1024;  // + one scale/bias copy per epilogue warp, barriers, slack
+  static_assert(!(RES && PROJ), "the projection replaces the residual tile");
   static_assert(kBytes <= 227 * 1024, "exceeds the shared memory of an SM");
 };
 
-template <int BN, bool RES>
-__global__ void __launch_bounds__(TcPersistSmem<BN, RES>::kThreads, 1)
+// PROJ: the residual operand is computed here instead of read: after the K blocks of the layer the ring carries the K
+// blocks of a 1x1 projection (tmA2: its input, tile or im2col map; tmW2: its weights) into a second accumulator, and
+// the epilogue rounds scale2 * acc2 + bias2 (act2) to bf16 - the value the projection layer would have stored - before
+// it adds it: the same bits as the two layers run apart, without the projection's output ever reaching global memory.
+template <int BN, bool RES, bool PROJ = false>
+__global__ void __launch_bounds__(TcPersistSmem<BN, RES, PROJ>::kThreads, 1)
 conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
-                                     const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmO, TcParams p) {
+                                     const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmO,
+                                     const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmW2, TcParams p) {
   extern __shared__ uint8_t smem_raw[];
-  using S = TcPersistSmem<BN, RES>;
+  using S = TcPersistSmem<BN, RES, PROJ>;
+  constexpr int kAccs = PROJ ? 2 : 1;   // accumulators per tile
   constexpr int kStages = S::kStages;
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
   float* s_sb = reinterpret_cast<float*>(gen + S::kAfter);  // [epilogue warps][scale BN | bias BN]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kAfter + S::kEpiWarps * 2 * BN * 4);
-  const uint32_t bar0 = base + S::kAfter + S::kEpiWarps * 2 * BN * 4;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kAfter + S::kEpiWarps * S::kSb * 4);
+  const uint32_t bar0 = base + S::kAfter + S::kEpiWarps * S::kSb * 4;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
   auto acc_full = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
@@ -697,6 +710,7 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = p.taps * p.cblocks;
+  const int num_kb2 = PROJ ? p.cblocks2 : 0;   // K blocks of the projection (one tap)
   const int n_tiles = (p.N + BN - 1) / BN;
   const int m_tiles = (p.M + kTcBM - 1) / kTcBM;
   const int total = n_tiles * m_tiles;
@@ -720,9 +734,13 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmO) : "memory");
     if (RES) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmR) : "memory");
+    if (PROJ) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA2) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW2) : "memory");
+    }
   }
-  if (warp == 1) {  // two accumulators of BN fp32 columns
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(2 * BN) : "memory");
+  if (warp == 1) {  // two tiles in flight, each with kAccs accumulators of BN fp32 columns
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(2 * kAccs * BN) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -788,6 +806,30 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
             tma_load_2d(sa, &tmA, full_bar(s), cb * kTcBK, m0);
           }
         }
+        if (PROJ && ok) {   // the projection's K blocks follow in the same ring
+          int cw2 = 0, ch2 = 0, cn2 = 0;
+          if (p.im2col2) {
+            const int hw = p.Ho * p.Wo;
+            cn2 = m0 / hw;
+            const int rem = m0 - cn2 * hw;
+            const int ho = rem / p.Wo;
+            cw2 = (rem - ho * p.Wo) * p.stride2;
+            ch2 = ho * p.stride2;
+          }
+          for (int kb = 0; kb < num_kb2; ++kb, ++g) {
+            const int s = g % kStages;
+            const uint32_t ph = (uint32_t)(g / kStages) & 1u;
+            const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
+            ok = mbar_wait(empty_bar(s), ph ^ 1u, p.err_flag);   // g >= num_kb >= w_ahead: never a pre-armed slot
+            if (!ok) break;
+            mbar_expect_tx(full_bar(s), S::kStage);
+            tma_load_3d(sb, &tmW2, full_bar(s), kb * kTcBK, 0, n0);
+            if (p.im2col2)
+              tma_load_im2col_4d(sa, &tmA2, full_bar(s), kb * kTcBK, cw2, ch2, cn2, (uint16_t)0, (uint16_t)0);
+            else
+              tma_load_2d(sa, &tmA2, full_bar(s), kb * kTcBK, m0);
+          }
+        }
       }
     }
   } else if (warp == 1) {
@@ -802,7 +844,7 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
           if (!ok) break;
           tc_fence_after();
         }
-        const uint32_t acc = tmem_base + (uint32_t)(b * BN);
+        const uint32_t acc = tmem_base + (uint32_t)(b * kAccs * BN);
         for (int kb = 0; kb < num_kb; ++kb, ++g) {
           const int s = g % kStages;
           const uint32_t ph = (uint32_t)(g / kStages) & 1u;
@@ -815,6 +857,20 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
             umma_bf16(acc, umma_desc(sa + k * 32), umma_desc(sb + k * 32), idesc, (uint32_t)((kb | k) != 0));
           umma_commit(empty_bar(s));
         }
+        if (PROJ) {
+          for (int kb = 0; kb < num_kb2 && ok; ++kb, ++g) {
+            const int s = g % kStages;
+            const uint32_t ph = (uint32_t)(g / kStages) & 1u;
+            ok = mbar_wait(full_bar(s), ph, p.err_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
+#pragma unroll
+            for (int k = 0; k < kTcBK / 16; ++k)
+              umma_bf16(acc + (uint32_t)BN, umma_desc(sa + k * 32), umma_desc(sb + k * 32), idesc, (uint32_t)((kb | k) != 0));
+            umma_commit(empty_bar(s));
+          }
+        }
         if (ok) umma_commit(acc_full(b));
       }
     }
@@ -823,7 +879,7 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
     const int row = q * 32 + lane;
     const int ew = warp - 2;
     const int h0 = BN == 128 ? (ew >> 2) : 0, h1 = h0 + 1;  // the 64-column half (halves) this warp owns
-    float* sc = s_sb + ew * 2 * BN;  // this warp's own copy: no barrier across warps inside the tile loop
+    float* sc = s_sb + ew * S::kSb;  // this warp's own copy: no barrier across warps inside the tile loop
     bool ok = true;
     int sc_n0 = -1;
     bool pending = false;  // lane 0: a bulk store group of this warp may still be reading shared memory
@@ -837,6 +893,10 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
           const bool in = n0 + i < p.N;
           sc[i] = (p.scale && in) ? p.scale[n0 + i] : 1.f;
           sc[BN + i] = (p.bias && in) ? p.bias[n0 + i] : 0.f;
+          if (PROJ) {
+            sc[2 * BN + i] = (p.scale2 && in) ? p.scale2[n0 + i] : 1.f;
+            sc[3 * BN + i] = (p.bias2 && in) ? p.bias2[n0 + i] : 0.f;
+          }
         }
         sc_n0 = n0;
       }
@@ -853,9 +913,24 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
       uint8_t* io = gen + S::kOOff + ob * S::kIoBytes;
       const uint32_t io_s = base + S::kOOff + ob * S::kIoBytes;
       const uint8_t* rin = gen + S::kROff + b * S::kIoBytes;
-      const uint32_t acc = tmem_base + (uint32_t)(b * BN) + ((uint32_t)(q * 32) << 16);
+      const uint32_t acc = tmem_base + (uint32_t)(b * kAccs * BN) + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
       for (int h = h0; h < h1; ++h) {
+        uint4 proj[8];   // PROJ: the projection's 64 values of this row, rounded to bf16 as the layer itself would store them
+        if (PROJ) {
+          float pa[32], pb[32];
+          tmem_ld32_issue(acc + (uint32_t)(BN + h * 64), pa);
+          tmem_ld32_issue(acc + (uint32_t)(BN + h * 64 + 32), pb);
+          tmem_ld_wait(pa, pb);
+#pragma unroll
+          for (int sub = 0; sub < 2; ++sub) {
+            const int c0 = h * 64 + sub * 32;
+            const float* v = sub ? pb : pa;
+#pragma unroll
+            for (int gq = 0; gq < 4; ++gq)
+              proj[sub * 4 + gq] = epilogue8_act<false>(p.act2, v + gq * 8, sc + 2 * BN + c0 + gq * 8, sc + 3 * BN + c0 + gq * 8, make_uint4(0u, 0u, 0u, 0u));
+          }
+        }
         float va[32], vb[32];  // both 32-column loads of the half in flight before one wait
         tmem_ld32_issue(acc + (uint32_t)(h * 64), va);
         tmem_ld32_issue(acc + (uint32_t)(h * 64 + 32), vb);
@@ -880,8 +955,8 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
           for (int gq = 0; gq < 4; ++gq) {
             if (n0 + c0 + gq * 8 >= p.N) break;   // columns past Cout: nothing to compute, the store clips them
             const int off = h * 16384 + row * 128 + (((sub * 4 + gq) ^ (lane & 7)) << 4);
-            const uint4 r = RES ? *reinterpret_cast<const uint4*>(rin + off) : make_uint4(0u, 0u, 0u, 0u);
-            *reinterpret_cast<uint4*>(io + off) = epilogue8_act<RES>(p.act, v + gq * 8, sc + c0 + gq * 8, sc + BN + c0 + gq * 8, r);
+            const uint4 r = RES ? *reinterpret_cast<const uint4*>(rin + off) : PROJ ? proj[sub * 4 + gq] : make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(io + off) = epilogue8_act<RES || PROJ>(p.act, v + gq * 8, sc + c0 + gq * 8, sc + BN + c0 + gq * 8, r);
           }
         }
       }
@@ -906,7 +981,7 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * kAccs * BN) : "memory");
   }
 }
 
@@ -1023,6 +1098,8 @@ inline ee_status_t tc_context_init(TcContext& c) {
   set(conv_igemm_tcgen05_persistent_kernel<64, true>, TcPersistSmem<64, true>::kBytes);
   set(conv_igemm_tcgen05_persistent_kernel<128, false>, TcPersistSmem<128, false>::kBytes);
   set(conv_igemm_tcgen05_persistent_kernel<128, true>, TcPersistSmem<128, true>::kBytes);
+  set(conv_igemm_tcgen05_persistent_kernel<64, false, true>, TcPersistSmem<64, false, true>::kBytes);
+  set(conv_igemm_tcgen05_persistent_kernel<128, false, true>, TcPersistSmem<128, false, true>::kBytes);
   if (e != cudaSuccess) return EE_ERR_CUDA;
   return EE_OK;
 }
@@ -1232,7 +1309,72 @@ inline cudaError_t tc_launch_persistent(int ctas, cudaStream_t st, const CUtenso
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_persistent_kernel<BN, RES>, a, w, r, o, p);
+  return cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_persistent_kernel<BN, RES, false>, a, w, r, o, a, w, p);
+}
+
+// The projection mode: a2 / w2 are the projection's input and weight maps.
+template <int BN>
+inline cudaError_t tc_launch_persistent_proj(int ctas, cudaStream_t st, const CUtensorMap& a, const CUtensorMap& w, const CUtensorMap& o,
+                                             const CUtensorMap& a2, const CUtensorMap& w2, const TcParams& p) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(ctas);
+  cfg.blockDim = dim3(TcPersistSmem<BN, false, true>::kThreads);
+  cfg.dynamicSmemBytes = TcPersistSmem<BN, false, true>::kBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_persistent_kernel<BN, false, true>, a, w, o, o, a2, w2, p);
+}
+
+// True when tc_launch runs layer L at batch B on the persistent kernel (several waves of 1x1 tiles, one K range).
+inline bool tc_runs_persistent(const TcContext& c, const TcLayer& L, int B) {
+  if (L.gather || L.halo || L.splits > 1 || L.kh * L.kw != 1) return false;
+  const long tiles = (long)cdiv((long)B * L.out_h * L.out_w, kTcBM) * cdiv(L.cout, L.bn);
+  return tiles >= 2 * c.sm_count;
+}
+
+// A layer L whose residual operand is the output of the 1x1 projection P (no padding, one K range, the same tile width
+// and output geometry) can compute that operand itself on the persistent kernel (see its PROJ note).
+inline bool tc_proj_supported(const TcLayer& L, const TcLayer& P) {
+  return !P.gather && !P.halo && P.splits == 1 && P.kh == 1 && P.kw == 1 && P.pad == 0 && P.pad_w == 0 && P.bn == L.bn && P.cout == L.cout &&
+         P.out_h == L.out_h && P.out_w == L.out_w && L.kh * L.kw == 1 && L.splits == 1 && !L.gather && !L.halo;
+}
+
+// L with the projection P in its launch: src -> L, src2 -> P; P's own output is never written.
+inline ee_status_t tc_launch_proj(TcContext& c, const TcLayer& L, const TcLayer& P, const void* src, const void* src2, void* dst, int B,
+                                  const float* scale, const float* bias, const float* scale2, const float* bias2, int* err_flag,
+                                  cudaStream_t st) {
+  if (((uintptr_t)src & 15) || ((uintptr_t)src2 & 15) || ((uintptr_t)dst & 15)) return EE_ERR_INVALID_ARG;
+  const CUtensorMap* t = nullptr;
+  ee_status_t s = tc_buffer_map(c, L, dst, B, 1, &t);
+  if (s != EE_OK) return s;
+  const CUtensorMap tmO = *t;
+  if ((s = tc_buffer_map(c, L, src, B, 0, &t)) != EE_OK) return s;
+  const CUtensorMap tmA = *t;
+  if ((s = tc_buffer_map(c, P, src2, B, 0, &t)) != EE_OK) return s;
+  const CUtensorMap tmA2 = *t;
+  TcParams p = {};
+  p.M = B * L.out_h * L.out_w;
+  p.N = L.cout;
+  p.taps = 1, p.kw = 1;
+  p.cblocks = cdiv(L.cin, kTcBK);
+  p.Ho = L.out_h, p.Wo = L.out_w, p.stride = L.stride, p.pad = L.pad, p.pad_w = L.pad_w;
+  p.im2col = L.im2col ? 1 : 0;
+  p.act = L.act;
+  p.scale = scale, p.bias = bias;
+  p.residual = nullptr;
+  p.out = (bf16*)dst;
+  p.err_flag = err_flag;
+  p.kb_per = L.kb_per;
+  p.rev = L.rev ? 1 : 0;
+  p.cblocks2 = cdiv(P.cin, kTcBK), p.im2col2 = P.im2col ? 1 : 0, p.stride2 = P.stride, p.act2 = P.act;
+  p.scale2 = scale2, p.bias2 = bias2;
+  const cudaError_t e = L.bn == 128 ? tc_launch_persistent_proj<128>(c.sm_count, st, tmA, L.tm_w, tmO, tmA2, P.tm_w, p)
+                                    : tc_launch_persistent_proj<64>(c.sm_count, st, tmA, L.tm_w, tmO, tmA2, P.tm_w, p);
+  return e == cudaSuccess ? EE_OK : EE_ERR_CUDA;
 }
 
 // Sets the number of K ranges of a layer (1 = no split).  Ranges are equal runs of ceil(num_kb / splits) K blocks, the last

@@ -876,6 +876,43 @@ def test_stem_with_the_pool_in_its_epilogue_equals_the_two_layers_run_apart(case
     assert util.rel_err(apart.float().cpu().numpy(), want, "bf16") <= util.TOL["bf16"]
 
 
+@pytest.mark.parametrize("B", [26, 9])
+def test_projection_inside_the_adding_layer_is_bit_identical_to_its_own_launch(B):
+    """The projection shortcut of a stage's first block computed inside the launch of the layer that adds it (the
+    default wherever that layer runs on the persistent kernel) against the two launches: logits and survivors' features
+    agree bit for bit, on plain launches and replayed graphs; the plan shows which projections are absorbed (B = 26: the
+    first three stages; B = 9: the first only)."""
+    spec = wl.resnet50_ee(seed=1, in_hw=224, n_classes=100, max_batch=26, alphas=[0.01] * 4)
+    run = util.GpuRunner(spec)
+    m, ws = run.m, run.ws
+    x = wl.make_input(spec, B, seed=4)
+    xd = eb.to_device("bf16", x)
+    absorbed = []
+    for s in range(m.n_stages):
+        m.set_proj_fusion(True)
+        on = [pl["launches"] for pl in m.plan(s, B)]
+        m.set_proj_fusion(False)
+        off = [pl["launches"] for pl in m.plan(s, B)]
+        absorbed.append(sum(off) - sum(on))
+        snaps = []
+        for fused, graphs in ((False, False), (True, False), (True, True), (True, True), (False, True)):
+            m.set_proj_fusion(fused)
+            m.set_graphs(graphs)
+            run.bufs[s].logits.fill_(0)
+            run.bufs[s].features_out.fill_(0)
+            m.stage_run(s, xd, B, run.bufs[s], ws)
+            torch.cuda.synchronize()
+            m.check()
+            n = int(run.bufs[s].n_surv_host[0])
+            snaps.append((n, run.bufs[s].logits[:B].clone(), run.bufs[s].features_out[:n].clone()))
+        assert snaps[0][0] == (B if s + 1 < m.n_stages else 0)     # flat logits: nobody leaves before the last exit
+        for n, z, f in snaps[1:]:
+            assert n == snaps[0][0] and torch.equal(z, snaps[0][1]) and torch.equal(f, snaps[0][2]), f"stage {s}"
+        xd = run.bufs[s].features_out[:B].clone()
+    run.check_guards()
+    assert absorbed == ([1, 1, 1, 0] if B == 26 else [1, 0, 0, 0])
+
+
 @pytest.mark.parametrize("B", [1, 3, 7])
 def test_multi_layer_launch_is_bit_identical_to_layer_by_layer(B):
     """Runs of layers executed as one persistent kernel with grid barriers between layers (an option) against the
