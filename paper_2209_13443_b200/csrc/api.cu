@@ -162,6 +162,7 @@ struct ee_model {
   int stage_kernel_max_batch = 1 << 30;
   size_t pair_counter_words = 0;
   unsigned* head_done = nullptr;       // one arrival counter per stage for the one-launch exit head; zero between launches
+  int proj_waves = 1;                  // tiles per SM from which a layer absorbs its projection
   bool proj_fusion = true;             // projection shortcuts computed inside the layer that adds them, where that applies
   bool fused_head = false;             // bf16 models: pool + FC + decision + scan as one cluster kernel where the shape allows (an option)
   long long wait_cycles = kTcWaitCycles;   // limit of the bounded device-side waits of the pair kernel and the self-test
@@ -396,7 +397,7 @@ bool proj_absorbed(const ee_model* m, const StagePlan& sp, int l, int B) {
   if (!m->proj_fusion || m->dtype != EE_BF16 || L.proj_from < 0) return false;
   const LayerPlan& P = sp.layers[L.proj_from];
   auto plain = [&](const LayerPlan& q) { return q.variant.empty() || q.variant[B] == (uint8_t)TCV_AUTO; };
-  return plain(L) && plain(P) && L.tc.splits == 1 && P.tc.splits == 1 && tc_runs_persistent(m->tc, L.tc, B);
+  return plain(L) && plain(P) && L.tc.splits == 1 && P.tc.splits == 1 && tc_runs_persistent(m->tc, L.tc, B, m->proj_waves);
 }
 
 bool stage_kernel_active(const ee_model* m, const StagePlan& sp, int B) {

@@ -1329,11 +1329,12 @@ inline cudaError_t tc_launch_persistent_proj(int ctas, cudaStream_t st, const CU
   return cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_persistent_kernel<BN, false, true>, a, w, o, o, a2, w2, p);
 }
 
-// True when tc_launch runs layer L at batch B on the persistent kernel (several waves of 1x1 tiles, one K range).
-inline bool tc_runs_persistent(const TcContext& c, const TcLayer& L, int B) {
+// True when layer L at batch B has at least `waves` tiles per SM on the persistent kernel (1x1, one K range).  tc_launch
+// itself takes that kernel from two waves on.
+inline bool tc_runs_persistent(const TcContext& c, const TcLayer& L, int B, int waves = 2) {
   if (L.gather || L.halo || L.splits > 1 || L.kh * L.kw != 1) return false;
   const long tiles = (long)cdiv((long)B * L.out_h * L.out_w, kTcBM) * cdiv(L.cout, L.bn);
-  return tiles >= 2 * c.sm_count;
+  return tiles >= (long)waves * c.sm_count;
 }
 
 // A layer L whose residual operand is the output of the 1x1 projection P (no padding, one K range, the same tile width
