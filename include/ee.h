@@ -228,11 +228,11 @@ ee_status_t ee_model_set_graphs(ee_model_t* model, int enabled);
 
 /* Projection shortcuts inside the layer that adds them.  On by default.  A 1x1 convolution without padding whose output
  * is read only as the residual operand of one later 1x1 layer (the projection shortcut of the first block of a stage)
- * is computed by that layer's launch into a second accumulator whenever the layer runs on the persistent tensor-core
- * kernel at the batch at hand (several waves of tiles, one K range, no table entry for either layer): the epilogue rounds
+ * is computed by that layer's launch (the persistent tensor-core kernel) into a second accumulator, provided both
+ * layers have one K range and no table entry: the epilogue rounds
  * the projection to bf16 exactly as the projection layer would have stored it and adds it, so results are bit-identical
  * to the two launches, and the projection's output is neither written nor read back.  ee_model_plan reports such a
- * projection with 0 launches at that batch.  ee_layer_run always runs a layer alone.  Errors: INVALID_ARG. */
+ * projection with 0 launches.  ee_layer_run always runs a layer alone.  Errors: INVALID_ARG. */
 ee_status_t ee_model_set_proj_fusion(ee_model_t* model, int enabled);
 
 /* One-launch exit head.  Off by default.  For bf16 models whose head has C % 8 == 0, C <= 2048 and K <= 1024 (16-byte

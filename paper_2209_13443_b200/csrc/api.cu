@@ -59,7 +59,7 @@ struct LayerPlan {
   bool pool_next = false;     // this layer's launch also does the pooling of the next layer
   bool fused_away = false;    // this (pooling) layer's work is done by the launch of the layer before it
   // A projection shortcut (1x1, no padding, read only as the residual operand of one later layer) can be computed inside
-  // that layer's launch whenever the layer runs on the persistent kernel at the batch at hand (see conv_tc.cuh, PROJ).
+  // that layer's launch, on the persistent kernel (see conv_tc.cuh, PROJ).
   int proj_into = -1;         // projection: the layer that can absorb it
   int proj_from = -1;         // absorbing layer: its projection
   bool side = false;          // runs on the model's branch stream
@@ -162,7 +162,7 @@ struct ee_model {
   int stage_kernel_max_batch = 1 << 30;
   size_t pair_counter_words = 0;
   unsigned* head_done = nullptr;       // one arrival counter per stage for the one-launch exit head; zero between launches
-  int proj_waves = 1;                  // tiles per SM from which a layer absorbs its projection
+  int proj_waves = 0;                  // tiles per SM from which a layer absorbs its projection (measured: a gain at every batch)
   bool proj_fusion = true;             // projection shortcuts computed inside the layer that adds them, where that applies
   bool fused_head = false;             // bf16 models: pool + FC + decision + scan as one cluster kernel where the shape allows (an option)
   long long wait_cycles = kTcWaitCycles;   // limit of the bounded device-side waits of the pair kernel and the self-test
@@ -390,8 +390,7 @@ ee_status_t append_launch_t(const void* src, void* dst, size_t bytes, const int3
   return EE_OK;
 }
 
-// True when layer `l` of the stage absorbs its projection at batch B: it would run on the persistent kernel anyway and no
-// table entry sends either layer elsewhere.
+// True when layer `l` of the stage absorbs its projection at batch B: no table entry sends either layer elsewhere.
 bool proj_absorbed(const ee_model* m, const StagePlan& sp, int l, int B) {
   const LayerPlan& L = sp.layers[l];
   if (!m->proj_fusion || m->dtype != EE_BF16 || L.proj_from < 0) return false;

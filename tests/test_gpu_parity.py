@@ -879,9 +879,8 @@ def test_stem_with_the_pool_in_its_epilogue_equals_the_two_layers_run_apart(case
 @pytest.mark.parametrize("B", [26, 9])
 def test_projection_inside_the_adding_layer_is_bit_identical_to_its_own_launch(B):
     """The projection shortcut of a stage's first block computed inside the launch of the layer that adds it (the
-    default wherever that layer has a tile per SM) against the two launches: logits and survivors' features
-    agree bit for bit, on plain launches and replayed graphs; the plan shows which projections are absorbed (B = 26: all
-    four stages; B = 9: the first two, whose layers still have a tile per SM)."""
+    default) against the two launches: logits and survivors' features
+    agree bit for bit, on plain launches and replayed graphs; the plan shows one launch less per stage."""
     spec = wl.resnet50_ee(seed=1, in_hw=224, n_classes=100, max_batch=26, alphas=[0.01] * 4)
     run = util.GpuRunner(spec)
     m, ws = run.m, run.ws
@@ -910,7 +909,7 @@ def test_projection_inside_the_adding_layer_is_bit_identical_to_its_own_launch(B
             assert n == snaps[0][0] and torch.equal(z, snaps[0][1]) and torch.equal(f, snaps[0][2]), f"stage {s}"
         xd = run.bufs[s].features_out[:B].clone()
     run.check_guards()
-    assert absorbed == ([1, 1, 1, 1] if B == 26 else [1, 1, 0, 0])
+    assert absorbed == [1, 1, 1, 1]
 
 
 @pytest.mark.parametrize("B", [1, 3, 7])
