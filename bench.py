@@ -377,7 +377,9 @@ def run_ours(args):
                     info_s = model.query(s)
                     es_ = 2 if spec.dtype == "bf16" else 4
                     fc_b = info_s["out_c"] * spec.stages[s].n_classes * es_
-                    byt = {"head_gap": n * info_s["out_bytes_per_sample"],
+                    gg = model.gap_partials(s, n)   # > 0: the head pools the block sums the last layer's epilogue wrote
+                    gap_b = n * (info_s["out_h"] * info_s["out_w"] // gg) * info_s["out_c"] * 4 if gg else n * info_s["out_bytes_per_sample"]
+                    byt = {"head_gap": gap_b,
                            "head_fc_softmax_scan": fc_b + n * info_s["out_c"] * 4,
                            "head_gap_fc_softmax_scan": n * info_s["out_bytes_per_sample"] + fc_b}.get(name, 0)
                     pl = per_layer.setdefault((s, i), {"kernel": name, "m": n, "n": spec.stages[s].n_classes, "k": info_s["out_c"],
@@ -389,7 +391,8 @@ def run_ours(args):
             if "head_gap_fc_softmax_scan" in fam:   # the one-launch head: the feature map and the FC weights, each once
                 fam["head_gap_fc_softmax_scan"]["bytes"] += n * info["out_bytes_per_sample"] + info["out_c"] * spec.stages[s].n_classes * es
             else:
-                fam["head_gap"]["bytes"] += n * info["out_bytes_per_sample"]
+                gg = model.gap_partials(s, n)
+                fam["head_gap"]["bytes"] += n * (info["out_h"] * info["out_w"] // gg) * info["out_c"] * 4 if gg else n * info["out_bytes_per_sample"]
                 fam["head_fc_softmax_scan"]["bytes"] += info["out_c"] * spec.stages[s].n_classes * es + n * info["out_c"] * 4
             if "gather_survivors" in fam and not spec.stages[s].always_exit:
                 fam["gather_survivors"]["bytes"] += 2 * ns * info["out_bytes_per_sample"]

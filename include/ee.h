@@ -235,6 +235,16 @@ ee_status_t ee_model_set_graphs(ee_model_t* model, int enabled);
  * projection with 0 launches.  ee_layer_run always runs a layer alone.  Errors: INVALID_ARG. */
 ee_status_t ee_model_set_proj_fusion(ee_model_t* model, int enabled);
 
+/* Pooling partials from the last layer's epilogue.  On by default.  bf16 models pool a stage's output (Section II-B: the
+ * exit head's global average) in blocks of G consecutive rows, G the largest power of two up to 32 that divides
+ * height * width: pairwise tree inside a block, blocks in a fixed order.  When G is 32 or 16 and the stage's last layer
+ * runs on the persistent tensor-core kernel at the batch at hand, that kernel's epilogue writes the block sums of the
+ * tiles it stores (a warp holds 32 rows: one or two blocks) and the head pools those instead of reading the feature map
+ * again; the logits are the same bits either way, and the same as ee_exit_head computes on the stored map.
+ * ee_model_gap_partials returns G when ee_stage_run takes that route for (stage, batch), else 0.  Errors: INVALID_ARG. */
+ee_status_t ee_model_set_gap_fusion(ee_model_t* model, int enabled);
+int ee_model_gap_partials(const ee_model_t* model, int stage, int batch);
+
 /* One-launch exit head.  Off by default.  For bf16 models whose head has C % 8 == 0, C <= 2048 and K <= 1024 (16-byte
  * aligned features and FC weights) global average pool, FC, softmax top-1, threshold and the survivor scan (Section II-B;
  * Section III-B steps 2-3) can run as one kernel of 8-CTA thread-block clusters, one cluster per tile of 1, 2 or 4

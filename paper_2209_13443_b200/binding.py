@@ -20,7 +20,7 @@ EE_OK = 0
 STATUS_NAMES = ["EE_OK", "EE_ERR_INVALID_ARG", "EE_ERR_SHAPE", "EE_ERR_CAPACITY", "EE_ERR_STAGE", "EE_ERR_UNSUPPORTED",
                 "EE_ERR_CUDA", "EE_ERR_TIMEOUT", "EE_ERR_INTERNAL"]
 EXPORTS = ["ee_model_create", "ee_model_destroy", "ee_model_query", "ee_stage_run", "ee_layer_run", "ee_batch_refill", "ee_exit_head",
-           "ee_exit_head_scratch_bytes", "ee_exit_head_static", "ee_gather_survivors", "ee_model_set_graphs", "ee_model_set_branches", "ee_model_set_fused_head", "ee_model_set_proj_fusion", "ee_model_head_launches", "ee_model_set_stage_kernel", "ee_model_set_chain", "ee_model_set_timing", "ee_model_get_timing",
+           "ee_exit_head_scratch_bytes", "ee_exit_head_static", "ee_gather_survivors", "ee_model_set_graphs", "ee_model_set_branches", "ee_model_set_fused_head", "ee_model_set_proj_fusion", "ee_model_set_gap_fusion", "ee_model_gap_partials", "ee_model_head_launches", "ee_model_set_stage_kernel", "ee_model_set_chain", "ee_model_set_timing", "ee_model_get_timing",
            "ee_model_plan", "ee_model_check", "ee_model_set_layer_variant", "ee_model_set_layer_splits", "ee_model_get_layer_config",
            "ee_model_set_wait_limit", "ee_model_selftest_wait", "ee_wait_count", "ee_run_until_exit", "ee_status_string", "ee_last_cuda_error"]
 
@@ -98,6 +98,9 @@ def load_library() -> C.CDLL:
     L.ee_model_set_branches.argtypes = [vp, i]
     L.ee_model_set_fused_head.argtypes = [vp, i]
     L.ee_model_set_proj_fusion.argtypes = [vp, i]
+    L.ee_model_set_gap_fusion.argtypes = [vp, i]
+    L.ee_model_gap_partials.argtypes = [vp, i, i]
+    L.ee_model_gap_partials.restype = i
     L.ee_model_head_launches.argtypes = [vp, i]
     L.ee_model_head_launches.restype = i
     L.ee_model_set_stage_kernel.argtypes = [vp, i, i]
@@ -318,6 +321,13 @@ class EEModel:
     def set_proj_fusion(self, enabled: bool):
         """Projection shortcuts computed inside the layer that adds them (bit-identical either way)."""
         _check(self._L.ee_model_set_proj_fusion(self._h, int(enabled)), "ee_model_set_proj_fusion")
+
+    def set_gap_fusion(self, enabled: bool):
+        """Pooling partials written by the last layer's epilogue (bit-identical either way)."""
+        _check(self._L.ee_model_set_gap_fusion(self._h, int(enabled)), "ee_model_set_gap_fusion")
+
+    def gap_partials(self, stage: int, batch: int) -> int:
+        return int(self._L.ee_model_gap_partials(self._h, stage, batch))
 
     def set_fused_head(self, enabled: bool):
         """One-launch exit head (cluster kernel) on / off; off = pooling kernel + FC/decision kernel."""

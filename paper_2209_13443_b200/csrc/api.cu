@@ -100,6 +100,11 @@ struct StagePlan {
   std::vector<size_t> slot_off;  // byte offsets at max_batch
   size_t head_off = 0, ws_bytes = 0, head_bytes = 0;
   size_t split_off = 0, split_bytes = 0;   // split-K partial tiles of the pair kernel, behind the head scratch
+  // Pooling partials: when the stage's last layer runs on the persistent tensor-core kernel its epilogue also writes
+  // the column sums of every block of gap_g (32 or 16) output rows; the head then pools those block sums instead of
+  // reading the feature map again (same bits: see gap_blocks_kernel).  0 = the map's height * width has no such block.
+  int out_layer = 0, gap_g = 0;
+  size_t gapp_off = 0, gapp_bytes = 0;
   int n_classes = 0;
   void* fc_w = nullptr;
   float* fc_b = nullptr;
@@ -163,6 +168,7 @@ struct ee_model {
   size_t pair_counter_words = 0;
   unsigned* head_done = nullptr;       // one arrival counter per stage for the one-launch exit head; zero between launches
   int proj_waves = 0;                  // tiles per SM from which a layer absorbs its projection (measured: a gain at every batch)
+  bool gap_fusion = true;              // pooling partials from the last layer's epilogue where that applies
   bool proj_fusion = true;             // projection shortcuts computed inside the layer that adds them, where that applies
   bool fused_head = false;             // bf16 models: pool + FC + decision + scan as one cluster kernel where the shape allows (an option)
   long long wait_cycles = kTcWaitCycles;   // limit of the bounded device-side waits of the pair kernel and the self-test
@@ -227,12 +233,14 @@ void layout_stage_tail(ee_model* m, StagePlan& sp) {
       need = std::max(need, std::max(pair_partial_bytes(L.tc, m->max_batch, 256), pair_partial_bytes(L.tc, m->max_batch, 128)));
   sp.split_off = align_up(sp.head_off + sp.head_bytes, 1024);
   sp.split_bytes = need;
-  sp.ws_bytes = sp.split_off + need;
+  sp.gapp_off = align_up(sp.split_off + need, 1024);
+  sp.gapp_bytes = sp.gap_g ? (size_t)m->max_batch * (sp.out_h * sp.out_w / sp.gap_g) * sp.out_c * sizeof(float) : 0;
+  sp.ws_bytes = sp.gapp_off + sp.gapp_bytes;
 }
 
 template <typename T>
 ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const void* res, void* dst, int B, float* partial,
-                         size_t partial_bytes, cudaStream_t st, bool fuse_pool = false) {
+                         size_t partial_bytes, cudaStream_t st, bool fuse_pool = false, float* gap_part = nullptr, int gap_g = 0) {
   ConvGeom g{B, L.in_h, L.in_w, L.d.cin, L.out_h, L.out_w, L.d.cout, L.d.kh, L.d.kw, L.d.stride, L.d.pad, L.d.pad_w, L.d.act};
   constexpr int V = Elem<T>::kVec;
   switch (L.kind) {
@@ -251,7 +259,7 @@ ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const
                           m->wait_cycles, st);
         else
           s = L.tc.halo ? halo_launch(m->tc, L.tc, src, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st)
-                        : tc_launch(m->tc, L.tc, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st);
+                        : tc_launch(m->tc, L.tc, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st, gap_part, gap_g);
       }
       if (s != EE_OK) return s;
       break;
@@ -312,7 +320,7 @@ ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const
 template <typename T>
 ee_status_t launch_head(ee_model* m, StagePlan& sp, const void* x, int B, int hw, const float* shift,
                         const int32_t* shift_cls, char* scratch, const ee_stage_in_t* in_ids, const ee_stage_out_t* out,
-                        cudaStream_t st, bool timed) {
+                        cudaStream_t st, bool timed, const float* gap_part = nullptr, int gap_g = 0) {
   const int C = sp.out_c, K = sp.n_classes;
   HeadLayout h = head_layout(m->max_batch, C, K);
   unsigned* cnt = (unsigned*)(scratch + h.off_cnt);
@@ -331,8 +339,32 @@ ee_status_t launch_head(ee_model* m, StagePlan& sp, const void* x, int B, int hw
   const bool vec = C % V == 0 && ((uintptr_t)x & 15) == 0;
   const int lanes = gap_lanes(hw);
   const int n_zero = m->max_batch + 1;   // the pooling kernel leaves the FC kernel's counters at zero
+  bool pooled = false;
+  if constexpr (sizeof(T) == 2) {
+    // bf16 maps pool in row blocks (gap_blocks_kernel): over the block sums the last layer's epilogue left, or over the map
+    const int sb = sp.gap_rev ? 1 : 0;
+    if (gap_part) {
+      const int nb = hw / gap_g, bl = gap_block_lanes(nb);
+      EE_CUDA(launch_pdl(gap_blocks_kernel<float, 4, 1>, dim3(cdiv(C / 4, bl), B), dim3(kGapThreads), st, gap_part, nb, hw, C, bl, gap, cnt, n_zero, sb));
+      pooled = true;
+    } else if (vec) {
+      const int G = gap_block_rows(hw), nb = hw / G, bl = gap_block_lanes(nb);
+      const dim3 bgrid(cdiv(C / V, bl), B);
+      auto go = [&](auto kernel) { return launch_pdl(kernel, bgrid, dim3(kGapThreads), st, (const T*)x, nb, hw, C, bl, gap, cnt, n_zero, sb); };
+      switch (G) {
+        case 32: EE_CUDA(go(gap_blocks_kernel<T, V, 32>)); break;
+        case 16: EE_CUDA(go(gap_blocks_kernel<T, V, 16>)); break;
+        case 8: EE_CUDA(go(gap_blocks_kernel<T, V, 8>)); break;
+        case 4: EE_CUDA(go(gap_blocks_kernel<T, V, 4>)); break;
+        case 2: EE_CUDA(go(gap_blocks_kernel<T, V, 2>)); break;
+        default: EE_CUDA(go(gap_blocks_kernel<T, V, 1>)); break;
+      }
+      pooled = true;
+    }
+  }
   dim3 ggrid(cdiv(vec ? C / V : C, lanes), B);
-  if (vec)
+  if (pooled) {
+  } else if (vec)
     EE_CUDA(launch_pdl(gap_kernel<T, V>, ggrid, dim3(kGapThreads), st, (const T*)x, hw, C, lanes, gap, cnt, n_zero, sp.gap_rev ? 1 : 0));
   else
     EE_CUDA(launch_pdl(gap_kernel<T, 1>, ggrid, dim3(kGapThreads), st, (const T*)x, hw, C, lanes, gap, cnt, n_zero, sp.gap_rev ? 1 : 0));
@@ -399,6 +431,17 @@ bool proj_absorbed(const ee_model* m, const StagePlan& sp, int l, int B) {
   return plain(L) && plain(P) && L.tc.splits == 1 && P.tc.splits == 1 && tc_runs_persistent(m->tc, L.tc, B, m->proj_waves);
 }
 
+// True when the stage's last layer writes pooling partials at batch B: it runs on the persistent kernel.
+bool gap_partials(const ee_model* m, const StagePlan& sp, int B) {
+  if (!m->gap_fusion || m->dtype != EE_BF16 || sp.gap_g == 0 || (m->stage_kernel && !m->timing && !sp.segments.empty() && B <= m->stage_kernel_max_batch))
+    return false;
+  if (m->fused_head && hc_supported(sp.out_c, sp.n_classes, nullptr, sp.fc_w)) return false;   // that head pools by itself
+  const LayerPlan& L = sp.layers[sp.out_layer];
+  if (L.kind != KK_TC || L.tc.cin != L.d.cin || L.tc.gather || L.tc.halo) return false;
+  if (!(L.variant.empty() || L.variant[B] == (uint8_t)TCV_AUTO)) return false;
+  return proj_absorbed(m, sp, sp.out_layer, B) || tc_runs_persistent(m->tc, L.tc, B);
+}
+
 bool stage_kernel_active(const ee_model* m, const StagePlan& sp, int B) {
   return m->dtype == EE_BF16 && m->stage_kernel && !m->timing && !sp.segments.empty() && B <= m->stage_kernel_max_batch;
 }
@@ -438,6 +481,7 @@ ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, c
   // where every kernel fills the machine by itself and the two cross-stream edges per shortcut are pure overhead.
   const bool mega = stage_kernel_active(m, sp, B);
   const bool par = m->branches && !m->timing && B <= kBranchMaxBatch && !mega;
+  float* gpart = gap_partials(m, sp, B) ? (float*)(ws + sp.gapp_off) : nullptr;   // the last layer's epilogue pools in row blocks
   for (size_t k = 0; k < sp.layers.size(); ++k) {
     if (mega && sp.seg_at[k] >= 0) {
       ee_status_t s = launch_segment(m, sp, sp.segments[sp.seg_at[k]], in, ws, B, st);
@@ -454,7 +498,7 @@ ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, c
       const void* psrc = P.src_slot < 0 ? in->features : ws + sp.slot_off[P.src_slot];
       const void* lsrc = L.src_slot < 0 ? in->features : ws + sp.slot_off[L.src_slot];
       ee_status_t ps = tc_launch_proj(m->tc, L.tc, P.tc, lsrc, psrc, ws + sp.slot_off[L.out_slot], B, L.scale_dev, L.bias_dev, P.scale_dev,
-                                      P.bias_dev, m->err_flag, st);
+                                      P.bias_dev, m->err_flag, st, (int)i == sp.out_layer ? gpart : nullptr, sp.gap_g);
       if (ps != EE_OK) return ps;
       record(m, sp, st, kKernelNames[L.kind]);
       continue;
@@ -470,7 +514,8 @@ ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, c
       ls = m->branch;
     }
     if (par && L.wait_for >= 0) EE_CUDA(cudaStreamWaitEvent(st, sp.layers[L.wait_for].ev_done, 0));   // join
-    ee_status_t s = m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, src, res, dst, B, partial, sp.split_bytes, ls, L.pool_next)
+    ee_status_t s = m->dtype == EE_BF16 ? launch_layer<bf16>(m, L, src, res, dst, B, partial, sp.split_bytes, ls, L.pool_next,
+                                                             (int)i == sp.out_layer ? gpart : nullptr, sp.gap_g)
                                         : launch_layer<float>(m, L, src, res, dst, B, partial, sp.split_bytes, ls);
     if (s != EE_OK) return s;
     if (par && L.side) EE_CUDA(cudaEventRecord(L.ev_done, m->branch));
@@ -479,7 +524,7 @@ ee_status_t enqueue_stage(ee_model* m, StagePlan& sp, const ee_stage_in_t* in, c
   const void* so = ws + sp.slot_off[sp.out_slot];
   const int hw = sp.out_h * sp.out_w;
   ee_status_t s = m->dtype == EE_BF16
-                      ? launch_head<bf16>(m, sp, so, B, hw, in->logit_shift, in->shift_class, ws + sp.head_off, in, out, st, true)
+                      ? launch_head<bf16>(m, sp, so, B, hw, in->logit_shift, in->shift_class, ws + sp.head_off, in, out, st, true, gpart, sp.gap_g)
                       : launch_head<float>(m, sp, so, B, hw, in->logit_shift, in->shift_class, ws + sp.head_off, in, out, st, true);
   if (s != EE_OK) return s;
   // B_exit goes to the host as soon as the decisions are taken: the copy runs on a side branch (also when the stage
@@ -869,9 +914,14 @@ ee_status_t ee_model_create(const ee_model_desc_t* desc, void* cuda_stream, ee_m
       if (L.res_slot >= 0) L.res_slot = slot_of[L.res_slot];
     }
     sp.out_slot = slot_of[out_layer];
+    sp.out_layer = out_layer;
     sp.out_h = oh[out_layer];
     sp.out_w = ow[out_layer];
     sp.out_c = oc[out_layer];
+    {
+      const int g = gap_block_rows(sp.out_h * sp.out_w);
+      sp.gap_g = desc->dtype == EE_BF16 && g >= 16 && sp.out_c % 8 == 0 ? g : 0;
+    }
     HeadLayout hl = head_layout(desc->max_batch, sp.out_c, sd.n_classes);
     sp.head_off = align_up(off, 1024);
     sp.head_bytes = hl.bytes;
@@ -1366,6 +1416,22 @@ int ee_model_head_launches(const ee_model_t* m, int stage) {
   if (!m || stage < 0 || stage >= (int)m->stages.size()) return 0;
   const StagePlan& sp = m->stages[stage];
   return m->dtype == EE_BF16 && m->fused_head && hc_supported(sp.out_c, sp.n_classes, nullptr, sp.fc_w) ? 1 : 2;
+}
+
+int ee_model_gap_partials(const ee_model_t* m, int stage, int batch) {
+  if (!m || stage < 0 || stage >= (int)m->stages.size() || batch < 1 || batch > m->max_batch) return 0;
+  return gap_partials(m, m->stages[stage], batch) ? m->stages[stage].gap_g : 0;
+}
+
+ee_status_t ee_model_set_gap_fusion(ee_model_t* m, int enabled) {
+  if (!m) return EE_ERR_INVALID_ARG;
+  m->gap_fusion = enabled != 0;
+  drop_chains(m);
+  for (auto& sp : m->stages) {
+    for (auto& g : sp.graphs) sp.retired.push_back(g.exec);
+    sp.graphs.clear();
+  }
+  return EE_OK;
 }
 
 ee_status_t ee_model_set_proj_fusion(ee_model_t* m, int enabled) {

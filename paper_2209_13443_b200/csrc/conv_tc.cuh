@@ -56,6 +56,11 @@ struct TcParams {
   int cblocks2, im2col2, stride2, act2;
   const float* scale2;
   const float* bias2;
+  // pooling partials of the persistent kernel: gap_g = 32 or 16 (0 = off): the epilogue also writes, for every block of
+  // gap_g consecutive output rows, the column sums of the bf16-rounded outputs to gap_part[row / gap_g][N] (fp32), summed
+  // pairwise over the rows with distances gap_g/2, ..., 2, 1 - the block sums of gap_blocks_kernel (head.cuh)
+  int gap_g;
+  float* gap_part;
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -250,6 +255,41 @@ __device__ __forceinline__ uint4 epilogue8_act(int act, const float* acc, const 
   if (act == EE_ACT_RELU) return epilogue8<EE_ACT_RELU, RES>(acc, scale, bias, res);
   if (act == EE_ACT_RELU6) return epilogue8<EE_ACT_RELU6, RES>(acc, scale, bias, res);
   return epilogue8<EE_ACT_NONE, RES>(acc, scale, bias, res);
+}
+
+// Column sums over the 32 rows a warp holds (ov: this lane's row, 64 bf16 columns as eight 16-byte groups), written as
+// block sums of G rows (see TcParams::gap_g).  Halving butterfly: in the step of distance d a lane keeps half of its
+// columns and receives its partner's values for them, so that every (block, column) sum is formed once, by the tree
+// ((r, r + G/2), then distance G/4, ...).  Afterwards lane l holds columns [2l, 2l + 2) of the block (G = 32) or
+// columns [4 (l % 16), + 4) of block l / 16 (G = 16).
+template <int G>
+__device__ __forceinline__ void gap_partial_store(const uint4* ov, int lane, float* dst, int cols_left, size_t block_stride, bool rows_ok) {
+  float f[64];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const uint32_t w[4] = {ov[i].x, ov[i].y, ov[i].z, ov[i].w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      f[8 * i + 2 * k] = __uint_as_float(w[k] << 16);
+      f[8 * i + 2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+    }
+  }
+#pragma unroll
+  for (int d = G / 2, n = 32; d >= 1; d >>= 1, n >>= 1) {
+    const bool up = (lane & d) != 0;
+#pragma unroll
+    for (int i = 0; i < n; ++i) {
+      const float send = up ? f[i] : f[i + n], keep = up ? f[i + n] : f[i];
+      f[i] = keep + __shfl_xor_sync(0xffffffffu, send, d);
+    }
+  }
+  if (!rows_ok) return;
+  if (G == 32) {
+    if (2 * lane < cols_left) *reinterpret_cast<float2*>(dst + 2 * lane) = make_float2(f[0], f[1]);
+  } else {
+    const int c = 4 * (lane & 15);
+    if (c < cols_left) *reinterpret_cast<float4*>(dst + (size_t)(lane >> 4) * block_stride + c) = make_float4(f[0], f[1], f[2], f[3]);
+  }
 }
 
 // ----------------------------------------------------------------------------- kernel
@@ -931,6 +971,9 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
               proj[sub * 4 + gq] = epilogue8_act<false>(p.act2, v + gq * 8, sc + 2 * BN + c0 + gq * 8, sc + 3 * BN + c0 + gq * 8, make_uint4(0u, 0u, 0u, 0u));
           }
         }
+        uint4 ov[8];           // this row's 64 outputs of the half (kept for the pooling partials)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ov[i] = make_uint4(0u, 0u, 0u, 0u);
         float va[32], vb[32];  // both 32-column loads of the half in flight before one wait
         tmem_ld32_issue(acc + (uint32_t)(h * 64), va);
         tmem_ld32_issue(acc + (uint32_t)(h * 64 + 32), vb);
@@ -956,8 +999,17 @@ conv_igemm_tcgen05_persistent_kernel(const __grid_constant__ CUtensorMap tmA, co
             if (n0 + c0 + gq * 8 >= p.N) break;   // columns past Cout: nothing to compute, the store clips them
             const int off = h * 16384 + row * 128 + (((sub * 4 + gq) ^ (lane & 7)) << 4);
             const uint4 r = RES ? *reinterpret_cast<const uint4*>(rin + off) : PROJ ? proj[sub * 4 + gq] : make_uint4(0u, 0u, 0u, 0u);
-            *reinterpret_cast<uint4*>(io + off) = epilogue8_act<RES || PROJ>(p.act, v + gq * 8, sc + c0 + gq * 8, sc + BN + c0 + gq * 8, r);
+            ov[sub * 4 + gq] = epilogue8_act<RES || PROJ>(p.act, v + gq * 8, sc + c0 + gq * 8, sc + BN + c0 + gq * 8, r);
+            *reinterpret_cast<uint4*>(io + off) = ov[sub * 4 + gq];
           }
+        }
+        if (p.gap_g) {   // rows past M hold zero-filled operands, but their bias and residual garbage must not be summed: whole blocks are skipped
+          const int r0 = m0 + q * 32;
+          if (p.gap_g == 32)
+            gap_partial_store<32>(ov, lane, p.gap_part + (size_t)(r0 / 32) * p.N + n0 + h * 64, p.N - n0 - h * 64, 0, r0 < p.M);
+          else
+            gap_partial_store<16>(ov, lane, p.gap_part + (size_t)(r0 / 16) * p.N + n0 + h * 64, p.N - n0 - h * 64, (size_t)p.N,
+                                  r0 + (lane >> 4) * 16 < p.M);
         }
       }
       if (RES) {  // the residual tile is consumed: the producer may prefetch the one of tile j + 2 into it
@@ -1347,7 +1399,7 @@ inline bool tc_proj_supported(const TcLayer& L, const TcLayer& P) {
 // L with the projection P in its launch: src -> L, src2 -> P; P's own output is never written.
 inline ee_status_t tc_launch_proj(TcContext& c, const TcLayer& L, const TcLayer& P, const void* src, const void* src2, void* dst, int B,
                                   const float* scale, const float* bias, const float* scale2, const float* bias2, int* err_flag,
-                                  cudaStream_t st) {
+                                  cudaStream_t st, float* gap_part = nullptr, int gap_g = 0) {
   if (((uintptr_t)src & 15) || ((uintptr_t)src2 & 15) || ((uintptr_t)dst & 15)) return EE_ERR_INVALID_ARG;
   const CUtensorMap* t = nullptr;
   ee_status_t s = tc_buffer_map(c, L, dst, B, 1, &t);
@@ -1373,6 +1425,7 @@ inline ee_status_t tc_launch_proj(TcContext& c, const TcLayer& L, const TcLayer&
   p.rev = L.rev ? 1 : 0;
   p.cblocks2 = cdiv(P.cin, kTcBK), p.im2col2 = P.im2col ? 1 : 0, p.stride2 = P.stride, p.act2 = P.act;
   p.scale2 = scale2, p.bias2 = bias2;
+  p.gap_part = gap_part, p.gap_g = gap_part ? gap_g : 0;
   const cudaError_t e = L.bn == 128 ? tc_launch_persistent_proj<128>(c.sm_count, st, tmA, L.tm_w, tmO, tmA2, P.tm_w, p)
                                     : tc_launch_persistent_proj<64>(c.sm_count, st, tmA, L.tm_w, tmO, tmA2, P.tm_w, p);
   return e == cudaSuccess ? EE_OK : EE_ERR_CUDA;
@@ -1390,8 +1443,9 @@ inline bool tc_set_splits(TcLayer& L, int splits) {
   return true;
 }
 
+// gap_part / gap_g: pooling partials (TcParams::gap_g); only a launch on the persistent kernel (tc_runs_persistent) writes them.
 inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, const void* res, void* dst, int B, const float* scale,
-                             const float* bias, int* err_flag, cudaStream_t st) {
+                             const float* bias, int* err_flag, cudaStream_t st, float* gap_part = nullptr, int gap_g = 0) {
   if (((uintptr_t)src & 15) || ((uintptr_t)dst & 15) || ((uintptr_t)res & 15)) return EE_ERR_INVALID_ARG;
   // copies: a later lookup may grow the cache and move its entries
   const CUtensorMap* t = nullptr;
@@ -1408,7 +1462,8 @@ inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, co
     if ((s = tc_buffer_map(c, L, res, B, 1, &t)) != EE_OK) return s;
     tmR = *t;
   }
-  TcParams p;
+  TcParams p = {};
+  p.gap_part = gap_part, p.gap_g = gap_part ? gap_g : 0;
   p.M = B * L.out_h * L.out_w;
   p.N = L.cout;
   p.taps = L.kh * L.kw;

@@ -90,6 +90,87 @@ inline int gap_lanes(int hw) {
   return kGapThreads / groups;
 }
 
+// ----------------------------------------------------------------------------- pooling in row blocks (bf16 models)
+//
+// gap[b][c] = (sum over the HW rows of sample b) / HW with the sum grouped in a way that a convolution's epilogue can
+// start: the rows are cut into nb = HW / G blocks of G consecutive rows, G the largest power of two up to 32 that
+// divides HW, so that a block never straddles two samples and, for G = 32 or 16, is exactly the rows one epilogue warp
+// (or half of it) holds.  Block sum: the pairwise tree T(g, o, s) = T(g/2, o, 2s) + T(g/2, o + s, 2s), T(1, o, .) =
+// row o - what a shuffle butterfly over the lanes with distances G/2, ..., 2, 1 computes.  Sample sum: row group q of
+// 256 / lanes adds the blocks q, q + groups, ... in ascending order, then the group sums are added in ascending
+// order.  A tensor-core kernel that writes the block sums of its output tile (conv_tc.cuh, gap partials) followed by
+// this kernel with G = 1 over those sums gives the same bits as this kernel over the stored feature map.
+inline int gap_block_rows(int hw) {
+  int g = 1;
+  while (g < 32 && hw % (2 * g) == 0) g *= 2;
+  return g;
+}
+// Channel vectors side by side in a CTA for nb blocks per sample: as many row groups as there are blocks, between 8 and 64.
+inline int gap_block_lanes(int nb) {
+  int groups = 8;
+  while (groups < 64 && groups * 2 <= nb) groups *= 2;
+  return kGapThreads / groups;
+}
+
+template <int g, int VEC, typename LD>
+__device__ __forceinline__ void gap_tree(LD&& load, int o, int s, float* out) {
+  if constexpr (g == 1) {
+    load(o, out);
+  } else {
+    float a[VEC], b[VEC];
+    gap_tree<g / 2, VEC>(load, o, 2 * s, a);
+    gap_tree<g / 2, VEC>(load, o + s, 2 * s, b);
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) out[e] = a[e] + b[e];
+  }
+}
+
+// T = bf16 (VEC 8, the feature map) or float (VEC 4, block sums written by a convolution's epilogue; G = 1).
+template <typename T, int VEC, int G>
+__global__ void __launch_bounds__(kGapThreads)
+gap_blocks_kernel(const T* __restrict__ x, int nb, int HW, int C, int lanes, float* __restrict__ gap, unsigned* __restrict__ zero_me,
+                  int n_zero, int rev) {
+  __shared__ float red[kGapThreads * VEC];
+  const int tid = threadIdx.x, b = rev ? (int)(gridDim.y - 1 - blockIdx.y) : (int)blockIdx.y;
+  const int cv = C / VEC;
+  const int groups = kGapThreads / lanes;
+  const int grp = tid / lanes, lv = tid - grp * lanes;
+  const int v = blockIdx.x * lanes + lv;
+  pdl_wait();
+  pdl_launch_dependents();
+  if (blockIdx.x == 0 && blockIdx.y == 0)
+    for (int i = tid; i < n_zero; i += kGapThreads) zero_me[i] = 0u;
+  float acc[VEC];
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+  if (v < cv) {
+    const T* p0 = x + (size_t)b * nb * G * C + (size_t)v * VEC;
+    for (int j = grp; j < nb; j += groups) {
+      const T* pb = p0 + (size_t)j * G * C;
+      float t[VEC];
+      gap_tree<G, VEC>([&](int row, float* out) {
+        Vec16<T> r;
+        r.load(pb + (size_t)row * C);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) out[e] = r.v[e];
+      }, 0, 1, t);
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) acc[e] += t[e];
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) red[(grp * lanes + lv) * VEC + e] = acc[e];
+  __syncthreads();
+  if (tid < lanes * VEC) {
+    const int c = blockIdx.x * lanes * VEC + tid;
+    if (c < cv * VEC) {
+      float sum = 0.f;
+      for (int q = 0; q < groups; ++q) sum += red[q * lanes * VEC + tid];
+      gap[(size_t)b * C + c] = sum / (float)HW;
+    }
+  }
+}
+
 struct DecideArgs {  // everything the exit decision needs besides the logits
   const float* shift;
   const int32_t* shift_cls;

@@ -912,6 +912,52 @@ def test_projection_inside_the_adding_layer_is_bit_identical_to_its_own_launch(B
     assert absorbed == [1, 1, 1, 1]
 
 
+@pytest.mark.parametrize("B", [26, 9, 1])
+def test_pooling_partials_from_the_epilogue_give_the_bits_of_pooling_the_stored_map(B):
+    """Where the last layer of a stage runs on the persistent kernel its epilogue writes block sums of the rows it holds
+    and the head pools those; elsewhere, and in ee_exit_head, the pooling kernel forms the same blocks from the stored
+    map.  Logits must agree bit for bit between the two routes, with ee_exit_head on the stage's own output, and - batch
+    invariance across the routes - with the sample alone in a batch of one (which never takes the epilogue route)."""
+    spec = wl.resnet50_ee(seed=1, in_hw=224, n_classes=100, max_batch=26, alphas=[0.01] * 4)
+    run = util.GpuRunner(spec)
+    m, ws = run.m, run.ws
+    x = wl.make_input(spec, B, seed=6)
+    xd = eb.to_device("bf16", x)
+    routes = []
+    for s in range(m.n_stages):
+        routes.append(m.gap_partials(s, B))
+        snaps = []
+        for fused, graphs in ((False, False), (True, False), (True, True), (True, True)):
+            m.set_gap_fusion(fused)
+            m.set_graphs(graphs)
+            assert m.gap_partials(s, B) == (routes[s] if fused else 0)
+            run.bufs[s].logits.fill_(0)
+            m.stage_run(s, xd, B, run.bufs[s], ws)
+            torch.cuda.synchronize()
+            m.check()
+            snaps.append((run.bufs[s].logits[:B].clone(), run.bufs[s].conf[:B].clone()))
+        for z, c in snaps[1:]:
+            assert torch.equal(z, snaps[0][0]) and torch.equal(c, snaps[0][1]), f"stage {s}"
+        n = int(run.bufs[s].n_surv_host[0])
+        if s + 1 < m.n_stages:
+            assert n == B
+            feat = run.bufs[s].features_out[:B].clone()
+            info = m.query(s)
+            hw = info["out_h"] * info["out_w"]
+            out2 = eb.StageBuffers(m, s)
+            scratch = torch.empty(m.exit_head_scratch_bytes(s) + 256, dtype=torch.uint8, device="cuda")
+            m.exit_head(s, feat, B, hw, out2, scratch)
+            torch.cuda.synchronize()
+            assert torch.equal(out2.logits[:B], snaps[0][0]), f"stage {s}: ee_exit_head on the stored map"
+            b = B - 1                                   # the last sample alone: stage on its input row
+            m.stage_run(s, xd[b:b + 1].contiguous(), 1, out2, ws)
+            torch.cuda.synchronize()
+            assert torch.equal(out2.logits[0], snaps[0][0][b]), f"stage {s}: batch of one"
+            xd = feat
+    run.check_guards()
+    assert routes == {26: [32, 16, 0, 0], 9: [32, 0, 0, 0], 1: [0, 0, 0, 0]}[B]
+
+
 @pytest.mark.parametrize("B", [1, 3, 7])
 def test_multi_layer_launch_is_bit_identical_to_layer_by_layer(B):
     """Runs of layers executed as one persistent kernel with grid barriers between layers (an option) against the
