@@ -34,8 +34,8 @@ if ROOT not in sys.path:
 # DRAM bytes (read + written) per launch of the tensor-core conv kernels, from one ncu capture of the default workload
 # (ResNet-50-shaped, B=64, calibrated exits: 52 launches per pass, 1735.2 MB).  Reported only for that workload; it
 # has to be taken again (or set to None) whenever one of those kernels changes.
-NCU_CONV_TRAFFIC_PER_LAUNCH = {("resnet50", 64): 33.34e6}
-NCU_CONV_TRAFFIC_WARM_L2 = {("resnet50", 64): 27.79e6}   # same capture with --cache-control none
+NCU_CONV_TRAFFIC_PER_LAUNCH = {("resnet50", 64): 31.72e6}
+NCU_CONV_TRAFFIC_WARM_L2 = {("resnet50", 64): 23.77e6}   # same capture with --cache-control none
 
 METRIC = "EE-CNN samples/sec on 1 B200 vs exit rate & batch 1-64; tensor-pipe % of peak"
 UNIT = "samples/s"
@@ -345,7 +345,7 @@ def run_ours(args):
             stage_batch[s] = n
             convs = [pl for pl in model.plan(s, n) if pl["kernel"].startswith("conv_igemm_tcgen05")]
             stage_flops[s] = sum(pl["flops"] for pl in convs)
-            stage_conv_launches[s] = len(convs)
+            stage_conv_launches[s] = sum(pl["launches"] for pl in convs)   # a projection computed inside another layer has none
             feat, ids, n = bufs[s].features_out, bufs[s].ids_out, ns
             if n == 0:
                 break
