@@ -302,7 +302,10 @@ ee_status_t ee_model_plan(const ee_model_t* model, int stage, int batch, int cap
  * tensor-core layer and every batch size 1..max_batch, which kernel variant runs the layer:
  *   0  one-CTA tiles (128 x 128 or 128 x 64; one-tile, persistent or cluster split-K kernels chosen from the grid),
  *   1  CTA pairs, 256 x 256 tiles (tcgen05 cta_group::2, persistent (tile, K-range) units),
- *   2  CTA pairs, 256 x 128 tiles.
+ *   2  CTA pairs, 256 x 128 tiles,
+ *   3  one-CTA tiles, the layer's K ranges as a cluster of CTAs per tile (reduce-scatter over distributed shared memory),
+ *   4  one-CTA tiles, the K ranges inside ONE CTA per tile, an accumulator in tensor memory per range (ranges x tile
+ *      width <= 512 columns, else as 3); variant 0 picks 3 while tiles x ranges stays within 1.25 waves of SMs, else 4.
  * The number of K ranges of a layer (`splits`) is one value per layer for all batch sizes and all variants, and the
  * partial sums of the ranges are always added in ascending order, so a sample's result is bit-identical whichever
  * variant the table picks for the batch it rides in.  Both setters drop the stage's captured graphs.

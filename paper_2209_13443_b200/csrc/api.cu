@@ -254,12 +254,14 @@ ee_status_t launch_layer(ee_model* m, const LayerPlan& L, const void* src, const
       const int v = L.variant.empty() ? (int)TCV_AUTO : (int)L.variant[B];
       ee_status_t s = EE_ERR_INTERNAL;
       if constexpr (sizeof(T) == 2) {
-        if (v != TCV_AUTO && pair_supported(L.tc, v))
+        const bool pair_v = v == TCV_PAIR256 || v == TCV_PAIR128;
+        const int range_mode = v == TCV_RANGES_CLUSTER ? 1 : v == TCV_RANGES_LOCAL ? 2 : 0;
+        if (pair_v && pair_supported(L.tc, v))
           s = pair_launch(m->tc, L.tc, v, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, partial, partial_bytes, m->pair_counters,
                           m->wait_cycles, st);
         else
           s = L.tc.halo ? halo_launch(m->tc, L.tc, src, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st)
-                        : tc_launch(m->tc, L.tc, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st, gap_part, gap_g);
+                        : tc_launch(m->tc, L.tc, src, res, dst, B, L.scale_dev, L.bias_dev, m->err_flag, st, gap_part, gap_g, range_mode);
       }
       if (s != EE_OK) return s;
       break;
@@ -1550,7 +1552,9 @@ ee_status_t ee_model_set_layer_variant(ee_model_t* m, int stage, int layer, int 
   if (layer < 0 || layer >= (int)sp.layers.size()) return EE_ERR_STAGE;
   if (batch_hi > m->max_batch) return EE_ERR_CAPACITY;
   LayerPlan& L = sp.layers[layer];
-  if (variant != TCV_AUTO && (L.kind != KK_TC || !pair_supported(L.tc, variant))) return EE_ERR_UNSUPPORTED;
+  const bool ranges_v = variant == TCV_RANGES_CLUSTER || variant == TCV_RANGES_LOCAL;
+  if (ranges_v && (L.kind != KK_TC || L.tc.gather || L.tc.halo)) return EE_ERR_UNSUPPORTED;
+  if (variant != TCV_AUTO && !ranges_v && (L.kind != KK_TC || !pair_supported(L.tc, variant))) return EE_ERR_UNSUPPORTED;
   if (L.variant.empty()) L.variant.assign((size_t)m->max_batch + 1, (uint8_t)TCV_AUTO);
   for (int b = batch_lo; b <= batch_hi; ++b) L.variant[b] = (uint8_t)variant;
   for (auto& g : sp.graphs) cudaGraphExecDestroy(g.exec);   // captured stages hold the old choice

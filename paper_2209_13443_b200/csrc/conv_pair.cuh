@@ -566,7 +566,7 @@ __global__ void wait_selftest_kernel(int* err_flag, long long limit, int* reache
 // ----------------------------------------------------------------------------- host side
 
 // Kernel variants a tensor-core layer can run as (the per-(layer, batch) table of LayerPlan holds one of these).
-enum TcVariant { TCV_AUTO = 0, TCV_PAIR256 = 1, TCV_PAIR128 = 2, TCV_COUNT = 3 };
+enum TcVariant { TCV_AUTO = 0, TCV_PAIR256 = 1, TCV_PAIR128 = 2, TCV_RANGES_CLUSTER = 3, TCV_RANGES_LOCAL = 4, TCV_COUNT = 5 };
 
 inline ee_status_t pair_context_init() {
   if (cudaFuncSetAttribute(conv_igemm_tcgen05_pair_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem<256>::kBytes) != cudaSuccess ||

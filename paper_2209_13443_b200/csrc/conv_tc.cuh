@@ -46,6 +46,9 @@ struct TcParams {
   bf16* out;
   int* err_flag;
   int kb_per;           // split-K: K blocks per range (a property of the layer)
+  int ranges;           // > 1 (one-CTA kernel without SPLIT): this CTA runs all `ranges` K ranges of its tile itself, each
+                        // into an accumulator of its own, and adds them in ascending order in the epilogue - the same
+                        // bits as `ranges` CTAs of a cluster reducing their partial tiles
   int rev;              // 1: walk the M tiles from the last one down (start where the producer of the input finished: its
                         // newest rows are the ones still in L2)
   // gather mode (layers whose pixel rows are not 16-byte units, e.g. a 3-channel stem): the epilogue warps build the A tile
@@ -452,8 +455,11 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmO) : "memory");
     if (RES) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmR) : "memory");
   }
-  if (warp == 1) {  // TMEM: BN fp32 columns x 128 lanes
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN) : "memory");
+  const int n_acc = SPLIT ? 1 : max(p.ranges, 1);   // accumulators of BN fp32 columns
+  uint32_t acc_cols = BN;                           // TMEM allocations are powers of two
+  while ((int)acc_cols < n_acc * BN) acc_cols *= 2;
+  if (warp == 1) {  // TMEM: acc_cols fp32 columns x 128 lanes
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(acc_cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -525,9 +531,10 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
         if (!ok) break;
         tc_fence_after();
         const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
+        const int r = n_acc > 1 ? i / p.kb_per : 0, ir = i - r * p.kb_per;   // local K range and position inside it
 #pragma unroll
         for (int k = 0; k < kTcBK / 16; ++k)
-          umma_bf16(tmem_base, umma_desc(sa + k * 32), umma_desc(sb + k * 32), idesc, (uint32_t)((i | k) != 0));
+          umma_bf16(tmem_base + (uint32_t)(r * BN), umma_desc(sa + k * 32), umma_desc(sb + k * 32), idesc, (uint32_t)((ir | k) != 0));
         umma_commit(empty_bar(s));  // frees the stage once these MMAs have read it
       }
       if (ok && num_kb > 0) umma_commit(accum_bar);  // accumulator complete: every MMA has also finished reading the ring
@@ -615,6 +622,16 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
           const int c0 = h * 64 + sub * 32;
           float v[32];
           tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+          if (n_acc > 1) {   // local K ranges: 0 + range 0 + range 1 + ... as the cluster reduction adds them
+#pragma unroll
+            for (int e = 0; e < 32; ++e) v[e] = 0.f + v[e];
+            for (int r = 1; r < n_acc; ++r) {
+              float t[32];
+              tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(r * BN + c0), t);
+#pragma unroll
+              for (int e = 0; e < 32; ++e) v[e] += t[e];
+            }
+          }
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
             if (n0 + c0 + g * 8 >= p.N) break;   // columns past Cout: nothing to compute, the store clips them
@@ -685,7 +702,7 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(acc_cols) : "memory");
   }
 }
 
@@ -1445,7 +1462,8 @@ inline bool tc_set_splits(TcLayer& L, int splits) {
 
 // gap_part / gap_g: pooling partials (TcParams::gap_g); only a launch on the persistent kernel (tc_runs_persistent) writes them.
 inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, const void* res, void* dst, int B, const float* scale,
-                             const float* bias, int* err_flag, cudaStream_t st, float* gap_part = nullptr, int gap_g = 0) {
+                             const float* bias, int* err_flag, cudaStream_t st, float* gap_part = nullptr, int gap_g = 0,
+                             int range_mode = 0) {
   if (((uintptr_t)src & 15) || ((uintptr_t)dst & 15) || ((uintptr_t)res & 15)) return EE_ERR_INVALID_ARG;
   // copies: a later lookup may grow the cache and move its entries
   const CUtensorMap* t = nullptr;
@@ -1476,7 +1494,17 @@ inline ee_status_t tc_launch(TcContext& c, const TcLayer& L, const void* src, co
   p.residual = (const bf16*)res;
   p.out = (bf16*)dst;
   p.err_flag = err_flag;
-  const bool split = L.splits > 1;
+  // A layer with several K ranges runs them as a cluster of CTAs per tile (more SMs pull operands: small grids) or, bit
+  // for bit the same, in ONE CTA per tile with an accumulator per range (no cluster, no exchange: grids that fill the GPU
+  // anyway).  range_mode: 0 = the cluster while the whole grid still fits one wave, 1 = cluster, 2 = one CTA.
+  const long tiles_all = (long)cdiv(p.M, kTcBM) * cdiv(L.cout, L.bn);
+  const bool can_local = L.splits > 1 && L.splits * L.bn <= 512 && !L.gather;
+  // Measured (3x3 256->256 on 14x14, 2 and 4 ranges): the cluster wins while tiles x ranges stays within about 1.25 waves
+  // and loses badly beyond; one CTA with 2 accumulators costs 1 us per layer over a single range, with 4 (all 512 TMEM
+  // columns: no second CTA, no overlap with the neighbouring kernels' prologues) 17 us.
+  const bool local = can_local && (range_mode == 2 || (range_mode == 0 && tiles_all * L.splits * 4 > 5L * c.sm_count));
+  const bool split = L.splits > 1 && !local;
+  p.ranges = local ? L.splits : 1;
   p.kb_per = L.kb_per;
   p.rev = L.rev ? 1 : 0;
   p.gx = (const bf16*)src;

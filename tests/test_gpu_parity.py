@@ -203,6 +203,52 @@ def test_pair_kernel_layer(geom):
             assert e <= util.TOL["bf16"], f"pair {geom} B={B} run {rep}: {e:.3e}"
 
 
+RANGE_GEOMS = [
+    # H, W, cin, cout, k, stride, pad, act, residual, K ranges
+    (14, 14, 256, 256, 3, 1, 1, wl.ACT_RELU, False, 4),
+    (14, 14, 256, 256, 3, 1, 1, wl.ACT_RELU, False, 3),
+    (14, 14, 1024, 256, 1, 1, 0, wl.ACT_RELU, False, 4),
+    (14, 14, 512, 512, 3, 2, 1, wl.ACT_RELU, False, 2),
+    (7, 7, 512, 2048, 1, 1, 0, wl.ACT_RELU, True, 2),
+    (7, 7, 2048, 512, 1, 1, 0, wl.ACT_NONE, False, 4),
+    (28, 28, 256, 64, 3, 1, 1, wl.ACT_RELU6, False, 8),     # 64-wide tiles: eight accumulators of 64 columns
+    (14, 14, 136, 72, 3, 1, 1, wl.ACT_RELU, False, 3),      # ragged channels and filters
+]
+
+
+@pytest.mark.parametrize("geom", RANGE_GEOMS)
+def test_k_ranges_in_one_cta_give_the_bits_of_the_cluster_of_ctas(geom):
+    """A layer's K ranges run as a cluster of CTAs per tile or, one accumulator per range, inside ONE CTA per tile: the
+    choice may change with the batch (table variants 3 and 4; by default the cluster while the grid fits one wave), the
+    bits may not.  Both against the oracle, and against each other bit for bit, at batches on both sides of the default
+    switch-over."""
+    H, W, cin, cout, k, stride, pad, act, residual, ranges = geom
+    max_batch = 40
+    spec = util.single_layer_model("bf16", H, W, cin, cout, k, stride, pad, act, residual, seed=hash(geom) % 1000, max_batch=max_batch)
+    layer = 1 if residual else 0
+    m = eb.EEModel(spec)
+    m.set_layer_splits(0, layer, ranges)
+    ws, ws_guard = util.guarded((m.query(0)["workspace_bytes"],), torch.uint8)
+    for B in (1, 6, 40):
+        x = wl.random_features((B, H, W, cin), seed=B, bf16=True, relu=False)
+        outs = eo.run_layers(spec, 0, x, keep_all=True)
+        res = eb.to_device("bf16", outs[0]) if residual else None
+        got = {}
+        for variant in (3, 4, 0, 4):
+            m.set_layer_variant(0, layer, 1, max_batch, variant)
+            out, guard = util.guarded(outs[layer].shape, torch.bfloat16)
+            m.layer_run(0, layer, eb.to_device("bf16", x), res, B, out, ws)
+            torch.cuda.synchronize()
+            m.check()
+            assert bool(torch.all(guard == util.CANARY)) and bool(torch.all(ws_guard == util.CANARY))
+            if variant in got:
+                assert torch.equal(out, got[variant])
+            got[variant] = out.clone()
+        assert torch.equal(got[3], got[4]) and torch.equal(got[0], got[3]), f"{geom} B={B}"
+        e = util.rel_err(got[4].float().cpu().numpy(), outs[layer], "bf16")
+        assert e <= util.TOL["bf16"], f"{geom} B={B}: {e:.3e}"
+
+
 @pytest.mark.parametrize("geom", HALO_GEOMS)
 def test_conv3x3_halo_layer(geom):
     H, W, cin, cout, act = geom
