@@ -922,6 +922,47 @@ def test_stem_with_the_pool_in_its_epilogue_equals_the_two_layers_run_apart(case
     assert util.rel_err(apart.float().cpu().numpy(), want, "bf16") <= util.TOL["bf16"]
 
 
+PROJ_BLOCKS = [  # H, W, cin, mid, cout, stride, act of the projection: 64-wide tiles, ragged channels, stride 2, an activation on the shortcut
+    (16, 16, 40, 48, 64, 1, wl.ACT_NONE), (16, 16, 64, 64, 136, 2, wl.ACT_NONE), (12, 20, 72, 40, 256, 2, wl.ACT_RELU),
+    (9, 9, 264, 64, 72, 1, wl.ACT_RELU6)]
+
+
+@pytest.mark.parametrize("blk", PROJ_BLOCKS)
+def test_projection_block_shapes_against_the_oracle_and_their_own_launches(blk):
+    """One block `1x1 -> 3x3 (stride) -> [1x1 projection of the input] -> 1x1 + projection` per case: the launch that
+    absorbs the projection against the oracle, and bit for bit against the layers launched one by one."""
+    H, W, cin, mid, cout, stride, pact = blk
+    rng = wl._rng(17, H, cin, cout)
+    layers = [wl._conv(rng, wl.OP_CONV, cin, mid, 1, 1, 0, wl.ACT_RELU, bf16=True, input_from=wl.FROM_STAGE_INPUT),
+              wl._conv(rng, wl.OP_CONV, mid, mid, 3, stride, 1, wl.ACT_RELU, bf16=True),
+              wl._conv(rng, wl.OP_CONV, cin, cout, 1, stride, 0, pact, gamma=0.7, bf16=True, input_from=wl.FROM_STAGE_INPUT),
+              wl._conv(rng, wl.OP_CONV, mid, cout, 1, 1, 0, wl.ACT_RELU, gamma=0.3, bf16=True, input_from=1, residual_from=2)]
+    fw, fb = wl._head(rng, cout, 5, 1.0, True)
+    spec = wl.Model("proj_block", "bf16", H, W, cin, [wl.Stage(layers, 5, fw, fb, 2.0, False)], 9)
+    run = util.GpuRunner(spec)
+    m, ws, out = run.m, run.ws, run.bufs[0]
+    for B in (1, 9):
+        assert [pl["launches"] for pl in m.plan(0, B)] == [1, 1, 0, 1]
+        x = wl.make_input(spec, B, seed=B)
+        xd = eb.to_device("bf16", x)
+        snaps = []
+        for fused in (True, False, True):
+            m.set_proj_fusion(fused)
+            out.features_out.fill_(0)
+            m.stage_run(0, xd, B, out, ws)
+            torch.cuda.synchronize()
+            m.check()
+            assert int(out.n_surv_host[0]) == B
+            snaps.append(out.features_out[:B].clone())
+        assert torch.equal(snaps[0], snaps[1]) and torch.equal(snaps[0], snaps[2])
+        want = eo.run_layers(spec, 0, x)
+        got = snaps[0].float().cpu().numpy()
+        # a chain of four bf16 layers: max-norm and L2 bars, and a bounded share of elements beyond 1e-2 (tests/util.py)
+        assert util.norm_err(got, want) <= util.STAGE_TOL["bf16"] and util.l2_err(got, want) <= util.STAGE_L2["bf16"], f"{blk} B={B}"
+        assert util.exceed_share(got, want, util.TOL["bf16"], util.STAGE_FLOOR) <= util.STAGE_EXCEED, f"{blk} B={B}"
+    run.check_guards()
+
+
 @pytest.mark.parametrize("B", [26, 9])
 def test_projection_inside_the_adding_layer_is_bit_identical_to_its_own_launch(B):
     """The projection shortcut of a stage's first block computed inside the launch of the layer that adds it (the
