@@ -955,6 +955,15 @@ def test_projection_block_shapes_against_the_oracle_and_their_own_launches(blk):
             assert int(out.n_surv_host[0]) == B
             snaps.append(out.features_out[:B].clone())
         assert torch.equal(snaps[0], snaps[1]) and torch.equal(snaps[0], snaps[2])
+        # the absorbing layer is also the stage's last one: its epilogue pools in row blocks where Ho * Wo has blocks of 32 rows
+        ho, wo = (H - 1) // stride + 1, (W - 1) // stride + 1
+        assert m.gap_partials(0, B) == (32 if (ho * wo) % 32 == 0 else 0)
+        z_on = out.logits[:B].clone()
+        m.set_gap_fusion(False)
+        m.stage_run(0, xd, B, out, ws)
+        torch.cuda.synchronize()
+        assert m.gap_partials(0, B) == 0 and torch.equal(out.logits[:B], z_on)
+        m.set_gap_fusion(True)
         want = eo.run_layers(spec, 0, x)
         got = snaps[0].float().cpu().numpy()
         # a chain of four bf16 layers: max-norm and L2 bars, and a bounded share of elements beyond 1e-2 (tests/util.py)
