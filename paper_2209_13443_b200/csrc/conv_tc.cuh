@@ -411,7 +411,7 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src
 // are contiguous in the NHWC input, then zeros; the weights are packed the same way.  While the main loop runs, the
 // four epilogue warps (one thread per tile row) read their pixel's taps and write them into the ring slot at the
 // position the 128-byte swizzle expects; the Toeplitz matrix still never touches global memory.
-template <int BN, int STAGES, bool RES, bool SPLIT, bool GATHER>
+template <int BN, int STAGES, bool RES, bool SPLIT, bool GATHER, bool LOCAL = false>   // LOCAL: TcParams::ranges accumulators in this CTA
 __global__ void __launch_bounds__(kTcThreads, 2)
 conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                           const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmO, TcParams p) {
@@ -455,9 +455,11 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmO) : "memory");
     if (RES) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmR) : "memory");
   }
-  const int n_acc = SPLIT ? 1 : max(p.ranges, 1);   // accumulators of BN fp32 columns
+  static_assert(!LOCAL || (!SPLIT && !GATHER), "local K ranges are a mode of the plain one-CTA kernel");
+  const int n_acc = LOCAL ? max(p.ranges, 1) : 1;   // accumulators of BN fp32 columns
   uint32_t acc_cols = BN;                           // TMEM allocations are powers of two
-  while ((int)acc_cols < n_acc * BN) acc_cols *= 2;
+  if (LOCAL)
+    while ((int)acc_cols < n_acc * BN) acc_cols *= 2;
   if (warp == 1) {  // TMEM: acc_cols fp32 columns x 128 lanes
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(acc_cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -531,7 +533,7 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
         if (!ok) break;
         tc_fence_after();
         const uint32_t sa = base + (uint32_t)s * S::kStage, sb = sa + S::kABytes;
-        const int r = n_acc > 1 ? i / p.kb_per : 0, ir = i - r * p.kb_per;   // local K range and position inside it
+        const int r = LOCAL ? i / p.kb_per : 0, ir = i - r * p.kb_per;   // local K range and position inside it
 #pragma unroll
         for (int k = 0; k < kTcBK / 16; ++k)
           umma_bf16(tmem_base + (uint32_t)(r * BN), umma_desc(sa + k * 32), umma_desc(sb + k * 32), idesc, (uint32_t)((ir | k) != 0));
@@ -622,7 +624,7 @@ conv_igemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
           const int c0 = h * 64 + sub * 32;
           float v[32];
           tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
-          if (n_acc > 1) {   // local K ranges: 0 + range 0 + range 1 + ... as the cluster reduction adds them
+          if constexpr (LOCAL) {   // local K ranges: 0 + range 0 + range 1 + ... as the cluster reduction adds them
 #pragma unroll
             for (int e = 0; e < 32; ++e) v[e] = 0.f + v[e];
             for (int r = 1; r < n_acc; ++r) {
@@ -1163,6 +1165,14 @@ inline ee_status_t tc_context_init(TcContext& c) {
   set(conv_igemm_tcgen05_kernel<128, 5, true, false, false>, TcSmem<128, 5, true>::kBytes);
   set(conv_igemm_tcgen05_kernel<128, 6, false, true, false>, TcSmem<128, 6, false>::kBytes);
   set(conv_igemm_tcgen05_kernel<128, 3, false, true, false>, TcSmem<128, 3, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 3, false, false, false, true>, TcSmem<64, 3, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 6, false, false, false, true>, TcSmem<64, 6, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 2, true, false, false, true>, TcSmem<64, 2, true>::kBytes);
+  set(conv_igemm_tcgen05_kernel<64, 5, true, false, false, true>, TcSmem<64, 5, true>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 3, false, false, false, true>, TcSmem<128, 3, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 6, false, false, false, true>, TcSmem<128, 6, false>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 2, true, false, false, true>, TcSmem<128, 2, true>::kBytes);
+  set(conv_igemm_tcgen05_kernel<128, 5, true, false, false, true>, TcSmem<128, 5, true>::kBytes);
   set(conv_igemm_tcgen05_persistent_kernel<64, false>, TcPersistSmem<64, false>::kBytes);
   set(conv_igemm_tcgen05_persistent_kernel<64, true>, TcPersistSmem<64, true>::kBytes);
   set(conv_igemm_tcgen05_persistent_kernel<128, false>, TcPersistSmem<128, false>::kBytes);
@@ -1334,7 +1344,7 @@ inline ee_status_t tc_buffer_map(const TcContext& c, const TcLayer& L, const voi
   return EE_OK;
 }
 
-template <int BN, int STAGES, bool RES, bool SPLIT, bool GATHER = false>
+template <int BN, int STAGES, bool RES, bool SPLIT, bool GATHER = false, bool LOCAL = false>
 inline cudaError_t tc_launch_t(dim3 grid, cudaStream_t st, const CUtensorMap& a, const CUtensorMap& w, const CUtensorMap& r,
                                const CUtensorMap& o, const TcParams& p) {
   cudaLaunchConfig_t cfg = {};
@@ -1354,12 +1364,16 @@ inline cudaError_t tc_launch_t(dim3 grid, cudaStream_t st, const CUtensorMap& a,
     attr[1].val.clusterDim.z = grid.z;
     cfg.numAttrs = 2;
   }
-  return cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_kernel<BN, STAGES, RES, SPLIT, GATHER>, a, w, r, o, p);
+  return cudaLaunchKernelEx(&cfg, conv_igemm_tcgen05_kernel<BN, STAGES, RES, SPLIT, GATHER, LOCAL>, a, w, r, o, p);
 }
 
 template <int BN>
 inline cudaError_t tc_launch_bn(bool deep, bool res, bool split, dim3 grid, cudaStream_t st, const CUtensorMap& a, const CUtensorMap& w,
                                 const CUtensorMap& r, const CUtensorMap& o, const TcParams& p) {
+  if (p.ranges > 1) {   // one CTA per tile with an accumulator per K range
+    if (res) return deep ? tc_launch_t<BN, 5, true, false, false, true>(grid, st, a, w, r, o, p) : tc_launch_t<BN, 2, true, false, false, true>(grid, st, a, w, r, o, p);
+    return deep ? tc_launch_t<BN, 6, false, false, false, true>(grid, st, a, w, r, o, p) : tc_launch_t<BN, 3, false, false, false, true>(grid, st, a, w, r, o, p);
+  }
   if (split) return deep ? tc_launch_t<BN, 6, false, true>(grid, st, a, w, r, o, p) : tc_launch_t<BN, 3, false, true>(grid, st, a, w, r, o, p);
   if (res) return deep ? tc_launch_t<BN, 5, true, false>(grid, st, a, w, r, o, p) : tc_launch_t<BN, 2, true, false>(grid, st, a, w, r, o, p);
   return deep ? tc_launch_t<BN, 6, false, false>(grid, st, a, w, r, o, p) : tc_launch_t<BN, 3, false, false>(grid, st, a, w, r, o, p);
