@@ -34,8 +34,8 @@ if ROOT not in sys.path:
 # DRAM bytes (read + written) per launch of the tensor-core conv kernels, from one ncu capture of the default workload
 # (ResNet-50-shaped, B=64, calibrated exits: 52 launches per pass, 1735.2 MB).  Reported only for that workload; it
 # has to be taken again (or set to None) whenever one of those kernels changes.
-NCU_CONV_TRAFFIC_PER_LAUNCH = {("resnet50", 64): 31.70e6}
-NCU_CONV_TRAFFIC_WARM_L2 = {("resnet50", 64): 23.78e6}   # same capture with --cache-control none
+NCU_CONV_TRAFFIC_PER_LAUNCH = {("resnet50", 64): 31.71e6}
+NCU_CONV_TRAFFIC_WARM_L2 = {("resnet50", 64): 23.72e6}   # same capture with --cache-control none
 
 METRIC = "EE-CNN samples/sec on 1 B200 vs exit rate & batch 1-64; tensor-pipe % of peak"
 UNIT = "samples/s"
